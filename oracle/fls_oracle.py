@@ -1,0 +1,325 @@
+"""CPU oracle for the FL+FSDP / FL+HSDP sync step and FedAvg.  TEST INFRASTRUCTURE ONLY.
+
+This file is the slow, plain definition that the CUDA library is checked against.
+It is numpy in float64, shares no code with the CUDA path and must never be
+imported by it: only the tests, the smoke check and the benchmark's CPU-baseline
+leg may call it.
+
+What the paper fixes and what it leaves open
+--------------------------------------------
+The paper defines the communication pattern, not the arithmetic:
+  * FSDP: every layer is split equally in S shards; the backward pass
+    reduce-scatters the gradients over the S ranks (Background, "Fully Sharded
+    Data Parallelism").
+  * HSDP: R x S mesh; reduce-scatter inside each sharding group, then an
+    all-reduce of corresponding gradient shards across the R replicas
+    (Background, "Hybrid Sharded Data Parallelism"; Section "HSDP" before Eq. 2).
+  * FL+FSDP / FL+HSDP: F federation groups with the same sharding policy train
+    independently and every A steps each shard is replaced by the (weighted)
+    average of the corresponding shards of all groups (Section "Augmenting
+    Sharded DP Through FL"; FedAvg as described in Background, "Federated
+    Learning").
+  * Optimiser: "AdamW, learning rate 3e-4", bf16 training (Experimental Setup).
+  * Cost model: Table of symbols and Eq. 1-5.
+Everything numeric that the paper does not state (mean vs sum, order, clipping
+rule, AdamW variant, rounding) follows the readings listed beside each function.
+
+Coordinates.  The oracle works on LOGICAL vectors: the P parameters of all units
+concatenated, unit after unit.  `plan()` and `pack_*`/`unpack_*` translate
+between logical vectors and the two physical orders of the flat buffers.
+Symbols: G groups (paper F), S shards, R_rep replicas (paper R), K = S*R_rep
+gradient buffers per group, H sync period (paper A).
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass, field
+from typing import List, Optional, Sequence
+
+import numpy as np
+
+CLIP_EPS = 1e-6  # added to the norm in the clip coefficient (reading: the common global-norm convention)
+
+
+# --------------------------------------------------------------------------- bf16 <-> values
+def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
+    """Exact value of bf16 bit patterns (uint16): a bf16 is the top half of an fp32."""
+    b = np.asarray(bits, dtype=np.uint16).astype(np.uint32) << np.uint32(16)
+    return b.view(np.float32).astype(np.float64)
+
+
+def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    """Round stored fp32 values to bf16, nearest-even on the 16 dropped bits; NaN stays NaN."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    u = x.view(np.uint32).astype(np.uint64)
+    keep_lsb = (u >> np.uint64(16)) & np.uint64(1)
+    rounded = (u + np.uint64(0x7FFF) + keep_lsb) >> np.uint64(16)
+    out = rounded.astype(np.uint16)
+    nan = np.isnan(x)
+    if nan.any():
+        out = np.where(nan, ((u >> np.uint64(16)) | np.uint64(0x0040)).astype(np.uint16), out)
+    return out
+
+
+# --------------------------------------------------------------------------- layout planner
+@dataclass
+class Layout:
+    """Flat-buffer layout of one group (identical for every group: the paper's
+    alignment constraint, Section "Augmenting Sharded DP Through FL")."""
+    unit_numel: List[int]          # n_u
+    S: int
+    Q: int
+    unit_shard_numel: List[int]    # M_u
+    unit_padded: List[int]         # n'_u = S*M_u
+    unit_offset: List[int]         # off_u  in the unsharded order (gradients, bf16 copy)
+    unit_shard_offset: List[int]   # soff_u inside one rank's shard buffer
+    n_params: int
+    n_padded: int
+    shard_numel: int
+    _addr_unsharded: Optional[np.ndarray] = field(default=None, repr=False)
+    _addr_sharded: Optional[np.ndarray] = field(default=None, repr=False)
+
+
+def plan(unit_numel: Sequence[int], S: int, Q: int = 1) -> Layout:
+    """Each unit ("layer") is split equally over S ranks in shards of size M_u
+    (Background, FSDP).  Reading for indivisible sizes: zero-pad the unit to
+    S*M_u with M_u = roundup(ceil(n_u/S), Q)."""
+    assert S >= 1 and Q >= 1 and len(unit_numel) >= 1
+    M, padded, off, soff = [], [], [], []
+    o = so = 0
+    for n in unit_numel:
+        assert n >= 1
+        per = -(-n // S)
+        m = -(-per // Q) * Q
+        M.append(m); padded.append(S * m); off.append(o); soff.append(so)
+        o += S * m; so += m
+    return Layout(list(unit_numel), S, Q, M, padded, off, soff, int(sum(unit_numel)), o, so)
+
+
+def _addresses(L: Layout):
+    """For every logical element: its index in the unsharded order and its address
+    in the rank-major shard order [S][shard_numel]."""
+    if L._addr_unsharded is None:
+        ju, ja = [], []
+        for u, n in enumerate(L.unit_numel):
+            i = np.arange(n, dtype=np.int64)
+            ju.append(L.unit_offset[u] + i)
+            s = i // L.unit_shard_numel[u]
+            k = L.unit_shard_offset[u] + i % L.unit_shard_numel[u]
+            ja.append(s * L.shard_numel + k)
+        L._addr_unsharded = np.concatenate(ju)
+        L._addr_sharded = np.concatenate(ja)
+    return L._addr_unsharded, L._addr_sharded
+
+
+def pack_unsharded(L: Layout, logical: np.ndarray) -> np.ndarray:
+    """Logical vector -> padded buffer in unsharded order (what backward produces /
+    the all-gather result).  Padding is zero."""
+    out = np.zeros(L.n_padded, dtype=logical.dtype)
+    out[_addresses(L)[0]] = logical
+    return out
+
+
+def pack_sharded(L: Layout, logical: np.ndarray) -> np.ndarray:
+    """Logical vector -> padded buffer in shard order: rank s holds, for every unit
+    in turn, elements [s*M_u, (s+1)*M_u) of that unit."""
+    out = np.zeros(L.n_padded, dtype=logical.dtype)
+    out[_addresses(L)[1]] = logical
+    return out
+
+
+def unpack_unsharded(L: Layout, buf: np.ndarray) -> np.ndarray:
+    return np.asarray(buf)[_addresses(L)[0]]
+
+
+def unpack_sharded(L: Layout, buf: np.ndarray) -> np.ndarray:
+    return np.asarray(buf)[_addresses(L)[1]]
+
+
+# --------------------------------------------------------------------------- one local step
+def reduce_mean(grads: Sequence[np.ndarray], S: int, R_rep: int = 1) -> np.ndarray:
+    """Mean gradient of one group, stored as fp32.
+
+    grads: K = R_rep*S float64 arrays (exact input values), buffer rho*S+sigma.
+    FSDP (R_rep = 1): the reduce-scatter sums the S rank gradients.
+    HSDP: first the reduce-scatter inside each sharding group (over sigma), then
+    the all-reduce across the R_rep replicas (over rho) -- shard level first,
+    replicate level second.  Reading: the reduction is a mean (sum, then one
+    division by K after the last level), kept in fp32 afterwards.
+    """
+    K = len(grads)
+    assert K == S * R_rep and K >= 1
+    outer = None
+    for rho in range(R_rep):
+        inner = None
+        for sigma in range(S):
+            x = np.asarray(grads[rho * S + sigma], dtype=np.float64)
+            inner = x.copy() if inner is None else inner + x
+        outer = inner if outer is None else outer + inner
+    return (outer / K).astype(np.float32)
+
+
+def grad_norm(gbar: np.ndarray) -> float:
+    """L2 norm of the whole group's mean gradient (all units together), in double."""
+    total = 0.0
+    g = np.asarray(gbar, dtype=np.float32)
+    for lo in range(0, g.size, 1 << 20):
+        c = g[lo:lo + (1 << 20)].astype(np.float64)
+        total += float(np.dot(c, c))
+    return math.sqrt(total)
+
+
+def clip_coef(norm: float, max_grad_norm: float) -> float:
+    """Global-norm clipping (the paper never mentions clipping; reading: scale the
+    mean gradient by min(1, clip/(norm+1e-6)); clip <= 0 disables it)."""
+    if not (max_grad_norm > 0.0):
+        return 1.0
+    c = max_grad_norm / (norm + CLIP_EPS)
+    if math.isnan(c):
+        return c                     # non-finite norms propagate, nothing is special-cased
+    return c if c < 1.0 else 1.0
+
+
+def adamw(theta, m, v, gbar, coef, t_new, lr, beta1, beta2, eps, weight_decay):
+    """AdamW on stored fp32 state, double arithmetic, fp32 stores (Experimental
+    Setup names only "AdamW"; reading: decoupled weight decay applied to theta
+    first, bias-corrected moments, eps added outside the square root)."""
+    th = np.asarray(theta, dtype=np.float32).astype(np.float64)
+    m_ = np.asarray(m, dtype=np.float32).astype(np.float64)
+    v_ = np.asarray(v, dtype=np.float32).astype(np.float64)
+    g = coef * np.asarray(gbar, dtype=np.float32).astype(np.float64)
+    th = th * (1.0 - lr * weight_decay)
+    m_ = beta1 * m_ + (1.0 - beta1) * g
+    v_ = beta2 * v_ + (1.0 - beta2) * g * g
+    mhat = m_ / (1.0 - beta1 ** t_new)
+    vhat = v_ / (1.0 - beta2 ** t_new)
+    th = th - lr * mhat / (np.sqrt(vhat) + eps)
+    th32 = th.astype(np.float32)
+    return th32, m_.astype(np.float32), v_.astype(np.float32), f32_to_bf16_bits(th32)
+
+
+@dataclass
+class GroupState:
+    """Logical fp32 state of one federation group plus its bf16 parameter copy."""
+    theta: np.ndarray
+    m: np.ndarray
+    v: np.ndarray
+    param_bf16: np.ndarray      # uint16 bit patterns
+
+
+@dataclass
+class Hyper:
+    lr: float = 3e-4
+    beta1: float = 0.9
+    beta2: float = 0.95
+    eps: float = 1e-8
+    weight_decay: float = 0.1
+    max_grad_norm: float = 1.0
+
+
+def sync_step_group(st: GroupState, grads: Sequence[np.ndarray], S: int, R_rep: int, t_new: int,
+                    hp: Hyper, lr: Optional[float] = None):
+    """One local step of one group: reduce -> norm -> clip -> AdamW.  Returns
+    (norm, coef, gbar).  Each group "proceeds independently of the others"
+    (Section FL+FSDP)."""
+    gbar = reduce_mean(grads, S, R_rep)
+    nrm = grad_norm(gbar)
+    c = clip_coef(nrm, hp.max_grad_norm)
+    st.theta, st.m, st.v, st.param_bf16 = adamw(
+        st.theta, st.m, st.v, gbar, c, t_new, hp.lr if lr is None else lr,
+        hp.beta1, hp.beta2, hp.eps, hp.weight_decay)
+    return nrm, c, gbar
+
+
+# --------------------------------------------------------------------------- FedAvg
+def fedavg_weights(sample_counts: Optional[Sequence[int]], G: int) -> np.ndarray:
+    if sample_counts is None:
+        sample_counts = [1] * G
+    n = np.asarray(sample_counts, dtype=np.float64)
+    assert n.size == G and (n >= 0).all() and n.sum() > 0
+    return n / n.sum()
+
+
+def fedavg_array(copies: Sequence[np.ndarray], w: np.ndarray) -> np.ndarray:
+    """Weighted average of G corresponding copies, double accumulate in ascending
+    group order, stored as fp32 (FedAvg: "a weighted average of all locally trained
+    models"; shard by shard over the F groups)."""
+    acc = None
+    for g, x in enumerate(copies):
+        term = w[g] * np.asarray(x, dtype=np.float32).astype(np.float64)
+        acc = term if acc is None else acc + term
+    return acc.astype(np.float32)
+
+
+def fedavg(states: Sequence[GroupState], sample_counts: Optional[Sequence[int]] = None,
+           opt_state: bool = False) -> None:
+    """After aggregation "every shard is equal to the average of its corresponding
+    shards in all the other federation groups": every group receives the same
+    averaged parameters (and the bf16 copy of them).  Reading: w_g = n_g / sum n;
+    m and v are averaged the same way only when `opt_state` is set."""
+    G = len(states)
+    w = fedavg_weights(sample_counts, G)
+    th = fedavg_array([s.theta for s in states], w)
+    bits = f32_to_bf16_bits(th)
+    if opt_state:
+        m = fedavg_array([s.m for s in states], w)
+        v = fedavg_array([s.v for s in states], w)
+    for s in states:
+        s.theta = th.copy(); s.param_bf16 = bits.copy()
+        if opt_state:
+            s.m = m.copy(); s.v = v.copy()
+
+
+# --------------------------------------------------------------------------- driver loop
+def run(states: List[GroupState], grads_for_step, S: int, R_rep: int, H: int, n_steps: int, hp: Hyper,
+        sample_counts=None, opt_state: bool = False, t0: int = 0):
+    """for step: every group takes one local step; after every H-th step FedAvg
+    ("every A training steps", "after the local update").  grads_for_step(step, g)
+    returns that group's K float64 gradient arrays (logical).  The step counter
+    is global and is not reset by FedAvg.  Returns the per-step list of norms."""
+    norms = []
+    t = t0
+    for _ in range(n_steps):
+        t += 1
+        row = []
+        for g, st in enumerate(states):
+            nrm, _, _ = sync_step_group(st, grads_for_step(t, g), S, R_rep, t, hp)
+            row.append(nrm)
+        norms.append(row)
+        if t % H == 0:
+            fedavg(states, sample_counts, opt_state)
+    return norms
+
+
+# --------------------------------------------------------------------------- communication-cost model
+def cost_all_gather(D, n, B=1.0):
+    return D * (n - 1) / (n * B)
+
+
+def cost_reduce_scatter(D, n, B=1.0):
+    return D * (n - 1) / (n * B)
+
+
+def cost_all_reduce(D, n, B=1.0):
+    return 2.0 * D * (n - 1) / (n * B)
+
+
+def cost_broadcast(D, n, B=1.0):
+    return D / B
+
+
+def comm_costs(unit_shard_bytes: Sequence[float], S: int, R: int, F: int, A: int,
+               B_S: float = 1.0, B_R: float = 1.0, B_F: float = 1.0) -> dict:
+    """Eq. 1-5 written as the sums of collectives they are defined by (the left-hand
+    forms), with the uniform M*L replaced by a sum over units.  With all
+    bandwidths 1 the values are bytes per step; with real bandwidths, seconds.
+    FL+HSDP with R = 1 "falls back to FL+FSDP" (Section FL+HSDP)."""
+    fsdp = hsdp = fl = bc = 0.0
+    for M in unit_shard_bytes:
+        f = 2 * cost_all_gather(M, S, B_S) + cost_reduce_scatter(M, S, B_S)
+        fsdp += f
+        hsdp += f + cost_all_reduce(M, R, B_R)
+        fl += cost_all_reduce(M, F, B_F) / A
+        bc += cost_broadcast(M, R, B_R) / A
+    fl_hsdp = hsdp + fl + bc if R > 1 else fsdp + fl
+    return dict(fsdp=fsdp, hsdp=hsdp, fl=fl, fl_fsdp=fsdp + fl, fl_hsdp=fl_hsdp)
