@@ -1,0 +1,306 @@
+#!/usr/bin/env python
+"""Benchmark of the sync step (+ FedAvg every H-th step) on synthetic buffers.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl ours|reference]
+
+A step is one fls_sync_step over all G groups, followed by fls_fedavg when the step counter is a
+multiple of H.  Metric: synced params/s = G*P*K / time (logical parameters, whole job).  Prints one
+JSON line on rank 0.  With N > 1 every rank runs an independent replica of the workload (the path has
+no inter-GPU exchange); the time is the maximum over ranks.
+`--impl reference` times the CPU oracle on a bounded sample of the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+import synthetic as sy
+
+METRIC = "synced_params_per_s"
+UNIT = "params/s"
+DEFAULT_CONFIG = "gpt2_small_fl_fsdp"
+# DRAM bytes per launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
+# dram__bytes_write.sum), per config; None until a capture of that workload exists under profiles/.
+NCU_TRAFFIC_BYTES = {}
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        return float(json.load(open(path))["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+# --------------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except Exception:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------------------- CPU oracle leg
+def oracle_sample(cfg: dict, sample_params: int):
+    """One oracle step of all G groups (+ FedAvg/H) on the first `sample_params` parameters.
+    Returns (params/s, seconds, threads)."""
+    from oracle import fls_oracle as orc
+    G, S, R = cfg["groups"], cfg["shard_dim"], cfg["replicate_dim"]
+    K = S * R
+    P = min(sample_params, cfg["n_params"])
+    hp = orc.Hyper(cfg["lr"], cfg["beta1"], cfg["beta2"], cfg["eps"], cfg["weight_decay"], cfg["max_grad_norm"])
+    th0 = sy.normal_fill_(torch.empty(P), sy.stream_key(cfg["seed"], sy.KIND_MASTER), cfg["master_sigma"]).numpy()
+    states = [orc.GroupState(th0.copy(), np.zeros(P, np.float32), np.zeros(P, np.float32), None) for _ in range(G)]
+    bits = [[sy.normal_fill_(torch.empty(P, dtype=torch.bfloat16), sy.stream_key(cfg["seed"], sy.KIND_GRAD, 1, g, k), cfg["grad_sigma"])
+             .view(torch.int16).numpy().view(np.uint16) for k in range(K)] for g in range(G)]
+    t0 = time.perf_counter()
+    for g in range(G):
+        grads = [orc.bf16_bits_to_f64(b) for b in bits[g]]
+        orc.sync_step_group(states[g], grads, S, R, 1, hp)
+    t_step = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    orc.fedavg(states, [sy.sample_count(cfg["seed"], g) for g in range(G)] if cfg["weights"] == "counts" else None)
+    t_avg = time.perf_counter() - t0
+    sec = t_step + t_avg / cfg["sync_period"]
+    return G * P / sec, t_step + t_avg, 1
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    sample = 1 << 22
+    vals, secs = [], []
+    for _ in range(args.warmup and 1):
+        oracle_sample(cfg, 1 << 18)
+    for _ in range(max(1, min(args.steps, 3))):
+        v, s, cores = oracle_sample(cfg, sample)
+        vals.append(v); secs.append(s)
+    value = float(np.mean(vals))
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": len(vals),
+            "warmup": 1 if args.warmup else 0, "ms_per_step": 1e3 * float(np.mean(secs)), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg["name"], "sample": f"first {sample} params of each of {cfg['groups']} groups"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
+                             "sample": f"one oracle step (+FedAvg/H) on the first {sample} params of each group"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------------------- GPU leg
+def fill_session(sess, cfg):
+    th_key = sy.stream_key(cfg["seed"], sy.KIND_MASTER)
+    for g in range(cfg["groups"]):
+        sy.normal_fill_(sess.master[g], th_key, cfg["master_sigma"])
+        sess.param_bf16[g].copy_(sess.master[g])
+        for k in range(sess.K):
+            scale = sy.uniform_scale(cfg["seed"], g, k) if cfg["per_buffer_scale"] else 1.0
+            sy.normal_fill_(sess.grads[g][k], sy.stream_key(cfg["seed"], sy.KIND_GRAD, 1, g, k), cfg["grad_sigma"], scale)
+    torch.cuda.synchronize()
+
+
+def run_ours(args, cfg):
+    import torch.distributed as dist
+    from paper_2609_20359_b200 import build
+    from paper_2609_20359_b200 import _binding as fls
+    from paper_2609_20359_b200.session import Session
+
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path); use --impl reference for the oracle")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        build.build()
+    if world > 1:
+        dist.barrier()
+
+    G, P = cfg["groups"], cfg["n_params"]
+    counts = [sy.sample_count(cfg["seed"], g) for g in range(G)] if cfg["weights"] == "counts" else None
+    sess = Session(P, cfg["unit_numel"], G, cfg["shard_dim"], cfg["replicate_dim"], cfg["sync_period"], cfg["grad_dtype"], 8,
+                   args.opt_state, cfg["lr"], cfg["beta1"], cfg["beta2"], cfg["eps"], cfg["weight_decay"], cfg["max_grad_norm"],
+                   device=f"cuda:{local}")
+    for kern, val in (("reduce", args.ctas_reduce), ("adamw", args.ctas_adamw), ("fedavg", args.ctas_fedavg)):
+        if val:
+            fls.fls_plan_tune(sess.plan, {"reduce": 0, "adamw": 1, "fedavg": 2}[kern], val, -1)
+    if args.descending_adamw:
+        fls.fls_plan_tune(sess.plan, fls.FLS_KERNEL_ADAMW, 0, 1)
+    fill_session(sess, cfg)
+    stream = torch.cuda.current_stream()
+
+    def one_step():
+        if sess.step(stream=stream):
+            sess.fedavg(counts, stream=stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def timed(n_steps, profiling):
+        fls.fls_set_profiling(sess.plan, profiling)
+        barrier()
+        l0 = fls.fls_get_launch_count(sess.plan)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(n_steps):
+            one_step()
+        e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms, fls.fls_get_launch_count(sess.plan) - l0
+
+    for _ in range(args.warmup):
+        one_step()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    ms_total, launches = timed(args.steps, False)
+    clocks = sampler.stop() if rank == 0 else None
+    # second pass over the same number of steps with events around every kernel: per-kernel durations
+    ms_prof, _ = timed(args.steps, True)
+    kms, kn = fls.fls_get_kernel_ms(sess.plan)
+    fls.fls_set_profiling(sess.plan, False)
+
+    # end to end: gradients start in pinned host memory, norms come back to the host, every step
+    e2e = None
+    if not args.no_e2e:
+        host = [[torch.empty(sess.n_padded, dtype=sess.grad_torch_dtype).pin_memory() for _ in range(sess.K)] for _ in range(G)]
+        for g in range(G):
+            for k in range(sess.K):
+                host[g][k].copy_(sess.grads[g][k])
+        norms = torch.zeros(G, dtype=torch.float32).pin_memory()
+        def e2e_step():
+            if sess.step_host(host, stream=stream, host_norms=norms):
+                sess.fedavg(counts, stream=stream)
+                torch.cuda.synchronize()
+        e2e_step()
+        barrier()
+        t0 = time.perf_counter()
+        n_e2e = max(2, min(args.steps, 4))
+        for _ in range(n_e2e):
+            e2e_step()
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        if world > 1:
+            t = torch.tensor([dt], device="cuda"); dist.all_reduce(t, op=dist.ReduceOp.MAX); dt = float(t.item())
+        eg = 4 if cfg["grad_dtype"] == "f32" else 2
+        e2e = {"value": world * G * P * n_e2e / dt, "unit": UNIT, "h2d_bytes_per_step": G * sess.K * sess.n_padded * eg,
+               "d2h_bytes_per_step": 4 * G, "steps": n_e2e, "ms_per_step": 1e3 * dt / n_e2e}
+        del host
+
+    if rank == 0:
+        peak, peak_kind = measured_peak_gbs()
+        N = sess.n_padded
+        eg = 4 if cfg["grad_dtype"] == "f32" else 2
+        per_launch = {"reduce": N * (sess.K * eg + 4), "adamw": N * 30, "fedavg": N * G * 10}
+        kernels = {}
+        for i, name in enumerate(("reduce", "adamw", "fedavg")):
+            if kn[i]:
+                avg_ms = kms[i] / kn[i]
+                kernels[name] = {"launches": kn[i], "avg_ms": avg_ms, "bytes_per_launch": per_launch[name],
+                                 "gbs": per_launch[name] / avg_ms / 1e6, "frac": per_launch[name] / avg_ms / 1e6 / peak,
+                                 "share": kms[i] / sum(kms)}
+        dom = max(kernels, key=lambda n: kernels[n]["share"])
+        rep = fls.fls_comm_report(sess.plan)
+        step_bytes = rep["hbm_bytes_sync_step"] + rep["hbm_bytes_fedavg"] / cfg["sync_period"]
+        ms_step = ms_total / args.steps
+        line = {
+            "metric": METRIC, "value": world * G * P * args.steps / (ms_total / 1e3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": cfg["name"], "n_params": P, "groups": G, "shard_dim": cfg["shard_dim"],
+                       "replicate_dim": cfg["replicate_dim"], "sync_period": cfg["sync_period"], "grad_dtype": cfg["grad_dtype"],
+                       "fedavg_opt_state": bool(args.opt_state), "l2": "working set exceeds L2, no flush needed",
+                       "parallelism": "replicas only" if world > 1 else "1 gpu"},
+            "hbm_gbs": step_bytes / ms_step / 1e6, "hbm_frac_of_measured_peak": step_bytes / ms_step / 1e6 / peak,
+            "hbm_frac_of_8tbs": step_bytes / ms_step / 1e6 / 8000.0,
+            "roofline": {"bound": "hbm", "kernel": dom, "achieved": kernels[dom]["gbs"], "peak": peak, "peak_kind": peak_kind,
+                         "unit": "GB/s", "frac": kernels[dom]["frac"], "traffic": NCU_TRAFFIC_BYTES.get((cfg["name"], dom))},
+            "kernels": kernels, "ms_per_step_profiled": ms_prof / args.steps,
+            "gpu_launches": launches, "clocks": clocks, "e2e": e2e,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            v, s, cores = oracle_sample(cfg, 1 << 22)
+            line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "seconds": s,
+                                    "sample": f"one oracle step (+FedAvg/H) on the first {1 << 22} params of each of {G} groups"}
+        print(json.dumps(line), flush=True)
+    sess.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=16)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default=DEFAULT_CONFIG, choices=[c["name"] for c in sy.CONFIGS])
+    ap.add_argument("--opt-state", action="store_true", help="FedAvg also averages m and v")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--ctas-reduce", type=int, default=0)
+    ap.add_argument("--ctas-adamw", type=int, default=0)
+    ap.add_argument("--ctas-fedavg", type=int, default=0)
+    ap.add_argument("--descending-adamw", action="store_true")
+    args = ap.parse_args()
+    cfg = sy.config_by_name(args.config)
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

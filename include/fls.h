@@ -1,0 +1,201 @@
+/*
+ * fls.h -- C ABI of libfls: the data-parallel arithmetic of FL+FSDP / FL+HSDP on one B200.
+ *
+ * What the library computes (paper: "Accelerating Sharded Data Parallelism at Scale with
+ * Federated Learning"):
+ *   - F federation groups apply the same sharding policy and train independently
+ *     (Section "Augmenting Sharded DP Through FL").  Here: G groups, one layout for all.
+ *   - Inside a group, FSDP reduce-scatters the gradients of every layer over the S ranks
+ *     (Background, FSDP); HSDP does so inside each of R sharding groups and then
+ *     all-reduces corresponding gradient shards across the R replicas (Background, HSDP;
+ *     Section "HSDP", Eq. 2).  Here: K = S*R gradient buffers per group are read from
+ *     HBM and reduced in that order; the result feeds a global-norm clip and AdamW on the
+ *     group's fp32 master/m/v shards, and a bf16 parameter copy is written.
+ *   - Every A steps the corresponding shards of all groups are replaced by their weighted
+ *     average (FedAvg; Background "Federated Learning", Sections FL+FSDP and FL+HSDP).
+ *   - Eq. 1-5 and the table of collective costs give the communication cost of each
+ *     scheme; fls_comm_report evaluates them for a plan.
+ * Symbols: G = paper F (groups), H = paper A (aggregation period), S = shards,
+ * R_rep = paper R (replicas; 1 for FSDP), L units = the paper's L sharded layers.
+ *
+ * Conventions
+ *   - Every function returns 0 (FLS_OK) or an error code > 0 and never throws, aborts or
+ *     prints.  fls_last_error() gives the calling thread's last message.
+ *   - "host" / "device" beside a pointer says where the memory it points to lives.
+ *   - The caller owns every device buffer and the stream.  The library owns the plan, its
+ *     host tables, a few CUDA events and one internal copy stream; on the device it uses
+ *     only the caller's workspace.  It allocates no bulk device memory.
+ *   - Nothing synchronises the device except where stated (fls_plan_bind,
+ *     fls_sync_step_host, fls_get_kernel_ms).
+ *   - A plan is not thread-safe; use one plan per host thread or lock around it.
+ */
+#ifndef FLS_H_
+#define FLS_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct fls_plan fls_plan; /* opaque, created by fls_plan_create, freed by fls_plan_destroy */
+
+enum { FLS_OK = 0, FLS_EINVAL = 1, FLS_EALIGN = 2, FLS_EPTR = 3, FLS_ESIZE = 4, FLS_ECUDA = 5, FLS_ESTATE = 6 };
+enum { FLS_GRAD_BF16 = 0, FLS_GRAD_F32 = 1 };
+enum { FLS_AVG_PARAMS = 1, FLS_AVG_OPT_STATE = 2 }; /* fedavg_what bit mask */
+enum { FLS_KERNEL_REDUCE = 0, FLS_KERNEL_ADAMW = 1, FLS_KERNEL_FEDAVG = 2, FLS_KERNEL_COUNT = 3 };
+enum { FLS_STATUS_NONFINITE_NORM = 1 };             /* sticky bits of the device status word */
+
+#define FLS_MAX_GROUPS 64        /* G <= 64 */
+#define FLS_MAX_GRAD_BUFFERS 64  /* K = shard_dim * replicate_dim <= 64 */
+#define FLS_BUFFER_ALIGN 32      /* every device buffer must start on a 32-byte boundary */
+
+/* Problem statement.  One layout is shared by all groups (the paper's alignment constraint:
+ * shards of different federation groups must correspond one to one). */
+typedef struct {
+  uint64_t n_params;          /* logical parameter count P = sum of unit_numel                          */
+  uint32_t n_units;           /* L; 0 with unit_numel == NULL means one unit of n_params                */
+  const uint64_t* unit_numel; /* host, L entries, copied: the bucket / FSDP-unit ("layer") table        */
+  uint32_t groups;            /* G >= 1                                                                 */
+  uint32_t shard_dim;         /* S >= 1                                                                 */
+  uint32_t replicate_dim;     /* R_rep >= 1; 1 = FL+FSDP, > 1 = FL+HSDP (shard level reduced first)     */
+  uint32_t sync_period;       /* H >= 1: FedAvg is due after every H-th step                            */
+  uint32_t grad_dtype;        /* FLS_GRAD_BF16 or FLS_GRAD_F32                                          */
+  uint32_t align_elems;       /* Q >= 1: every unit's shard length is rounded up to a multiple of Q.
+                                 Q = 1 pads a unit to a multiple of S exactly; multiples of 8 keep every
+                                 shard on the vector path (otherwise element-wise loads are used)      */
+  uint32_t fedavg_what;       /* FLS_AVG_PARAMS, optionally | FLS_AVG_OPT_STATE (m and v averaged too)  */
+  uint32_t reserved;          /* must be 0                                                              */
+  double lr, beta1, beta2, eps, weight_decay;
+  double max_grad_norm;       /* <= 0 disables clipping (the norm is still computed)                    */
+} fls_plan_desc;
+
+/* Layout computed by the planner.  Arrays are owned by the plan and live as long as it does.
+ *   unit u is zero-padded to S*M_u elements, M_u = roundup(ceil(n_u/S), Q);
+ *   UNSHARDED order (gradient buffers, bf16 parameter copy): element i of unit u at unit_offset[u] + i;
+ *   SHARD order (master, m, v): rank s = i / M_u holds it at s*shard_numel + unit_shard_offset[u] + i % M_u.
+ * Padding elements must be zero in every buffer the caller fills; the library keeps them zero. */
+typedef struct {
+  uint64_t n_padded;                 /* N_pad = sum S*M_u: element count of EVERY buffer below          */
+  uint64_t shard_numel;              /* N_pad / S                                                       */
+  uint32_t n_units;
+  uint32_t grad_buffers;             /* K = S*R_rep per group                                           */
+  const uint64_t* unit_offset;       /* host, L entries                                                 */
+  const uint64_t* unit_shard_numel;  /* host, L entries: M_u                                            */
+  const uint64_t* unit_shard_offset; /* host, L entries                                                 */
+  uint64_t workspace_bytes;          /* size the caller must provide in fls_buffers.workspace           */
+  uint32_t n_segments;               /* contiguous (unit, shard) runs the kernels walk                  */
+  uint32_t vector_path;              /* 1 if every segment is 8-element aligned in both orders          */
+} fls_layout;
+
+/* Device buffers, all caller-owned, each N_pad elements, FLS_BUFFER_ALIGN-aligned, non-overlapping.
+ * The pointer ARRAYS are host memory and are copied by fls_plan_bind. */
+typedef struct {
+  const void* const* grads; /* host array of G*K device pointers, index g*K + rho*S + sigma; bf16 or fp32;
+                               unsharded order; read-only to the library, never cleared by it            */
+  float* const* master;     /* host array of G device pointers: fp32 parameters, shard order, in/out     */
+  float* const* m;          /* same: first moment                                                        */
+  float* const* v;          /* same: second moment                                                       */
+  void* const* param_bf16;  /* host array of G device pointers: bf16 copy, unsharded order, output       */
+  void* workspace;          /* device, >= workspace_bytes; holds the reduced gradient, the norm partials,
+                               per-group norm / clip coefficient, the status word and the segment table  */
+  uint64_t workspace_bytes;
+} fls_buffers;
+
+/* Communication cost of one training step, one value per equation of the paper. */
+typedef struct { double fsdp, hsdp, fl, fl_fsdp, fl_hsdp; } fls_cost5; /* Eq. 1, 2, 3, 4, 5 */
+typedef struct {
+  fls_cost5 paper_bytes; /* Eq. 1-5 as printed with the bandwidths taken out: message size D = M_u, the unit's
+                            shard in bytes of the gradient dtype, summed over units instead of M*L            */
+  fls_cost5 wire_bytes;  /* bytes one rank sends per step when D of all-gather / reduce-scatter is the whole
+                            unit (S*M_u), the convention of the NCCL performance notes the paper cites        */
+  fls_cost5 seconds;     /* Eq. 1-5 with B_S, B_R, B_F; NaN when no bandwidths were given                     */
+  double hbm_bytes_sync_step; /* bytes one fls_sync_step must move in this library: G*N_pad*(K*e_g + 34)      */
+  double hbm_bytes_fedavg;    /* bytes one fls_fedavg must move: G*N_pad*10, or *26 with optimizer state      */
+} fls_comm_costs;
+
+/* Layout planner + validation (flat-buffer layout: padding to the shard multiple, per-unit offsets).
+ * Host only: touches no GPU.  Errors: FLS_EINVAL for a null argument, G, S, R_rep, H or Q = 0, G or K
+ * above the maxima, sum(unit_numel) != n_params, a zero-length unit, beta outside [0,1), eps <= 0, lr < 0,
+ * an unknown dtype or fedavg_what without FLS_AVG_PARAMS.  On error *out is NULL. */
+int fls_plan_create(const fls_plan_desc* desc, fls_plan** out);
+
+/* Copies the layout summary into *out (host). */
+int fls_plan_query(const fls_plan* plan, fls_layout* out);
+
+/* Validates and records the caller's buffers, uploads the segment table into the workspace and clears
+ * the status word.  Uses the current CUDA device; synchronises it.  May be called again to rebind.
+ * Errors: FLS_EPTR (null, host or overlapping buffers), FLS_EALIGN, FLS_ESIZE (workspace too small),
+ * FLS_ECUDA. */
+int fls_plan_bind(fls_plan* plan, const fls_buffers* buffers);
+
+/* One local training step of all G groups ("each federation group proceeds independently"), enqueued
+ * on `cuda_stream` (a cudaStream_t; NULL = default stream).  Per group: mean of the K gradient buffers
+ * in fp32, ascending buffer order inside a sharding group, then ascending replica order (reduce-scatter
+ * over S, then all-reduce over R: Background FSDP/HSDP, Eq. 2), one multiply by 1/K; L2 norm of the mean
+ * gradient over the whole group; c = min(1, max_grad_norm/(norm + 1e-6)); AdamW with decoupled weight
+ * decay and bias correction on master/m/v in place; bf16 copy of the new parameters (round to nearest
+ * even).  `lr` overrides the plan's learning rate for this step; pass NaN to use the plan's.  The step
+ * counter t is incremented; *fedavg_due (host, may be NULL) is set to (t % H == 0).
+ * Errors: FLS_ESTATE if not bound, FLS_ECUDA on a launch failure (state is then undefined). */
+int fls_sync_step(fls_plan* plan, double lr, void* cuda_stream, int* fedavg_due);
+
+/* Same step with the gradients in HOST memory: host_grads is a host array of G*K host pointers (same
+ * order and size as fls_buffers.grads; pinned memory for full speed).  Each group's gradients are copied
+ * into the bound device gradient buffers on an internal stream while the previous group computes; after
+ * the last group the G norms are copied to host_norms (host, G floats, may be NULL) and the call waits
+ * for `cuda_stream`.  This is the end-to-end form of fls_sync_step. */
+int fls_sync_step_host(fls_plan* plan, const void* const* host_grads, double lr, void* cuda_stream,
+                       float* host_norms, int* fedavg_due);
+
+/* FedAvg: every group's parameters become sum_g w_g x_g, w_g = n_g / sum n ("a weighted average of all
+ * locally trained models"; shard by shard across the federation groups, after which every shard equals
+ * the average of its counterparts).  fp32 accumulation in ascending group order; all G master copies and
+ * all G bf16 copies are rewritten; m and v too if the plan has FLS_AVG_OPT_STATE.  sample_counts: host,
+ * G entries, NULL = equal weights.  The step counter is unchanged.
+ * Errors: FLS_EINVAL if all counts are zero, FLS_ESTATE, FLS_ECUDA. */
+int fls_fedavg(fls_plan* plan, const uint64_t* sample_counts, void* cuda_stream);
+
+/* Device pointers (inside the workspace) to G floats each: the gradient norm and the clip coefficient of
+ * the last step, valid once that step has completed on its stream.  Either output may be NULL. */
+int fls_get_norms(const fls_plan* plan, const float** dev_norms, const float** dev_coefs);
+
+/* Device pointer to the reduced (mean) gradient of the LAST group processed: N_pad floats, shard order. */
+int fls_get_reduced_grad(const fls_plan* plan, const float** dev_gbar);
+
+/* Device pointer to the sticky status word (FLS_STATUS_* bits).  Non-finite values are not errors:
+ * they propagate by IEEE rules and set a bit here. */
+int fls_get_status(const fls_plan* plan, const uint32_t** dev_status);
+
+/* Step counter t (starts at 0; the first step uses exponent 1 in the bias corrections).  fls_set_step
+ * resumes from a checkpoint: master/m/v are the caller's, t is the only other state. */
+int fls_get_step(const fls_plan* plan, uint64_t* t);
+int fls_set_step(fls_plan* plan, uint64_t t);
+
+/* Eq. 1-5 for this plan (L units, M_u, S, R = R_rep, F = G, A = H).  bw_bytes_per_s: host, {B_S, B_R, B_F}
+ * or NULL.  With R_rep = 1 the FL+HSDP entry equals the FL+FSDP one (the paper's fallback).  Host only. */
+int fls_comm_report(const fls_plan* plan, const double* bw_bytes_per_s, fls_comm_costs* out);
+
+/* Launch shape of one kernel (FLS_KERNEL_*): resident CTAs per SM used to size the persistent grid, and
+ * whether the kernel walks the tiles in descending order.  0 / negative keep the current value. */
+int fls_plan_tune(fls_plan* plan, uint32_t kernel, int ctas_per_sm, int descending);
+
+/* Per-kernel timing with CUDA events recorded on the caller's stream around every launch.
+ * fls_set_profiling(plan, 1) turns it on; fls_get_kernel_ms waits for the recorded events, adds their
+ * durations into ms[FLS_KERNEL_COUNT] / launches[FLS_KERNEL_COUNT] (host) and clears the record. */
+int fls_set_profiling(fls_plan* plan, int enabled);
+int fls_get_kernel_ms(fls_plan* plan, double* ms, uint64_t* launches);
+
+/* Number of kernels this plan has launched so far. */
+int fls_get_launch_count(const fls_plan* plan, uint64_t* launches);
+
+/* Frees the plan and its events/stream.  Device buffers are the caller's and are not touched. */
+int fls_plan_destroy(fls_plan* plan);
+
+/* Message of the last error on the calling thread ("" if none).  Host string owned by the library. */
+const char* fls_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FLS_H_ */

@@ -1,0 +1,21 @@
+"""libfls: the FL+FSDP / FL+HSDP sync step and FedAvg on one B200.
+
+Thin ctypes binding of the C ABI declared in include/fls.h.  Every step of the path runs in the
+CUDA library; this package only marshals arguments.  There is no CPU fallback: the first use of any
+fls_* name loads libfls.so and raises if it is missing (build it with
+`python -m paper_2609_20359_b200.build`).
+"""
+import importlib
+
+__all__ = ["build"]
+
+
+def __getattr__(name):
+    # loaded on first use so that `python -m paper_2609_20359_b200.build` can run before the library exists
+    if name.startswith("__"):
+        raise AttributeError(name)
+    binding = importlib.import_module("._binding", __name__)
+    try:
+        return getattr(binding, name)
+    except AttributeError:
+        raise AttributeError(f"module {__name__!r} has no attribute {name!r}") from None

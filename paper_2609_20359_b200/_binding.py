@@ -1,0 +1,251 @@
+"""ctypes binding of libfls.so: same names as the C ABI, argument marshalling only."""
+from __future__ import annotations
+
+import ctypes as C
+import math
+import os
+from typing import Optional, Sequence
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libfls.so")
+
+FLS_OK, FLS_EINVAL, FLS_EALIGN, FLS_EPTR, FLS_ESIZE, FLS_ECUDA, FLS_ESTATE = range(7)
+FLS_GRAD_BF16, FLS_GRAD_F32 = 0, 1
+FLS_AVG_PARAMS, FLS_AVG_OPT_STATE = 1, 2
+FLS_KERNEL_REDUCE, FLS_KERNEL_ADAMW, FLS_KERNEL_FEDAVG, FLS_KERNEL_COUNT = 0, 1, 2, 3
+FLS_STATUS_NONFINITE_NORM = 1
+FLS_MAX_GROUPS = 64
+FLS_MAX_GRAD_BUFFERS = 64
+FLS_BUFFER_ALIGN = 32
+
+EXPORTS = [
+    "fls_plan_create", "fls_plan_query", "fls_plan_bind", "fls_sync_step", "fls_sync_step_host", "fls_fedavg",
+    "fls_get_norms", "fls_get_reduced_grad", "fls_get_status", "fls_get_step", "fls_set_step", "fls_comm_report",
+    "fls_plan_tune", "fls_set_profiling", "fls_get_kernel_ms", "fls_get_launch_count", "fls_plan_destroy",
+    "fls_last_error",
+]
+
+
+class FlsError(RuntimeError):
+    def __init__(self, code: int, message: str):
+        super().__init__(f"libfls error {code}: {message}")
+        self.code = code
+
+
+class fls_plan_desc(C.Structure):
+    _fields_ = [("n_params", C.c_uint64), ("n_units", C.c_uint32), ("unit_numel", C.POINTER(C.c_uint64)),
+                ("groups", C.c_uint32), ("shard_dim", C.c_uint32), ("replicate_dim", C.c_uint32),
+                ("sync_period", C.c_uint32), ("grad_dtype", C.c_uint32), ("align_elems", C.c_uint32),
+                ("fedavg_what", C.c_uint32), ("reserved", C.c_uint32),
+                ("lr", C.c_double), ("beta1", C.c_double), ("beta2", C.c_double), ("eps", C.c_double),
+                ("weight_decay", C.c_double), ("max_grad_norm", C.c_double)]
+
+
+class fls_layout(C.Structure):
+    _fields_ = [("n_padded", C.c_uint64), ("shard_numel", C.c_uint64), ("n_units", C.c_uint32),
+                ("grad_buffers", C.c_uint32), ("unit_offset", C.POINTER(C.c_uint64)),
+                ("unit_shard_numel", C.POINTER(C.c_uint64)), ("unit_shard_offset", C.POINTER(C.c_uint64)),
+                ("workspace_bytes", C.c_uint64), ("n_segments", C.c_uint32), ("vector_path", C.c_uint32)]
+
+
+class fls_buffers(C.Structure):
+    _fields_ = [("grads", C.POINTER(C.c_void_p)), ("master", C.POINTER(C.c_void_p)), ("m", C.POINTER(C.c_void_p)),
+                ("v", C.POINTER(C.c_void_p)), ("param_bf16", C.POINTER(C.c_void_p)), ("workspace", C.c_void_p),
+                ("workspace_bytes", C.c_uint64)]
+
+
+class fls_cost5(C.Structure):
+    _fields_ = [(n, C.c_double) for n in ("fsdp", "hsdp", "fl", "fl_fsdp", "fl_hsdp")]
+
+    def as_dict(self):
+        return {n: getattr(self, n) for n, _ in self._fields_}
+
+
+class fls_comm_costs(C.Structure):
+    _fields_ = [("paper_bytes", fls_cost5), ("wire_bytes", fls_cost5), ("seconds", fls_cost5),
+                ("hbm_bytes_sync_step", C.c_double), ("hbm_bytes_fedavg", C.c_double)]
+
+
+def _load() -> C.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} not found: build it with `python -m paper_2609_20359_b200.build` "
+                          "(there is no CPU fallback)")
+    lib = C.CDLL(LIB_PATH)
+    P = C.c_void_p
+    lib.fls_plan_create.argtypes = [C.POINTER(fls_plan_desc), C.POINTER(P)]
+    lib.fls_plan_query.argtypes = [P, C.POINTER(fls_layout)]
+    lib.fls_plan_bind.argtypes = [P, C.POINTER(fls_buffers)]
+    lib.fls_sync_step.argtypes = [P, C.c_double, P, C.POINTER(C.c_int)]
+    lib.fls_sync_step_host.argtypes = [P, C.POINTER(C.c_void_p), C.c_double, P, C.POINTER(C.c_float), C.POINTER(C.c_int)]
+    lib.fls_fedavg.argtypes = [P, C.POINTER(C.c_uint64), P]
+    lib.fls_get_norms.argtypes = [P, C.POINTER(P), C.POINTER(P)]
+    lib.fls_get_reduced_grad.argtypes = [P, C.POINTER(P)]
+    lib.fls_get_status.argtypes = [P, C.POINTER(P)]
+    lib.fls_get_step.argtypes = [P, C.POINTER(C.c_uint64)]
+    lib.fls_set_step.argtypes = [P, C.c_uint64]
+    lib.fls_comm_report.argtypes = [P, C.POINTER(C.c_double), C.POINTER(fls_comm_costs)]
+    lib.fls_plan_tune.argtypes = [P, C.c_uint32, C.c_int, C.c_int]
+    lib.fls_set_profiling.argtypes = [P, C.c_int]
+    lib.fls_get_kernel_ms.argtypes = [P, C.POINTER(C.c_double), C.POINTER(C.c_uint64)]
+    lib.fls_get_launch_count.argtypes = [P, C.POINTER(C.c_uint64)]
+    lib.fls_plan_destroy.argtypes = [P]
+    lib.fls_last_error.argtypes = []
+    lib.fls_last_error.restype = C.c_char_p
+    for name in EXPORTS:
+        if name != "fls_last_error":
+            getattr(lib, name).restype = C.c_int
+    return lib
+
+
+lib = _load()
+
+
+def _check(rc: int) -> None:
+    if rc != FLS_OK:
+        raise FlsError(rc, lib.fls_last_error().decode())
+
+
+def _ptr(t) -> int:
+    """Device (or pinned host) address of a torch tensor, or a raw integer address."""
+    return int(t) if isinstance(t, int) else int(t.data_ptr())
+
+
+def _ptr_array(items: Sequence) -> C.Array:
+    return (C.c_void_p * len(items))(*[_ptr(t) for t in items])
+
+
+def _stream_handle(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return int(torch.cuda.current_stream().cuda_stream)
+    return int(stream) if isinstance(stream, int) else int(stream.cuda_stream)
+
+
+def fls_plan_create(n_params: int, unit_numel: Optional[Sequence[int]] = None, groups: int = 1, shard_dim: int = 1,
+                    replicate_dim: int = 1, sync_period: int = 1, grad_dtype: int = FLS_GRAD_BF16, align_elems: int = 8,
+                    fedavg_what: int = FLS_AVG_PARAMS, lr: float = 3e-4, beta1: float = 0.9, beta2: float = 0.95,
+                    eps: float = 1e-8, weight_decay: float = 0.1, max_grad_norm: float = 1.0) -> int:
+    """Returns the opaque plan handle."""
+    d = fls_plan_desc()
+    d.n_params = n_params
+    if unit_numel is not None:
+        arr = (C.c_uint64 * len(unit_numel))(*unit_numel)
+        d.n_units, d.unit_numel = len(unit_numel), arr
+    d.groups, d.shard_dim, d.replicate_dim, d.sync_period = groups, shard_dim, replicate_dim, sync_period
+    d.grad_dtype, d.align_elems, d.fedavg_what = grad_dtype, align_elems, fedavg_what
+    d.lr, d.beta1, d.beta2, d.eps, d.weight_decay, d.max_grad_norm = lr, beta1, beta2, eps, weight_decay, max_grad_norm
+    out = C.c_void_p()
+    _check(lib.fls_plan_create(C.byref(d), C.byref(out)))
+    return out.value
+
+
+def fls_plan_query(plan: int) -> dict:
+    lay = fls_layout()
+    _check(lib.fls_plan_query(plan, C.byref(lay)))
+    n = lay.n_units
+    return dict(n_padded=lay.n_padded, shard_numel=lay.shard_numel, n_units=n, grad_buffers=lay.grad_buffers,
+                unit_offset=[lay.unit_offset[i] for i in range(n)],
+                unit_shard_numel=[lay.unit_shard_numel[i] for i in range(n)],
+                unit_shard_offset=[lay.unit_shard_offset[i] for i in range(n)],
+                workspace_bytes=lay.workspace_bytes, n_segments=lay.n_segments, vector_path=bool(lay.vector_path))
+
+
+def fls_plan_bind(plan: int, grads: Sequence, master: Sequence, m: Sequence, v: Sequence, param_bf16: Sequence,
+                  workspace, workspace_bytes: Optional[int] = None) -> None:
+    """grads: G*K tensors (index g*K + rho*S + sigma); master/m/v/param_bf16: G tensors; workspace: a byte tensor."""
+    b = fls_buffers()
+    keep = [_ptr_array(grads), _ptr_array(master), _ptr_array(m), _ptr_array(v), _ptr_array(param_bf16)]
+    b.grads, b.master, b.m, b.v, b.param_bf16 = keep
+    b.workspace = _ptr(workspace)
+    b.workspace_bytes = workspace_bytes if workspace_bytes is not None else workspace.numel() * workspace.element_size()
+    _check(lib.fls_plan_bind(plan, C.byref(b)))
+
+
+def fls_sync_step(plan: int, lr: float = math.nan, stream=None) -> bool:
+    """One local step of all groups; returns True when FedAvg is due."""
+    due = C.c_int(0)
+    _check(lib.fls_sync_step(plan, lr, _stream_handle(stream), C.byref(due)))
+    return bool(due.value)
+
+
+def fls_sync_step_host(plan: int, host_grads: Sequence, lr: float = math.nan, stream=None, host_norms=None) -> bool:
+    """Same with gradients in (pinned) host tensors; host_norms: optional float32 CPU tensor of G entries."""
+    due = C.c_int(0)
+    arr = _ptr_array(host_grads)
+    norms = C.cast(_ptr(host_norms), C.POINTER(C.c_float)) if host_norms is not None else None
+    _check(lib.fls_sync_step_host(plan, arr, lr, _stream_handle(stream), norms, C.byref(due)))
+    return bool(due.value)
+
+
+def fls_fedavg(plan: int, sample_counts: Optional[Sequence[int]] = None, stream=None) -> None:
+    arr = (C.c_uint64 * len(sample_counts))(*sample_counts) if sample_counts is not None else None
+    _check(lib.fls_fedavg(plan, arr, _stream_handle(stream)))
+
+
+def fls_get_norms(plan: int):
+    """(device address of G norms, device address of G clip coefficients)."""
+    a, b = C.c_void_p(), C.c_void_p()
+    _check(lib.fls_get_norms(plan, C.byref(a), C.byref(b)))
+    return a.value, b.value
+
+
+def fls_get_reduced_grad(plan: int) -> int:
+    a = C.c_void_p()
+    _check(lib.fls_get_reduced_grad(plan, C.byref(a)))
+    return a.value
+
+
+def fls_get_status(plan: int) -> int:
+    a = C.c_void_p()
+    _check(lib.fls_get_status(plan, C.byref(a)))
+    return a.value
+
+
+def fls_get_step(plan: int) -> int:
+    t = C.c_uint64()
+    _check(lib.fls_get_step(plan, C.byref(t)))
+    return t.value
+
+
+def fls_set_step(plan: int, t: int) -> None:
+    _check(lib.fls_set_step(plan, t))
+
+
+def fls_comm_report(plan: int, bw_bytes_per_s: Optional[Sequence[float]] = None) -> dict:
+    out = fls_comm_costs()
+    bw = (C.c_double * 3)(*bw_bytes_per_s) if bw_bytes_per_s is not None else None
+    _check(lib.fls_comm_report(plan, bw, C.byref(out)))
+    return dict(paper_bytes=out.paper_bytes.as_dict(), wire_bytes=out.wire_bytes.as_dict(), seconds=out.seconds.as_dict(),
+                hbm_bytes_sync_step=out.hbm_bytes_sync_step, hbm_bytes_fedavg=out.hbm_bytes_fedavg)
+
+
+def fls_plan_tune(plan: int, kernel: int, ctas_per_sm: int = 0, descending: int = -1) -> None:
+    _check(lib.fls_plan_tune(plan, kernel, ctas_per_sm, descending))
+
+
+def fls_set_profiling(plan: int, enabled: bool) -> None:
+    _check(lib.fls_set_profiling(plan, int(enabled)))
+
+
+def fls_get_kernel_ms(plan: int):
+    ms = (C.c_double * FLS_KERNEL_COUNT)()
+    n = (C.c_uint64 * FLS_KERNEL_COUNT)()
+    _check(lib.fls_get_kernel_ms(plan, ms, n))
+    return list(ms), list(n)
+
+
+def fls_get_launch_count(plan: int) -> int:
+    n = C.c_uint64()
+    _check(lib.fls_get_launch_count(plan, C.byref(n)))
+    return n.value
+
+
+def fls_plan_destroy(plan: int) -> None:
+    _check(lib.fls_plan_destroy(plan))
+
+
+def fls_last_error() -> str:
+    return lib.fls_last_error().decode()
+
+
+__all__ = [n for n in dir() if n.startswith(("fls_", "FLS_"))] + ["FlsError", "lib", "LIB_PATH", "EXPORTS"]

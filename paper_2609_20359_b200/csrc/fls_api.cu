@@ -1,0 +1,534 @@
+// C ABI of libfls (see include/fls.h for the contract of every call).
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <limits>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "fls_kernels.h"
+
+using namespace fls;
+
+namespace {
+
+thread_local std::string g_err;
+
+int fail(int code, const char* fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  g_err = buf;
+  return code;
+}
+
+int cuda_fail(cudaError_t e, const char* what) {
+  return fail(FLS_ECUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+struct TimedLaunch {
+  cudaEvent_t begin, end;
+  int kernel;
+};
+
+}  // namespace
+
+struct fls_plan {
+  fls_plan_desc desc{};
+  std::vector<uint64_t> units;
+  Layout lay;
+  uint32_t K = 0;
+  uint64_t start_mask = 0, end_mask = 0;
+
+  bool bound = false;
+  int device = -1;
+  int sm_count = 0;
+  std::vector<const void*> grads;
+  std::vector<float*> master, m, v;
+  std::vector<uint16_t*> pbf16;
+  char* ws = nullptr;
+
+  uint64_t step = 0;
+  uint64_t launches = 0;
+  int ctas_per_sm[FLS_KERNEL_COUNT] = {4, 4, 2};
+  int descending[FLS_KERNEL_COUNT] = {0, 0, 0};
+
+  bool profiling = false;
+  std::vector<TimedLaunch> timed;
+  std::vector<cudaEvent_t> event_pool;
+
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t ev_begin = nullptr;
+  std::vector<cudaEvent_t> ev_copied;
+
+  const Segment* d_segs() const { return reinterpret_cast<const Segment*>(ws + kWsSegments); }
+  float* d_gbar() const { return reinterpret_cast<float*>(ws + lay.ws_scratch_offset); }
+  float* d_norms() const { return reinterpret_cast<float*>(ws + kWsNorms); }
+  float* d_coefs() const { return reinterpret_cast<float*>(ws + kWsCoefs); }
+  double* d_normsq() const { return reinterpret_cast<double*>(ws + kWsNormSq); }
+  double* d_partials() const { return reinterpret_cast<double*>(ws + kWsPartials); }
+  uint32_t* d_status() const { return reinterpret_cast<uint32_t*>(ws + kWsStatus); }
+  uint32_t* d_ticket() const { return reinterpret_cast<uint32_t*>(ws + kWsStatus) + 1; }
+
+  unsigned grid_for(int kernel) const {
+    uint64_t g = uint64_t(sm_count) * uint64_t(ctas_per_sm[kernel]);
+    g = std::min<uint64_t>(g, lay.n_tiles);
+    g = std::min<uint64_t>(g, kMaxBlocks);
+    return unsigned(std::max<uint64_t>(g, 1));
+  }
+
+  cudaEvent_t take_event() {
+    if (!event_pool.empty()) {
+      cudaEvent_t e = event_pool.back();
+      event_pool.pop_back();
+      return e;
+    }
+    cudaEvent_t e = nullptr;
+    cudaEventCreate(&e);
+    return e;
+  }
+};
+
+namespace {
+
+struct Range {
+  uintptr_t lo, hi;
+  const char* what;
+  int index;
+  bool output;
+};
+
+// Brackets one kernel launch with events when profiling is on.
+template <typename F>
+cudaError_t timed_launch(fls_plan* p, int kernel, cudaStream_t st, F&& launch) {
+  TimedLaunch t{nullptr, nullptr, kernel};
+  if (p->profiling) {
+    t.begin = p->take_event();
+    t.end = p->take_event();
+    if (!t.begin || !t.end) return cudaErrorMemoryAllocation;
+    cudaEventRecord(t.begin, st);
+  }
+  cudaError_t e = launch();
+  if (p->profiling) {
+    cudaEventRecord(t.end, st);
+    p->timed.push_back(t);
+  }
+  if (e == cudaSuccess) p->launches++;
+  return e;
+}
+
+int run_group(fls_plan* p, uint32_t g, double lr, uint64_t t_new, cudaStream_t st) {
+  const fls_plan_desc& d = p->desc;
+  ReduceArgs ra{};
+  for (uint32_t k = 0; k < p->K; ++k) ra.grad[k] = p->grads[size_t(g) * p->K + k];
+  ra.gbar = p->d_gbar();
+  ra.segs = p->d_segs();
+  ra.n_tiles = p->lay.n_tiles;
+  ra.n_seg = uint32_t(p->lay.segments.size());
+  ra.K = p->K;
+  ra.S = d.shard_dim;
+  ra.k_float = float(p->K);
+  ra.start_mask = p->start_mask;
+  ra.end_mask = p->end_mask;
+  ra.partials = p->d_partials();
+  ra.ticket = p->d_ticket();
+  ra.norm_out = p->d_norms() + g;
+  ra.coef_out = p->d_coefs() + g;
+  ra.normsq_out = p->d_normsq() + g;
+  ra.status = p->d_status();
+  ra.max_grad_norm = d.max_grad_norm;
+  ra.descending = p->descending[FLS_KERNEL_REDUCE];
+  const bool f32 = d.grad_dtype == FLS_GRAD_F32;
+  cudaError_t e = timed_launch(p, FLS_KERNEL_REDUCE, st,
+                               [&] { return launch_reduce(ra, f32, p->grid_for(FLS_KERNEL_REDUCE), st); });
+  if (e != cudaSuccess) return cuda_fail(e, "reduce kernel launch");
+
+  // Scalars of the AdamW step, in double on the host, handed to the kernel as fp32.
+  const double bc1 = 1.0 - std::pow(d.beta1, double(t_new));
+  const double bc2 = 1.0 - std::pow(d.beta2, double(t_new));
+  AdamArgs aa{};
+  aa.gbar = p->d_gbar();
+  aa.theta = p->master[g];
+  aa.m = p->m[g];
+  aa.v = p->v[g];
+  aa.pbf16 = p->pbf16[g];
+  aa.segs = p->d_segs();
+  aa.n_tiles = p->lay.n_tiles;
+  aa.n_seg = ra.n_seg;
+  aa.descending = p->descending[FLS_KERNEL_ADAMW];
+  aa.coef = p->d_coefs() + g;
+  aa.decay = float(1.0 - lr * d.weight_decay);
+  aa.beta1 = float(d.beta1);
+  aa.omb1 = float(1.0 - d.beta1);
+  aa.beta2 = float(d.beta2);
+  aa.omb2 = float(1.0 - d.beta2);
+  aa.step_size = float(lr / bc1);
+  aa.inv_sqrt_bc2 = float(1.0 / std::sqrt(bc2));
+  aa.eps = float(d.eps);
+  e = timed_launch(p, FLS_KERNEL_ADAMW, st, [&] { return launch_adamw(aa, p->grid_for(FLS_KERNEL_ADAMW), st); });
+  if (e != cudaSuccess) return cuda_fail(e, "adamw kernel launch");
+  return FLS_OK;
+}
+
+bool step_preamble(fls_plan* p, double* lr) {
+  if (std::isnan(*lr)) *lr = p->desc.lr;
+  return *lr >= 0.0 && std::isfinite(*lr);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* fls_last_error(void) { return g_err.c_str(); }
+
+int fls_plan_create(const fls_plan_desc* desc, fls_plan** out) {
+  if (out) *out = nullptr;
+  if (!desc || !out) return fail(FLS_EINVAL, "fls_plan_create: null argument");
+  const fls_plan_desc& d = *desc;
+  if (d.groups == 0 || d.shard_dim == 0 || d.replicate_dim == 0 || d.sync_period == 0 || d.align_elems == 0)
+    return fail(FLS_EINVAL, "groups, shard_dim, replicate_dim, sync_period and align_elems must be >= 1");
+  if (d.groups > FLS_MAX_GROUPS) return fail(FLS_EINVAL, "groups = %u exceeds %d", d.groups, FLS_MAX_GROUPS);
+  const uint64_t K = uint64_t(d.shard_dim) * d.replicate_dim;
+  if (K > FLS_MAX_GRAD_BUFFERS)
+    return fail(FLS_EINVAL, "shard_dim*replicate_dim = %llu exceeds %d", (unsigned long long)K, FLS_MAX_GRAD_BUFFERS);
+  if (d.grad_dtype != FLS_GRAD_BF16 && d.grad_dtype != FLS_GRAD_F32) return fail(FLS_EINVAL, "unknown grad_dtype %u", d.grad_dtype);
+  if (!(d.fedavg_what & FLS_AVG_PARAMS) || (d.fedavg_what & ~uint32_t(FLS_AVG_PARAMS | FLS_AVG_OPT_STATE)))
+    return fail(FLS_EINVAL, "fedavg_what must be FLS_AVG_PARAMS, optionally | FLS_AVG_OPT_STATE");
+  if (d.reserved != 0) return fail(FLS_EINVAL, "reserved must be 0");
+  if (!(d.beta1 >= 0.0 && d.beta1 < 1.0) || !(d.beta2 >= 0.0 && d.beta2 < 1.0)) return fail(FLS_EINVAL, "betas must lie in [0, 1)");
+  if (!(d.eps > 0.0) || !std::isfinite(d.eps)) return fail(FLS_EINVAL, "eps must be positive");
+  if (!(d.lr >= 0.0) || !std::isfinite(d.lr)) return fail(FLS_EINVAL, "lr must be finite and >= 0");
+  if (!std::isfinite(d.weight_decay) || d.weight_decay < 0.0) return fail(FLS_EINVAL, "weight_decay must be finite and >= 0");
+  if (std::isnan(d.max_grad_norm)) return fail(FLS_EINVAL, "max_grad_norm is NaN");
+  if (d.n_params == 0) return fail(FLS_EINVAL, "n_params must be >= 1");
+
+  std::vector<uint64_t> units;
+  if (d.n_units == 0 && d.unit_numel == nullptr) {
+    units.push_back(d.n_params);
+  } else {
+    if (d.n_units == 0 || d.unit_numel == nullptr) return fail(FLS_EINVAL, "n_units and unit_numel must be given together");
+    units.assign(d.unit_numel, d.unit_numel + d.n_units);
+  }
+  unsigned __int128 sum = 0;
+  for (uint64_t n : units) sum += n;
+  if (sum != d.n_params) return fail(FLS_EINVAL, "sum(unit_numel) differs from n_params");
+
+  fls_plan* p = new (std::nothrow) fls_plan();
+  if (!p) return fail(FLS_EINVAL, "out of host memory");
+  p->desc = d;
+  p->units = units;
+  p->desc.unit_numel = nullptr;   // the caller's table is not kept; p->units is the copy
+  p->desc.n_units = uint32_t(units.size());
+  const std::string msg = build_layout(units, d.shard_dim, d.align_elems, &p->lay);
+  if (!msg.empty()) {
+    delete p;
+    return fail(FLS_EINVAL, "layout: %s", msg.c_str());
+  }
+  p->K = uint32_t(K);
+  for (uint32_t k = 0; k < p->K; ++k) {
+    if (k % d.shard_dim == 0) p->start_mask |= 1ull << k;
+    if (k % d.shard_dim == d.shard_dim - 1) p->end_mask |= 1ull << k;
+  }
+  *out = p;
+  return FLS_OK;
+}
+
+int fls_plan_query(const fls_plan* plan, fls_layout* out) {
+  if (!plan || !out) return fail(FLS_EINVAL, "fls_plan_query: null argument");
+  out->n_padded = plan->lay.n_padded;
+  out->shard_numel = plan->lay.shard_numel;
+  out->n_units = uint32_t(plan->units.size());
+  out->grad_buffers = plan->K;
+  out->unit_offset = plan->lay.unit_offset.data();
+  out->unit_shard_numel = plan->lay.unit_shard_numel.data();
+  out->unit_shard_offset = plan->lay.unit_shard_offset.data();
+  out->workspace_bytes = plan->lay.workspace_bytes;
+  out->n_segments = uint32_t(plan->lay.segments.size());
+  out->vector_path = plan->lay.vector_path ? 1u : 0u;
+  return FLS_OK;
+}
+
+int fls_plan_bind(fls_plan* p, const fls_buffers* b) {
+  if (!p || !b) return fail(FLS_EINVAL, "fls_plan_bind: null argument");
+  if (!b->grads || !b->master || !b->m || !b->v || !b->param_bf16 || !b->workspace)
+    return fail(FLS_EPTR, "fls_plan_bind: null pointer table or workspace");
+  if (b->workspace_bytes < p->lay.workspace_bytes)
+    return fail(FLS_ESIZE, "workspace has %llu bytes, %llu needed", (unsigned long long)b->workspace_bytes,
+                (unsigned long long)p->lay.workspace_bytes);
+  const uint32_t G = p->desc.groups, K = p->K;
+  const uint64_t N = p->lay.n_padded;
+  const uint64_t eg = p->desc.grad_dtype == FLS_GRAD_F32 ? 4 : 2;
+
+  std::vector<Range> ranges;
+  auto add = [&](const void* ptr, uint64_t bytes, const char* what, int idx, bool output) {
+    ranges.push_back(Range{reinterpret_cast<uintptr_t>(ptr), reinterpret_cast<uintptr_t>(ptr) + bytes, what, idx, output});
+  };
+  for (uint32_t i = 0; i < G * K; ++i) add(b->grads[i], N * eg, "grads", int(i), false);
+  for (uint32_t g = 0; g < G; ++g) {
+    add(b->master[g], N * 4, "master", int(g), true);
+    add(b->m[g], N * 4, "m", int(g), true);
+    add(b->v[g], N * 4, "v", int(g), true);
+    add(b->param_bf16[g], N * 2, "param_bf16", int(g), true);
+  }
+  add(b->workspace, p->lay.workspace_bytes, "workspace", 0, true);
+
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+  for (const Range& r : ranges) {
+    if (r.lo == 0) return fail(FLS_EPTR, "%s[%d] is null", r.what, r.index);
+    if (r.lo % FLS_BUFFER_ALIGN != 0) return fail(FLS_EALIGN, "%s[%d] is not %d-byte aligned", r.what, r.index, FLS_BUFFER_ALIGN);
+    cudaPointerAttributes attr{};
+    e = cudaPointerGetAttributes(&attr, reinterpret_cast<const void*>(r.lo));
+    if (e != cudaSuccess) {
+      cudaGetLastError();
+      return fail(FLS_EPTR, "%s[%d]: %s", r.what, r.index, cudaGetErrorString(e));
+    }
+    if (attr.type != cudaMemoryTypeDevice && attr.type != cudaMemoryTypeManaged)
+      return fail(FLS_EPTR, "%s[%d] is not device memory", r.what, r.index);
+    if (attr.type == cudaMemoryTypeDevice && attr.device != dev)
+      return fail(FLS_EPTR, "%s[%d] lives on device %d, current device is %d", r.what, r.index, attr.device, dev);
+  }
+  // outputs may overlap nothing; gradient buffers may only overlap each other exactly (a caller may
+  // feed one buffer to several replicas) but never an output
+  std::vector<size_t> order(ranges.size());
+  for (size_t i = 0; i < order.size(); ++i) order[i] = i;
+  std::sort(order.begin(), order.end(), [&](size_t x, size_t y) { return ranges[x].lo < ranges[y].lo; });
+  for (size_t q = 0; q < order.size(); ++q) {
+    const Range& r0 = ranges[order[q]];
+    for (size_t w = q + 1; w < order.size() && ranges[order[w]].lo < r0.hi; ++w) {
+      const Range& r1 = ranges[order[w]];
+      if (r0.output || r1.output)
+        return fail(FLS_EPTR, "%s[%d] overlaps %s[%d]", r0.what, r0.index, r1.what, r1.index);
+    }
+  }
+
+  int sms = 0;
+  e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
+  p->device = dev;
+  p->sm_count = sms;
+  p->grads.assign(b->grads, b->grads + size_t(G) * K);
+  p->master.assign(b->master, b->master + G);
+  p->m.assign(b->m, b->m + G);
+  p->v.assign(b->v, b->v + G);
+  p->pbf16.resize(G);
+  for (uint32_t g = 0; g < G; ++g) p->pbf16[g] = static_cast<uint16_t*>(b->param_bf16[g]);
+  p->ws = static_cast<char*>(b->workspace);
+
+  e = cudaMemset(p->ws, 0, size_t(kWsSegments));
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMemset(workspace head)");
+  e = cudaMemcpy(p->ws + kWsSegments, p->lay.segments.data(), p->lay.segments.size() * sizeof(Segment), cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(segment table)");
+  e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceSynchronize");
+  if (!p->copy_stream) {
+    e = cudaStreamCreateWithFlags(&p->copy_stream, cudaStreamNonBlocking);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaStreamCreate");
+    e = cudaEventCreateWithFlags(&p->ev_begin, cudaEventDisableTiming);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaEventCreate");
+    p->ev_copied.resize(G, nullptr);
+    for (uint32_t g = 0; g < G; ++g) {
+      e = cudaEventCreateWithFlags(&p->ev_copied[g], cudaEventDisableTiming);
+      if (e != cudaSuccess) return cuda_fail(e, "cudaEventCreate");
+    }
+  }
+  p->bound = true;
+  return FLS_OK;
+}
+
+int fls_sync_step(fls_plan* p, double lr, void* cuda_stream, int* fedavg_due) {
+  if (!p) return fail(FLS_EINVAL, "fls_sync_step: null plan");
+  if (!p->bound) return fail(FLS_ESTATE, "fls_sync_step: plan has no buffers bound");
+  if (!step_preamble(p, &lr)) return fail(FLS_EINVAL, "fls_sync_step: lr must be finite and >= 0");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const uint64_t t_new = p->step + 1;
+  for (uint32_t g = 0; g < p->desc.groups; ++g) {
+    const int rc = run_group(p, g, lr, t_new, st);
+    if (rc != FLS_OK) return rc;
+  }
+  p->step = t_new;
+  if (fedavg_due) *fedavg_due = (t_new % p->desc.sync_period == 0) ? 1 : 0;
+  return FLS_OK;
+}
+
+int fls_sync_step_host(fls_plan* p, const void* const* host_grads, double lr, void* cuda_stream, float* host_norms,
+                       int* fedavg_due) {
+  if (!p || !host_grads) return fail(FLS_EINVAL, "fls_sync_step_host: null argument");
+  if (!p->bound) return fail(FLS_ESTATE, "fls_sync_step_host: plan has no buffers bound");
+  if (!step_preamble(p, &lr)) return fail(FLS_EINVAL, "fls_sync_step_host: lr must be finite and >= 0");
+  const uint32_t G = p->desc.groups, K = p->K;
+  for (uint32_t i = 0; i < G * K; ++i)
+    if (!host_grads[i]) return fail(FLS_EPTR, "host_grads[%u] is null", i);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const uint64_t bytes = p->lay.n_padded * (p->desc.grad_dtype == FLS_GRAD_F32 ? 4ull : 2ull);
+  const uint64_t t_new = p->step + 1;
+  // the copies may not overtake work already queued on the caller's stream that still reads the buffers
+  cudaError_t e = cudaEventRecord(p->ev_begin, st);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaEventRecord");
+  e = cudaStreamWaitEvent(p->copy_stream, p->ev_begin, 0);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaStreamWaitEvent");
+  for (uint32_t g = 0; g < G; ++g) {
+    for (uint32_t k = 0; k < K; ++k) {
+      e = cudaMemcpyAsync(const_cast<void*>(p->grads[size_t(g) * K + k]), host_grads[size_t(g) * K + k], bytes,
+                          cudaMemcpyHostToDevice, p->copy_stream);
+      if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpyAsync(host gradients)");
+    }
+    e = cudaEventRecord(p->ev_copied[g], p->copy_stream);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaEventRecord");
+    e = cudaStreamWaitEvent(st, p->ev_copied[g], 0);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaStreamWaitEvent");
+    const int rc = run_group(p, g, lr, t_new, st);
+    if (rc != FLS_OK) return rc;
+  }
+  if (host_norms) {
+    e = cudaMemcpyAsync(host_norms, p->d_norms(), sizeof(float) * G, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpyAsync(norms)");
+  }
+  e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+  p->step = t_new;
+  if (fedavg_due) *fedavg_due = (t_new % p->desc.sync_period == 0) ? 1 : 0;
+  return FLS_OK;
+}
+
+int fls_fedavg(fls_plan* p, const uint64_t* sample_counts, void* cuda_stream) {
+  if (!p) return fail(FLS_EINVAL, "fls_fedavg: null plan");
+  if (!p->bound) return fail(FLS_ESTATE, "fls_fedavg: plan has no buffers bound");
+  const uint32_t G = p->desc.groups;
+  long double total = 0;
+  for (uint32_t g = 0; g < G; ++g) total += sample_counts ? (long double)sample_counts[g] : 1.0L;
+  if (!(total > 0)) return fail(FLS_EINVAL, "fls_fedavg: all sample counts are zero");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  FedavgArgs fa{};
+  for (uint32_t g = 0; g < G; ++g) {
+    const double n = sample_counts ? double(sample_counts[g]) : 1.0;
+    fa.w[g] = float(n / double(total));
+  }
+  fa.segs = p->d_segs();
+  fa.n_tiles = p->lay.n_tiles;
+  fa.n_seg = uint32_t(p->lay.segments.size());
+  fa.G = G;
+  fa.descending = p->descending[FLS_KERNEL_FEDAVG];
+  const int n_arrays = (p->desc.fedavg_what & FLS_AVG_OPT_STATE) ? 3 : 1;
+  for (int arr = 0; arr < n_arrays; ++arr) {
+    for (uint32_t g = 0; g < G; ++g) {
+      fa.x[g] = arr == 0 ? p->master[g] : (arr == 1 ? p->m[g] : p->v[g]);
+      fa.pbf16[g] = p->pbf16[g];
+    }
+    fa.write_bf16 = arr == 0 ? 1 : 0;
+    cudaError_t e = timed_launch(p, FLS_KERNEL_FEDAVG, st, [&] { return launch_fedavg(fa, p->grid_for(FLS_KERNEL_FEDAVG), st); });
+    if (e != cudaSuccess) return cuda_fail(e, "fedavg kernel launch");
+  }
+  return FLS_OK;
+}
+
+int fls_get_norms(const fls_plan* p, const float** dev_norms, const float** dev_coefs) {
+  if (!p) return fail(FLS_EINVAL, "fls_get_norms: null plan");
+  if (!p->bound) return fail(FLS_ESTATE, "fls_get_norms: plan has no buffers bound");
+  if (dev_norms) *dev_norms = p->d_norms();
+  if (dev_coefs) *dev_coefs = p->d_coefs();
+  return FLS_OK;
+}
+
+int fls_get_reduced_grad(const fls_plan* p, const float** dev_gbar) {
+  if (!p || !dev_gbar) return fail(FLS_EINVAL, "fls_get_reduced_grad: null argument");
+  if (!p->bound) return fail(FLS_ESTATE, "fls_get_reduced_grad: plan has no buffers bound");
+  *dev_gbar = p->d_gbar();
+  return FLS_OK;
+}
+
+int fls_get_status(const fls_plan* p, const uint32_t** dev_status) {
+  if (!p || !dev_status) return fail(FLS_EINVAL, "fls_get_status: null argument");
+  if (!p->bound) return fail(FLS_ESTATE, "fls_get_status: plan has no buffers bound");
+  *dev_status = p->d_status();
+  return FLS_OK;
+}
+
+int fls_get_step(const fls_plan* p, uint64_t* t) {
+  if (!p || !t) return fail(FLS_EINVAL, "fls_get_step: null argument");
+  *t = p->step;
+  return FLS_OK;
+}
+
+int fls_set_step(fls_plan* p, uint64_t t) {
+  if (!p) return fail(FLS_EINVAL, "fls_set_step: null plan");
+  p->step = t;
+  return FLS_OK;
+}
+
+int fls_comm_report(const fls_plan* p, const double* bw, fls_comm_costs* out) {
+  if (!p || !out) return fail(FLS_EINVAL, "fls_comm_report: null argument");
+  if (bw)
+    for (int i = 0; i < 3; ++i)
+      if (!(bw[i] > 0.0)) return fail(FLS_EINVAL, "fls_comm_report: bandwidths must be positive");
+  comm_report(p->lay, p->desc, bw, out);
+  return FLS_OK;
+}
+
+int fls_plan_tune(fls_plan* p, uint32_t kernel, int ctas_per_sm, int descending) {
+  if (!p || kernel >= FLS_KERNEL_COUNT) return fail(FLS_EINVAL, "fls_plan_tune: bad argument");
+  if (ctas_per_sm > 0) p->ctas_per_sm[kernel] = std::min(ctas_per_sm, 32);
+  if (descending >= 0) p->descending[kernel] = descending ? 1 : 0;
+  return FLS_OK;
+}
+
+int fls_set_profiling(fls_plan* p, int enabled) {
+  if (!p) return fail(FLS_EINVAL, "fls_set_profiling: null plan");
+  p->profiling = enabled != 0;
+  return FLS_OK;
+}
+
+int fls_get_kernel_ms(fls_plan* p, double* ms, uint64_t* launches) {
+  if (!p || !ms || !launches) return fail(FLS_EINVAL, "fls_get_kernel_ms: null argument");
+  for (int k = 0; k < FLS_KERNEL_COUNT; ++k) {
+    ms[k] = 0.0;
+    launches[k] = 0;
+  }
+  int rc = FLS_OK;
+  for (const TimedLaunch& t : p->timed) {
+    cudaError_t e = cudaEventSynchronize(t.end);
+    float f = 0.f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&f, t.begin, t.end);
+    if (e != cudaSuccess) {
+      rc = cuda_fail(e, "cudaEventElapsedTime");
+    } else {
+      ms[t.kernel] += double(f);
+      launches[t.kernel] += 1;
+    }
+    p->event_pool.push_back(t.begin);
+    p->event_pool.push_back(t.end);
+  }
+  p->timed.clear();
+  return rc;
+}
+
+int fls_get_launch_count(const fls_plan* p, uint64_t* launches) {
+  if (!p || !launches) return fail(FLS_EINVAL, "fls_get_launch_count: null argument");
+  *launches = p->launches;
+  return FLS_OK;
+}
+
+int fls_plan_destroy(fls_plan* p) {
+  if (!p) return FLS_OK;
+  for (const TimedLaunch& t : p->timed) {
+    cudaEventDestroy(t.begin);
+    cudaEventDestroy(t.end);
+  }
+  for (cudaEvent_t e : p->event_pool) cudaEventDestroy(e);
+  for (cudaEvent_t e : p->ev_copied)
+    if (e) cudaEventDestroy(e);
+  if (p->ev_begin) cudaEventDestroy(p->ev_begin);
+  if (p->copy_stream) cudaStreamDestroy(p->copy_stream);
+  delete p;
+  return FLS_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,48 @@
+// Internal declarations shared by the host code and the kernels of libfls.
+#pragma once
+#include <cstdint>
+#include <string>
+#include <vector>
+
+#include "fls.h"
+
+namespace fls {
+
+constexpr int kThreads = 256;            // threads per CTA, all kernels
+constexpr int kVec = 8;                  // elements per thread per tile
+constexpr int kTile = kThreads * kVec;   // 2048 elements per tile
+constexpr int kMaxBlocks = 4096;         // upper bound on any grid (size of the norm-partials array)
+
+// A run of elements that is contiguous in both the unsharded order (index j) and the shard order
+// (address a): one rank's slice of one unit, or several merged when they are adjacent in both.
+struct Segment {
+  uint64_t tile_begin;  // first tile of this segment
+  uint64_t tile_end;    // one past its last tile
+  uint64_t j0;          // start in the unsharded order (gradients, bf16 copy)
+  uint64_t a0;          // start in the shard order (master, m, v, reduced gradient)
+  uint64_t len;         // elements
+  uint64_t aligned;     // 1 if j0 and a0 are multiples of kVec: 128/256-bit accesses allowed
+};
+
+// Workspace layout (byte offsets); the head is fixed, the segment table and the scratch follow.
+constexpr uint64_t kWsStatus = 0;        // uint32 status, uint32 ticket counter
+constexpr uint64_t kWsNorms = 256;       // float[64]
+constexpr uint64_t kWsCoefs = 512;       // float[64]
+constexpr uint64_t kWsNormSq = 768;      // double[64]
+constexpr uint64_t kWsPartials = 1280;   // double[kMaxBlocks]
+constexpr uint64_t kWsSegments = kWsPartials + 8ull * kMaxBlocks;
+
+struct Layout {
+  std::vector<uint64_t> unit_numel, unit_offset, unit_shard_numel, unit_shard_offset;
+  std::vector<Segment> segments;
+  uint64_t n_params = 0, n_padded = 0, shard_numel = 0, n_tiles = 0;
+  uint64_t ws_scratch_offset = 0, workspace_bytes = 0;
+  bool vector_path = true;
+};
+
+// Host planner: fills `out` from the unit table; returns an error message or "" on success.
+std::string build_layout(const std::vector<uint64_t>& unit_numel, uint32_t S, uint32_t Q, Layout* out);
+
+void comm_report(const Layout& lay, const fls_plan_desc& d, const double* bw, fls_comm_costs* out);
+
+}  // namespace fls

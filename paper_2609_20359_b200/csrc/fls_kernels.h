@@ -1,0 +1,56 @@
+// Kernel argument blocks and launchers (implemented in fls_kernels.cu).
+#pragma once
+#include <cuda_runtime.h>
+
+#include "fls_internal.h"
+
+namespace fls {
+
+struct ReduceArgs {
+  const void* grad[FLS_MAX_GRAD_BUFFERS];  // device, K buffers of this group, index rho*S + sigma
+  float* gbar;                             // device, reduced gradient (shard order)
+  const Segment* segs;                     // device
+  uint64_t n_tiles;
+  uint32_t n_seg;
+  uint32_t K, S;
+  float k_float;                           // K as float: the mean divides by it once
+  uint64_t start_mask, end_mask;           // bit k set: buffer k opens / closes a sharding group
+  double* partials;                        // device, one per CTA
+  uint32_t* ticket;                        // device, zero between launches
+  float* norm_out;
+  float* coef_out;
+  double* normsq_out;
+  uint32_t* status;
+  double max_grad_norm;
+  int descending;
+};
+
+struct AdamArgs {
+  const float* gbar;
+  float *theta, *m, *v;
+  uint16_t* pbf16;
+  const Segment* segs;
+  uint64_t n_tiles;
+  uint32_t n_seg;
+  int descending;
+  const float* coef;                       // device, written by the reduce kernel of the same group
+  float decay, beta1, omb1, beta2, omb2, step_size, inv_sqrt_bc2, eps;
+};
+
+struct FedavgArgs {
+  float* x[FLS_MAX_GROUPS];                // device, the G copies (in/out)
+  uint16_t* pbf16[FLS_MAX_GROUPS];         // device, the G bf16 copies (out), used if write_bf16
+  float w[FLS_MAX_GROUPS];
+  const Segment* segs;
+  uint64_t n_tiles;
+  uint32_t n_seg;
+  uint32_t G;
+  int write_bf16;
+  int descending;
+};
+
+cudaError_t launch_reduce(const ReduceArgs& a, bool f32, unsigned grid, cudaStream_t st);
+cudaError_t launch_adamw(const AdamArgs& a, unsigned grid, cudaStream_t st);
+cudaError_t launch_fedavg(const FedavgArgs& a, unsigned grid, cudaStream_t st);
+
+}  // namespace fls

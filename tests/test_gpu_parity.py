@@ -1,0 +1,340 @@
+"""GPU parity: the CUDA library against the CPU oracle, element by element, on the same seeded
+inputs, through the C ABI.  Tolerances: |d| <= 1e-6*max(1,|x|) on fp32 master/m/v (plus relative
+gates on m and v, whose magnitudes make the absolute gate weak), <= 1 bf16 ulp on the bf16 copy."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import synthetic as sy
+from oracle import fls_oracle as orc
+from tests.harness import Case, assert_bf16_close, assert_state_close, bf16_bits
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def fls():
+    from paper_2609_20359_b200 import build
+    build.build()
+    import paper_2609_20359_b200._binding as b
+    return b
+
+
+def test_generator_is_bit_identical_on_cpu_and_gpu():
+    key = sy.stream_key(77, sy.KIND_GRAD, 3, 1, 2)
+    for dt in (torch.float32, torch.bfloat16):
+        a = sy.normal_fill_(torch.empty(300_001, dtype=dt), key, 1e-3, 1.37, start=12345)
+        b = sy.normal_fill_(torch.empty(300_001, dtype=dt, device="cuda"), key, 1e-3, 1.37, start=12345)
+        assert torch.equal(a.view(torch.int16 if dt == torch.bfloat16 else torch.int32),
+                           b.cpu().view(torch.int16 if dt == torch.bfloat16 else torch.int32))
+    idx = torch.tensor([0, 1, 299_999, 12, 7_000_000_000], dtype=torch.int64)
+    assert torch.equal(sy.normal_at(idx, key, 1e-3), sy.normal_at(idx.cuda(), key, 1e-3).cpu())
+
+
+# ------------------------------------------------------------------ the tiny FL+FSDP workload
+@pytest.mark.parametrize("Q,clip", [(1, 1.0), (8, 1.0), (8, 0.1)])
+def test_tiny_fl_fsdp_8_steps(fls, Q, clip):
+    """P = 1,000,003, G = 2, K = S = 4, H = 4, 8 steps, equal weights.  Q = 1 pads to a multiple of
+    S only (shard length 250,001: the buffer tail leaves the vector path); clip 1.0 is inactive
+    (norm ~ 0.5), clip 0.1 is active."""
+    cfg = sy.CONFIGS[0]
+    hp = orc.Hyper(max_grad_norm=clip)
+    c = Case(cfg["unit_numel"], cfg["groups"], cfg["shard_dim"], 1, cfg["sync_period"], Q, seed=cfg["seed"], hp=hp)
+    active = []
+    for _ in range(cfg["steps"]):
+        row = c.step()
+        active += [co < 1.0 for _, co in row]
+        c.compare()
+    assert all(active) if clip < 0.5 else not any(active)
+    # after the last FedAvg (step 8) all groups hold the same parameters, bit for bit
+    assert torch.equal(c.sess.master[0], c.sess.master[1]) and torch.equal(c.sess.param_bf16[0], c.sess.param_bf16[1])
+    assert c.sess.status() == 0
+    c.close()
+
+
+# ------------------------------------------------------------------ layouts, reduction orders, dtypes
+@pytest.mark.parametrize("units,G,S,R_rep,Q,dtype", [
+    ([17], 2, 4, 1, 1, "bf16"),                         # the brute-force size
+    ([1], 1, 1, 1, 1, "bf16"),                          # a single parameter
+    ([5000, 1, 12345, 2048, 77], 2, 4, 1, 8, "bf16"),   # several units, aligned shards, ragged tiles
+    ([5000, 1, 12345, 2048, 77], 2, 3, 1, 1, "bf16"),   # unaligned shards: element-wise path
+    ([40000, 30011], 2, 4, 2, 8, "bf16"),               # two-level order, K = 8
+    ([40000, 30011], 1, 8, 8, 8, "bf16"),               # K = 64
+    ([40000, 30011], 2, 3, 1, 8, "bf16"),               # K = 3: mean is not a power-of-two scale
+    ([40000, 30011], 2, 5, 2, 8, "f32"),                # fp32 gradients, K = 10 (two load batches)
+    ([70001], 3, 2, 2, 1, "f32"),                       # fp32 gradients, unaligned tail
+    ([300000], 1, 1, 1, 8, "bf16"),                     # K = 1: plain AdamW on the gradient itself
+])
+def test_layouts_and_orders(fls, units, G, S, R_rep, Q, dtype):
+    hp = orc.Hyper(max_grad_norm=0.05)
+    c = Case(units, G, S, R_rep, H=2, Q=Q, grad_dtype=dtype, opt_state=True, hp=hp, per_buffer_scale=True)
+    counts = [sy.sample_count(5, g) for g in range(G)]
+    for _ in range(3):
+        c.step(counts)
+        c.compare()
+    c.close()
+
+
+def test_reduced_gradient_matches_oracle_exactly_for_bf16(fls):
+    """With bf16 inputs the fp32 running sum is exact here, so the mean gradient is bit-identical."""
+    c = Case([40000, 30011], 1, 4, 2, H=10, Q=8)
+    grads = c.load_grads(1)
+    c.sess.step()
+    torch.cuda.synchronize()
+    want = orc.pack_sharded(c.L, orc.reduce_mean(grads[0], 4, 2))
+    assert np.array_equal(c.sess.reduced_grad().cpu().numpy(), want)
+    c.close()
+
+
+def test_two_level_order_differs_from_flat_where_fp32_rounds(fls):
+    """fp32 gradients spanning many binades: the shard-then-replicate order and the flat order round
+    differently; each matches the oracle run in the same order (to fp32 rounding of the sum)."""
+    units, P = [4096], 4096
+    def big(t, g, k):
+        x = sy.normal_fill_(torch.empty(P), sy.stream_key(9, sy.KIND_GRAD, t, g, k), 1.0)
+        return x * (10.0 ** (k % 4 * 2))
+    res = {}
+    for (S, R_rep) in ((8, 1), (4, 2)):
+        c = Case(units, 1, S, R_rep, H=10, Q=8, grad_dtype="f32", hp=orc.Hyper(max_grad_norm=0.0))
+        grads = c.load_grads(1, big)
+        c.sess.step()
+        torch.cuda.synchronize()
+        got = c.sess.reduced_grad().cpu().numpy()
+        want = orc.reduce_mean(grads[0], S, R_rep)
+        assert np.allclose(got, want, rtol=8 * 2 ** -24, atol=0)
+        res[(S, R_rep)] = got
+        c.close()
+    assert not np.array_equal(res[(8, 1)], res[(4, 2)])
+
+
+# ------------------------------------------------------------------ FedAvg
+@pytest.mark.parametrize("G,opt_state,counts", [(1, True, [9]), (3, False, [1, 2, 5]), (8, True, None), (9, True, "rand"), (64, False, "rand")])
+def test_fedavg(fls, G, opt_state, counts):
+    units = [3000, 517] if G < 64 else [999]
+    c = Case(units, G, 2, 1, H=1, Q=8, opt_state=opt_state, hp=orc.Hyper(max_grad_norm=0.01))
+    if counts == "rand":
+        counts = [sy.sample_count(11, g) for g in range(G)]
+    before = [m.clone() for m in c.sess.m]
+    c.step(counts, fedavg=False)                 # groups diverge (different gradients)
+    if G > 1:
+        assert not torch.equal(c.sess.master[0], c.sess.master[1])
+    m_after_step = [m.clone() for m in c.sess.m]
+    orc.fedavg(c.states, counts, opt_state)
+    c.sess.fedavg(counts)
+    c.compare(check_norms=False)
+    for g in range(1, G):                         # every copy equals the average, bit for bit
+        assert torch.equal(c.sess.master[g], c.sess.master[0]) and torch.equal(c.sess.param_bf16[g], c.sess.param_bf16[0])
+        if opt_state:
+            assert torch.equal(c.sess.v[g], c.sess.v[0])
+    if not opt_state:                             # params only: m and v untouched
+        assert all(torch.equal(a, b) for a, b in zip(m_after_step, c.sess.m))
+    del before
+    c.close()
+
+
+def test_fedavg_g1_is_bit_exact_identity_and_idempotent(fls):
+    c = Case([5000], 1, 2, 1, H=1, Q=8, opt_state=True)
+    c.step(fedavg=False)
+    snap = (c.sess.master[0].clone(), c.sess.m[0].clone(), c.sess.v[0].clone())
+    c.sess.fedavg([123])
+    torch.cuda.synchronize()
+    assert torch.equal(snap[0], c.sess.master[0]) and torch.equal(snap[1], c.sess.m[0]) and torch.equal(snap[2], c.sess.v[0])
+    c.close()
+    c = Case([5000], 4, 2, 1, H=1, Q=8)
+    c.step([3, 1, 4, 1])
+    once = c.sess.master[0].clone()
+    c.sess.fedavg([3, 1, 4, 1])                   # identical copies: identity up to the rounding of sum(w)
+    torch.cuda.synchronize()
+    assert torch.allclose(once, c.sess.master[0], rtol=2e-7, atol=0)
+    c.close()
+
+
+# ------------------------------------------------------------------ whole-loop properties
+def test_h1_equal_weights_equals_fsdp_over_all_replicas(fls):
+    """Same mean gradient in every group (group g reads group 0's buffers rotated by g): FL+FSDP with
+    H = 1, equal weights and averaged optimizer state matches one FSDP group over all R*G buffers."""
+    R, G, P = 4, 3, 20000
+    fl = Case([P], G, R, 1, H=1, Q=8, opt_state=True, hp=orc.Hyper(max_grad_norm=0.02))
+    big = Case([P], 1, R * G, 1, H=10 ** 6, Q=8, hp=orc.Hyper(max_grad_norm=0.02))
+    base = lambda t, k: fl.grad_logical(t, 0, k)
+    for _ in range(3):
+        fl.step(None, override=lambda t, g, k: base(t, (k + g) % R))
+        big.step(None, override=lambda t, g, k: base(t, k % R))
+    a, b = fl.sess.master[0].cpu().numpy(), big.sess.master[0].cpu().numpy()
+    assert_state_close(a, b, "fl vs fsdp master")
+    assert_state_close(fl.sess.m[2].cpu().numpy(), big.sess.m[0].cpu().numpy(), "m", 1e-5, 1e-12)
+    fl.close(); big.close()
+
+
+def test_determinism_and_resume(fls):
+    def run(split):
+        c = Case([50000, 1234], 2, 4, 1, H=2, Q=8, opt_state=True, hp=orc.Hyper(max_grad_norm=0.02))
+        for t in range(4):
+            if split and t == 2:       # checkpoint: a new plan over the same tensors, step counter restored
+                from paper_2609_20359_b200 import _binding as b
+                old = c.sess.plan
+                c.sess.plan = b.fls_plan_create(c.P, c.units, 2, 4, 1, 2, b.FLS_GRAD_BF16, 8, 3, c.hp.lr, c.hp.beta1, c.hp.beta2,
+                                                c.hp.eps, c.hp.weight_decay, c.hp.max_grad_norm)
+                b.fls_plan_destroy(old)
+                c.sess.bind()
+                b.fls_set_step(c.sess.plan, 2)
+            c.step()
+        out = [x.clone() for x in c.sess.master + c.sess.m + c.sess.v + c.sess.param_bf16]
+        c.close()
+        return out
+    a, b, r = run(False), run(False), run(True)
+    assert all(torch.equal(x, y) for x, y in zip(a, b)), "two identical runs differ"
+    assert all(torch.equal(x, y) for x, y in zip(a, r)), "resume from a checkpoint differs"
+
+
+def test_padding_stays_zero_and_q_does_not_change_logical_results(fls):
+    outs = []
+    for Q in (1, 8, 64):
+        c = Case([1000, 37, 4001], 2, 4, 1, H=2, Q=Q, hp=orc.Hyper(max_grad_norm=0.02))
+        for _ in range(2):
+            c.step()
+        c.compare()
+        pad = np.ones(c.L.n_padded, bool); pad[orc._addresses(c.L)[1]] = False
+        assert not c.sess.master[0].cpu().numpy()[pad].any() and not c.sess.v[1].cpu().numpy()[pad].any()
+        outs.append(orc.unpack_sharded(c.L, c.sess.master[0].cpu().numpy()))
+        c.close()
+    # the vector and element-wise paths use the same fp32 operations: identical logical results
+    assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[1], outs[2])
+
+
+def test_lr_override_and_clip_disabled(fls):
+    c = Case([30000], 1, 2, 1, H=100, Q=8, hp=orc.Hyper(max_grad_norm=0.0))
+    c.step(lr=1e-3)
+    c.step(lr=0.0)
+    c.compare()
+    assert c.sess.coefs().cpu().tolist() == [1.0]
+    c.close()
+
+
+def test_nonfinite_gradients_propagate_and_set_status(fls):
+    c = Case([10000], 2, 2, 1, H=100, Q=8)
+    def poisoned(t, g, k):
+        x = c.grad_logical(t, g, k)
+        if g == 1 and k == 0:
+            x[77] = float("inf")
+        return x
+    c.step(override=poisoned)
+    assert c.sess.status() & 1
+    assert math.isinf(c.sess.norms()[1].item()) and c.sess.coefs()[1].item() == 0.0
+    th1 = c.sess.master[1].cpu().numpy()
+    assert np.isnan(th1[77]) and np.isfinite(np.delete(th1, 77)).all()      # 0 * inf = NaN only where the inf was
+    assert np.isfinite(c.sess.master[0].cpu().numpy()).all()                 # the other group is untouched
+    c.close()
+
+
+def test_step_from_host_buffers_matches_device_step(fls):
+    a = Case([50000, 777], 2, 2, 2, H=2, Q=8, hp=orc.Hyper(max_grad_norm=0.02))
+    b = Case([50000, 777], 2, 2, 2, H=2, Q=8, hp=orc.Hyper(max_grad_norm=0.02))
+    for t in range(1, 3):
+        a.step()
+        host = [[torch.from_numpy(orc.pack_unsharded(b.L, bf16_bits(b.grad_logical(t, g, k)).view(np.int16))).view(torch.bfloat16).pin_memory()
+                 for k in range(b.K)] for g in range(b.G)]
+        norms = torch.zeros(b.G, dtype=torch.float32)
+        due = b.sess.step_host(host, host_norms=norms)
+        if due:
+            b.sess.fedavg(None)
+        torch.cuda.synchronize()
+        assert torch.equal(norms, a.sess.norms().cpu())
+    for x, y in zip(a.sess.master + a.sess.v + a.sess.param_bf16, b.sess.master + b.sess.v + b.sess.param_bf16):
+        assert torch.equal(x, y)
+    a.close(); b.close()
+
+
+# ------------------------------------------------------------------ argument errors that need a device
+def test_bind_rejects_bad_buffers(fls):
+    from paper_2609_20359_b200.session import Session
+    s = Session(4096, None, groups=2, shard_dim=2, align_elems=8)
+    flat = [t for row in s.grads for t in row]
+    def bind(grads=flat, master=s.master, m=s.m, v=s.v, pb=s.param_bf16, ws=s.workspace, ws_bytes=None):
+        fls.fls_plan_bind(s.plan, grads, master, m, v, pb, ws, ws_bytes)
+    with pytest.raises(fls.FlsError) as e:
+        bind(master=[s.master[0], torch.zeros(4096)])                       # host memory
+    assert e.value.code == fls.FLS_EPTR
+    with pytest.raises(fls.FlsError) as e:
+        bind(m=[s.m[0], s.m[1].view(torch.uint8)[4:].view(torch.float32)])  # misaligned
+    assert e.value.code == fls.FLS_EALIGN
+    with pytest.raises(fls.FlsError) as e:
+        bind(ws_bytes=1024)
+    assert e.value.code == fls.FLS_ESIZE
+    with pytest.raises(fls.FlsError) as e:
+        bind(v=[s.v[0], s.v[0]])                                            # two outputs alias
+    assert e.value.code == fls.FLS_EPTR
+    with pytest.raises(fls.FlsError) as e:
+        bind(grads=[s.master[0].view(torch.bfloat16)[:4096]] + flat[1:])    # a gradient aliases an output
+    assert e.value.code == fls.FLS_EPTR
+    with pytest.raises(fls.FlsError) as e:
+        bind(master=[s.master[0], 0])
+    assert e.value.code == fls.FLS_EPTR
+    bind(grads=[flat[0]] * len(flat))                                       # inputs may be shared
+    bind()
+    s.step(); torch.cuda.synchronize()
+    s.close()
+
+
+# ------------------------------------------------------------------ full size, in the benchmark's launch configuration
+def test_full_size_gpt2_small_sampled(fls):
+    """P = 124,439,808, G = 4, K = 8 (the benchmark workload).  The oracle computes every group's
+    norm over the full gradient (chunked), then the step and FedAvg at sampled positions: first and
+    last tiles, tile and shard boundaries, and random indices."""
+    from paper_2609_20359_b200.session import Session
+    cfg = sy.CONFIGS[1]
+    P, G, K = cfg["n_params"], cfg["groups"], cfg["shard_dim"]
+    hp = orc.Hyper()
+    s = Session(P, cfg["unit_numel"], G, K, 1, cfg["sync_period"], "bf16", 8, False)
+    th_key = sy.stream_key(cfg["seed"], sy.KIND_MASTER)
+    for g in range(G):
+        sy.normal_fill_(s.master[g], th_key, cfg["master_sigma"])
+        for k in range(K):
+            sy.normal_fill_(s.grads[g][k], sy.stream_key(cfg["seed"], sy.KIND_GRAD, 1, g, k), cfg["grad_sigma"],
+                            sy.uniform_scale(cfg["seed"], g, k))
+    counts = [sy.sample_count(cfg["seed"], g) for g in range(G)]
+    rng = np.random.default_rng(3)
+    idx = np.unique(np.concatenate([np.arange(0, 4096), np.arange(P - 4096, P), rng.integers(0, P, 200_000),
+                                    (np.arange(1, K)[:, None] * (P // K) + np.arange(-8, 8)[None, :]).ravel()]))
+    tidx = torch.from_numpy(idx)
+    th0 = sy.normal_at(tidx, th_key, cfg["master_sigma"]).numpy()
+    # oracle norms over the full buffers (gradients come from the generator, copied to the host)
+    norms, gbar_s = [], []
+    CH = 1 << 23
+    for g in range(G):
+        tot = 0.0
+        for lo in range(0, P, CH):
+            chunk = [orc.bf16_bits_to_f64(bf16_bits(s.grads[g][k][lo:lo + CH])) for k in range(K)]
+            gb = orc.reduce_mean(chunk, K, 1)
+            tot += orc.grad_norm(gb) ** 2
+        norms.append(math.sqrt(tot))
+        samp = [orc.bf16_bits_to_f64(bf16_bits(sy.normal_at(tidx, sy.stream_key(cfg["seed"], sy.KIND_GRAD, 1, g, k), cfg["grad_sigma"],
+                                                             sy.uniform_scale(cfg["seed"], g, k), torch.bfloat16))) for k in range(K)]
+        gbar_s.append(orc.reduce_mean(samp, K, 1))
+    due = s.step()
+    torch.cuda.synchronize()
+    assert not due
+    got_n = s.norms().cpu().numpy().astype(np.float64)
+    assert np.allclose(got_n, norms, rtol=1e-6, atol=0), (got_n, norms)
+    assert np.array_equal(s.reduced_grad()[tidx.cuda()].cpu().numpy(), gbar_s[G - 1])
+    states = []
+    for g in range(G):
+        c = orc.clip_coef(norms[g], hp.max_grad_norm)
+        assert c < 1.0
+        z = np.zeros(idx.size, np.float32)
+        th, m, v, bits = orc.adamw(th0, z, z, gbar_s[g], c, 1, hp.lr, hp.beta1, hp.beta2, hp.eps, hp.weight_decay)
+        states.append(orc.GroupState(th, m, v, bits))
+        assert_state_close(s.master[g][tidx.cuda()].cpu().numpy(), th, f"master[{g}]")
+        assert_state_close(s.m[g][tidx.cuda()].cpu().numpy(), m, f"m[{g}]", 1e-5, 1e-12)
+        assert_state_close(s.v[g][tidx.cuda()].cpu().numpy(), v, f"v[{g}]", 1e-5, 1e-18)
+        assert_bf16_close(bf16_bits(s.param_bf16[g][tidx.cuda()]), bits, f"bf16[{g}]")
+    orc.fedavg(states, counts)
+    s.fedavg(counts)
+    torch.cuda.synchronize()
+    for g in range(G):
+        assert_state_close(s.master[g][tidx.cuda()].cpu().numpy(), states[g].theta, f"fedavg master[{g}]")
+        assert_bf16_close(bf16_bits(s.param_bf16[g][tidx.cuda()]), states[g].param_bf16, f"fedavg bf16[{g}]")
+    assert torch.equal(s.master[0], s.master[G - 1])
+    s.close()
