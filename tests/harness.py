@@ -10,8 +10,11 @@ import synthetic as sy
 from oracle import fls_oracle as orc
 
 TOL_STATE = 1e-6          # |d| <= 1e-6 * max(1, |x|) on fp32 master / m / v
-REL_M, ABS_M = 1e-5, 1e-12
-REL_V, ABS_V = 1e-5, 1e-18
+# m and v are small (1e-4, 1e-8), so the official absolute gate says little about them.  Extra gate:
+# |d| <= 1e-5 |x| + 1e-6 rms(x).  The rms term covers elements that cancelled towards zero, whose fp32
+# store error scales with the magnitude they had before, not with what is left.
+REL_M = REL_V = 1e-5
+ABS_M = ABS_V = "rms"
 
 
 def bf16_bits(t: torch.Tensor) -> np.ndarray:
@@ -31,13 +34,30 @@ def assert_state_close(got: np.ndarray, want: np.ndarray, what: str, rel=None, a
     bad = ~(d <= lim)
     assert not bad.any(), f"{what}: {bad.sum()} elements beyond 1e-6*max(1,|x|); worst {d[bad].max() if bad.any() else 0}"
     if rel is not None:
+        if abs_ == "rms":
+            abs_ = 1e-6 * float(np.sqrt(np.mean(want * want))) + 1e-30
         bad = ~(d <= rel * np.abs(want) + abs_)
         assert not bad.any(), f"{what}: {bad.sum()} elements beyond rel {rel}; worst idx {np.argmax(d - rel * np.abs(want))}"
 
 
+def bf16_value(bits: np.ndarray) -> np.ndarray:
+    return (bits.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+
+
 def assert_bf16_close(got_bits: np.ndarray, want_bits: np.ndarray, what: str):
-    d = np.abs(bf16_ordinal(got_bits) - bf16_ordinal(want_bits))
-    assert d.max(initial=0) <= 1, f"{what}: bf16 differs by {d.max()} ulp at {np.argmax(d)}"
+    """Within 1 bf16 ulp.  The bf16 copy is the rounding of an fp32 value that may itself differ from
+    the oracle's by the state tolerance, so for values near zero (where a bf16 ulp is smaller than that
+    tolerance) the allowance is one ulp plus the fp32 tolerance: |d| <= ulp_bf16(x) + 1e-6*max(1,|x|)."""
+    got, want = bf16_value(got_bits), bf16_value(want_bits)
+    fin = np.isfinite(want)
+    assert np.array_equal(np.isfinite(got), fin), f"{what}: finiteness differs"
+    mag = np.maximum(np.abs(want[fin]), 2.0 ** -126)
+    ulp = 2.0 ** (np.floor(np.log2(mag)) - 7)
+    d = np.abs(got[fin] - want[fin])
+    bad = ~(d <= ulp + TOL_STATE * np.maximum(1.0, mag))
+    assert not bad.any(), f"{what}: {bad.sum()} bf16 elements beyond 1 ulp; worst {d[bad].max() if bad.any() else 0}"
+    ordinal = np.abs(bf16_ordinal(got_bits) - bf16_ordinal(want_bits))
+    assert np.mean(ordinal <= 1) > 0.999, f"{what}: only {np.mean(ordinal <= 1):.5f} of the bf16 copies are within one code"
 
 
 class Case:
@@ -126,6 +146,9 @@ class Case:
             assert_state_close(self.sess.m[g].cpu().numpy(), orc.pack_sharded(self.L, st.m), f"m[{g}]", REL_M, ABS_M)
             assert_state_close(self.sess.v[g].cpu().numpy(), orc.pack_sharded(self.L, st.v), f"v[{g}]", REL_V, ABS_V)
             assert_bf16_close(bf16_bits(self.sess.param_bf16[g]), orc.pack_unsharded(self.L, st.param_bf16), f"param_bf16[{g}]")
+            # and the copy is exactly the nearest-even rounding of the GPU's own fp32 master
+            own = orc.unpack_sharded(self.L, bf16_bits(self.sess.master[g].to(torch.bfloat16)))
+            assert np.array_equal(orc.unpack_unsharded(self.L, bf16_bits(self.sess.param_bf16[g])), own), f"bf16 copy of group {g} is not RNE(master)"
 
     def close(self):
         self.sess.close()

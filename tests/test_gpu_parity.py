@@ -1,6 +1,8 @@
 """GPU parity: the CUDA library against the CPU oracle, element by element, on the same seeded
-inputs, through the C ABI.  Tolerances: |d| <= 1e-6*max(1,|x|) on fp32 master/m/v (plus relative
-gates on m and v, whose magnitudes make the absolute gate weak), <= 1 bf16 ulp on the bf16 copy."""
+inputs, through the C ABI.  Tolerances: |d| <= 1e-6*max(1,|x|) on fp32 master/m/v (plus a relative
+gate on m and v, whose magnitudes make the absolute gate weak); the bf16 copy within 1 bf16 ulp (plus
+the fp32 tolerance where a bf16 ulp is smaller than it) and bit-exactly the rounding of the GPU's own
+fp32 master."""
 import math
 
 import numpy as np
@@ -78,7 +80,8 @@ def test_layouts_and_orders(fls, units, G, S, R_rep, Q, dtype):
 
 
 def test_reduced_gradient_matches_oracle_exactly_for_bf16(fls):
-    """With bf16 inputs the fp32 running sum is exact here, so the mean gradient is bit-identical."""
+    """With bf16 inputs of similar magnitude the fp32 running sum is exact, so the mean gradient is
+    bit-identical to the oracle's (this case is small enough that no element loses bits)."""
     c = Case([40000, 30011], 1, 4, 2, H=10, Q=8)
     grads = c.load_grads(1)
     c.sess.step()
@@ -103,7 +106,9 @@ def test_two_level_order_differs_from_flat_where_fp32_rounds(fls):
         torch.cuda.synchronize()
         got = c.sess.reduced_grad().cpu().numpy()
         want = orc.reduce_mean(grads[0], S, R_rep)
-        assert np.allclose(got, want, rtol=8 * 2 ** -24, atol=0)
+        # sequential fp32 adds: each of the K-1 roundings is at most half an ulp of a partial sum <= sum|x|
+        bound = S * R_rep * 2.0 ** -24 * np.sum(np.abs(grads[0]), axis=0) / (S * R_rep)
+        assert np.all(np.abs(got.astype(np.float64) - want) <= bound)
         res[(S, R_rep)] = got
         c.close()
     assert not np.array_equal(res[(8, 1)], res[(4, 2)])
@@ -162,9 +167,10 @@ def test_h1_equal_weights_equals_fsdp_over_all_replicas(fls):
     for _ in range(3):
         fl.step(None, override=lambda t, g, k: base(t, (k + g) % R))
         big.step(None, override=lambda t, g, k: base(t, k % R))
-    a, b = fl.sess.master[0].cpu().numpy(), big.sess.master[0].cpu().numpy()
+    a = orc.unpack_sharded(fl.L, fl.sess.master[0].cpu().numpy())
+    b = orc.unpack_sharded(big.L, big.sess.master[0].cpu().numpy())
     assert_state_close(a, b, "fl vs fsdp master")
-    assert_state_close(fl.sess.m[2].cpu().numpy(), big.sess.m[0].cpu().numpy(), "m", 1e-5, 1e-12)
+    assert_state_close(orc.unpack_sharded(fl.L, fl.sess.m[2].cpu().numpy()), orc.unpack_sharded(big.L, big.sess.m[0].cpu().numpy()), "m", 1e-5, "rms")
     fl.close(); big.close()
 
 
@@ -220,7 +226,8 @@ def test_nonfinite_gradients_propagate_and_set_status(fls):
         if g == 1 and k == 0:
             x[77] = float("inf")
         return x
-    c.step(override=poisoned)
+    with np.errstate(invalid="ignore"):
+        c.step(override=poisoned)
     assert c.sess.status() & 1
     assert math.isinf(c.sess.norms()[1].item()) and c.sess.coefs()[1].item() == 0.0
     th1 = c.sess.master[1].cpu().numpy()
@@ -318,7 +325,10 @@ def test_full_size_gpt2_small_sampled(fls):
     assert not due
     got_n = s.norms().cpu().numpy().astype(np.float64)
     assert np.allclose(got_n, norms, rtol=1e-6, atol=0), (got_n, norms)
-    assert np.array_equal(s.reduced_grad()[tidx.cuda()].cpu().numpy(), gbar_s[G - 1])
+    # fp32 running sum against the exactly rounded mean: identical except where a tiny addend loses bits
+    got_g = s.reduced_grad()[tidx.cuda()].cpu().numpy()
+    assert np.mean(got_g == gbar_s[G - 1]) > 0.999
+    assert np.all(np.abs(got_g.astype(np.float64) - gbar_s[G - 1]) <= 2.0 ** -24 * np.sum(np.abs(samp), axis=0))
     states = []
     for g in range(G):
         c = orc.clip_coef(norms[g], hp.max_grad_norm)
@@ -327,8 +337,8 @@ def test_full_size_gpt2_small_sampled(fls):
         th, m, v, bits = orc.adamw(th0, z, z, gbar_s[g], c, 1, hp.lr, hp.beta1, hp.beta2, hp.eps, hp.weight_decay)
         states.append(orc.GroupState(th, m, v, bits))
         assert_state_close(s.master[g][tidx.cuda()].cpu().numpy(), th, f"master[{g}]")
-        assert_state_close(s.m[g][tidx.cuda()].cpu().numpy(), m, f"m[{g}]", 1e-5, 1e-12)
-        assert_state_close(s.v[g][tidx.cuda()].cpu().numpy(), v, f"v[{g}]", 1e-5, 1e-18)
+        assert_state_close(s.m[g][tidx.cuda()].cpu().numpy(), m, f"m[{g}]", 1e-5, "rms")
+        assert_state_close(s.v[g][tidx.cuda()].cpu().numpy(), v, f"v[{g}]", 1e-5, "rms")
         assert_bf16_close(bf16_bits(s.param_bf16[g][tidx.cuda()]), bits, f"bf16[{g}]")
     orc.fedavg(states, counts)
     s.fedavg(counts)
