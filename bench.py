@@ -294,8 +294,18 @@ def main():
     ap.add_argument("--ctas-adamw", type=int, default=0)
     ap.add_argument("--ctas-fedavg", type=int, default=0)
     ap.add_argument("--descending-adamw", action="store_true")
+    # slices of a workload, for profiler captures that must stay small (same kernels, fewer bytes)
+    ap.add_argument("--n-params", type=int, default=0, help="override P (single flat unit)")
+    ap.add_argument("--groups", type=int, default=0, help="override G")
+    ap.add_argument("--sync-period", type=int, default=0, help="override H")
     args = ap.parse_args()
     cfg = sy.config_by_name(args.config)
+    if args.n_params:
+        cfg.update(n_params=args.n_params, unit_numel=[args.n_params], name=cfg["name"] + f"[P={args.n_params}]")
+    if args.groups:
+        cfg.update(groups=args.groups, name=cfg["name"] + f"[G={args.groups}]")
+    if args.sync_period:
+        cfg.update(sync_period=args.sync_period, name=cfg["name"] + f"[H={args.sync_period}]")
     if args.impl == "reference":
         run_reference(args, cfg)
     else:

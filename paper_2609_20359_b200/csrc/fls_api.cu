@@ -45,7 +45,9 @@ struct fls_plan {
   std::vector<uint64_t> units;
   Layout lay;
   uint32_t K = 0;
-  uint64_t start_mask = 0, end_mask = 0;
+  uint64_t end_mask = 0;
+  uint32_t fold_mask = 0;
+  int reduce_sg = -1;
 
   bool bound = false;
   int device = -1;
@@ -57,7 +59,7 @@ struct fls_plan {
 
   uint64_t step = 0;
   uint64_t launches = 0;
-  int ctas_per_sm[FLS_KERNEL_COUNT] = {4, 4, 2};
+  int ctas_per_sm[FLS_KERNEL_COUNT] = {2, 2, 2};
   int descending[FLS_KERNEL_COUNT] = {0, 0, 0};
 
   bool profiling = false;
@@ -135,7 +137,9 @@ int run_group(fls_plan* p, uint32_t g, double lr, uint64_t t_new, cudaStream_t s
   ra.K = p->K;
   ra.S = d.shard_dim;
   ra.k_float = float(p->K);
-  ra.start_mask = p->start_mask;
+  ra.inv_k = 1.0f / float(p->K);
+  ra.k_is_pow2 = (p->K & (p->K - 1)) == 0 ? 1u : 0u;
+  ra.fold_mask = p->fold_mask;
   ra.end_mask = p->end_mask;
   ra.partials = p->d_partials();
   ra.ticket = p->d_ticket();
@@ -147,7 +151,7 @@ int run_group(fls_plan* p, uint32_t g, double lr, uint64_t t_new, cudaStream_t s
   ra.descending = p->descending[FLS_KERNEL_REDUCE];
   const bool f32 = d.grad_dtype == FLS_GRAD_F32;
   cudaError_t e = timed_launch(p, FLS_KERNEL_REDUCE, st,
-                               [&] { return launch_reduce(ra, f32, p->grid_for(FLS_KERNEL_REDUCE), st); });
+                               [&] { return launch_reduce(ra, f32, p->reduce_sg, p->grid_for(FLS_KERNEL_REDUCE), st); });
   if (e != cudaSuccess) return cuda_fail(e, "reduce kernel launch");
 
   // Scalars of the AdamW step, in double on the host, handed to the kernel as fp32.
@@ -232,9 +236,18 @@ int fls_plan_create(const fls_plan_desc* desc, fls_plan** out) {
     return fail(FLS_EINVAL, "layout: %s", msg.c_str());
   }
   p->K = uint32_t(K);
-  for (uint32_t k = 0; k < p->K; ++k) {
-    if (k % d.shard_dim == 0) p->start_mask |= 1ull << k;
+  // level structure of the gradient reduction: which buffers / batches of 8 close a sharding group
+  for (uint32_t k = 0; k < p->K; ++k)
     if (k % d.shard_dim == d.shard_dim - 1) p->end_mask |= 1ull << k;
+  const uint32_t S = d.shard_dim;
+  if (d.replicate_dim == 1 || S % 8 == 0) {
+    p->reduce_sg = 0;
+    for (uint32_t k0 = 0; k0 < p->K; k0 += 8)
+      if (std::min(k0 + 8, p->K) % S == 0) p->fold_mask |= 1u << (k0 / 8);
+  } else if (S == 1 || S == 2 || S == 4) {
+    p->reduce_sg = int(S);
+  } else {
+    p->reduce_sg = -1;
   }
   *out = p;
   return FLS_OK;

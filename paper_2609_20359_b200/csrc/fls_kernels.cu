@@ -3,12 +3,12 @@
 // (bf16) and 256-bit (fp32) global accesses.  No shared-memory staging and no tensor cores: nothing
 // here is a contraction, and each byte is touched once.
 //
-//   reduce_kernel  : K gradient buffers -> mean gradient (fp32, shard order) + squared-norm partials;
+//   fls_reduce_kernel  : K gradient buffers -> mean gradient (fp32, shard order) + squared-norm partials;
 //                    the last CTA to finish adds the partials in index order and writes the group's
 //                    norm and clip coefficient (no floating-point atomics: the result does not depend
 //                    on which CTA is last).
-//   adamw_kernel   : clip + AdamW on master/m/v in place + bf16 copy in unsharded order.
-//   fedavg_kernel  : weighted average of G copies written back to all G (+ bf16 copies).
+//   fls_adamw_kernel   : clip + AdamW on master/m/v in place + bf16 copy in unsharded order.
+//   fls_fedavg_kernel  : weighted average of G copies written back to all G (+ bf16 copies).
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -153,8 +153,14 @@ __device__ __forceinline__ void unpack(const Raw<1, true>& x, float (&f)[1]) { f
 // Mean of the K buffers at elements j .. j+N-1.  Buffers are consumed in ascending index k = rho*S +
 // sigma, eight loads in flight at a time.  `inner` is the running sum of the current sharding group
 // (the reduce-scatter level); when the group's last buffer has been added it is folded into `outer`
-// (the all-reduce level across replicas).  The first addend of each level initialises it.
-template <int N, bool F32>
+// (the all-reduce level across replicas).  Both start at zero, so every level is a plain ascending
+// sum (0 + x is exact).  SG fixes the level structure at compile time so the hot loop holds only
+// unpack + add:
+//   SG =  0 : every batch of 8 lies inside one sharding group (FSDP, or S a multiple of 8); bit i of
+//             fold_mask says that batch i closes a group.
+//   SG = 1, 2, 4 : S == SG, a batch holds 8/SG whole groups.
+//   SG = -1 : any other shape; bit k of end_mask says that buffer k closes a group.
+template <int N, bool F32, int SG>
 __device__ __forceinline__ void reduce_elems(const ReduceArgs& a, uint64_t j, float (&mean)[N]) {
   float inner[N], outer[N];
 #pragma unroll
@@ -164,28 +170,66 @@ __device__ __forceinline__ void reduce_elems(const ReduceArgs& a, uint64_t j, fl
 #pragma unroll
     for (int b = 0; b < 8; ++b)
       if (k0 + b < a.K) load_raw(raw[b], a.grad[k0 + b], j);
+    if constexpr (SG == 0) {
 #pragma unroll
-    for (int b = 0; b < 8; ++b) {
-      const uint32_t k = k0 + b;
-      if (k < a.K) {
-        float x[N];
-        unpack(raw[b], x);
-        const bool first = (a.start_mask >> k) & 1ull, last = (a.end_mask >> k) & 1ull;
+      for (int b = 0; b < 8; ++b) {
+        if (k0 + b < a.K) {
+          float x[N];
+          unpack(raw[b], x);
 #pragma unroll
-        for (int e = 0; e < N; ++e) inner[e] = first ? x[e] : inner[e] + x[e];
-        if (last) {
+          for (int e = 0; e < N; ++e) inner[e] += x[e];
+        }
+      }
+      if ((a.fold_mask >> (k0 >> 3)) & 1u) {
 #pragma unroll
-          for (int e = 0; e < N; ++e) outer[e] = (k < a.S) ? inner[e] : outer[e] + inner[e];
+        for (int e = 0; e < N; ++e) { outer[e] += inner[e]; inner[e] = 0.f; }
+      }
+    } else if constexpr (SG > 0) {
+#pragma unroll
+      for (int g0 = 0; g0 < 8; g0 += SG) {
+        if (k0 + g0 < a.K) {
+          float s[N];
+          unpack(raw[g0], s);
+#pragma unroll
+          for (int i = 1; i < SG; ++i) {
+            float x[N];
+            unpack(raw[g0 + i], x);
+#pragma unroll
+            for (int e = 0; e < N; ++e) s[e] += x[e];
+          }
+#pragma unroll
+          for (int e = 0; e < N; ++e) outer[e] += s[e];
+        }
+      }
+    } else {
+#pragma unroll
+      for (int b = 0; b < 8; ++b) {
+        const uint32_t k = k0 + b;
+        if (k < a.K) {
+          float x[N];
+          unpack(raw[b], x);
+#pragma unroll
+          for (int e = 0; e < N; ++e) inner[e] += x[e];
+          if ((a.end_mask >> k) & 1ull) {
+#pragma unroll
+            for (int e = 0; e < N; ++e) { outer[e] += inner[e]; inner[e] = 0.f; }
+          }
         }
       }
     }
   }
+  // one scaling by 1/K after the last level: a multiply when 1/K is exact, else an IEEE division
+  if (a.k_is_pow2) {
 #pragma unroll
-  for (int e = 0; e < N; ++e) mean[e] = __fdiv_rn(outer[e], a.k_float);
+    for (int e = 0; e < N; ++e) mean[e] = outer[e] * a.inv_k;
+  } else {
+#pragma unroll
+    for (int e = 0; e < N; ++e) mean[e] = __fdiv_rn(outer[e], a.k_float);
+  }
 }
 
-template <bool F32>
-__global__ void __launch_bounds__(kThreads) reduce_kernel(const __grid_constant__ ReduceArgs a) {
+template <bool F32, int SG>
+__global__ void __launch_bounds__(kThreads, 2) fls_reduce_kernel(const __grid_constant__ ReduceArgs a) {
   __shared__ double sh[kThreads / 32];
   __shared__ bool is_last;
   double dsum = 0.0;
@@ -198,7 +242,7 @@ __global__ void __launch_bounds__(kThreads) reduce_kernel(const __grid_constant_
       const Slice s = slice_of(w.cur, tile);
       if (s.vec) {
         float g[8];
-        reduce_elems<8, F32>(a, s.j, g);
+        reduce_elems<8, F32, SG>(a, s.j, g);
         F8 o;
         float sq = 0.f;
 #pragma unroll
@@ -208,7 +252,7 @@ __global__ void __launch_bounds__(kThreads) reduce_kernel(const __grid_constant_
       } else {
         for (uint32_t e = 0; e < s.n; ++e) {
           float g[1];
-          reduce_elems<1, F32>(a, s.j + e, g);
+          reduce_elems<1, F32, -1>(a, s.j + e, g);
           a.gbar[s.a + e] = g[0];
           dsum += double(g[0] * g[0]);
         }
@@ -256,7 +300,7 @@ __device__ __forceinline__ void adamw_one(const AdamArgs& a, float c, float gbar
   th = fmaf(-a.step_size, __fdiv_rn(m, denom), th);         // step_size = lr / (1 - beta1^t)
 }
 
-__global__ void __launch_bounds__(kThreads) adamw_kernel(const __grid_constant__ AdamArgs a) {
+__global__ void __launch_bounds__(kThreads, 3) fls_adamw_kernel(const __grid_constant__ AdamArgs a) {
   if (blockIdx.x >= a.n_tiles) return;
   const float c = __ldcg(a.coef);
   Walker w;
@@ -293,7 +337,7 @@ __global__ void __launch_bounds__(kThreads) adamw_kernel(const __grid_constant__
 // ------------------------------------------------------------------------------------------------
 // K3: FedAvg.  x_bar = sum_g w_g x_g, ascending g, written to all G copies.
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kThreads) fedavg_kernel(const __grid_constant__ FedavgArgs a) {
+__global__ void __launch_bounds__(kThreads, 2) fls_fedavg_kernel(const __grid_constant__ FedavgArgs a) {
   if (blockIdx.x >= a.n_tiles) return;
   Walker w;
   w.init(a.segs, a.n_seg, a.descending);
@@ -316,7 +360,7 @@ __global__ void __launch_bounds__(kThreads) fedavg_kernel(const __grid_constant_
           if (g < a.G) {
             const float wg = a.w[g];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) acc.v[e] = (g == 0) ? wg * raw[b].v[e] : fmaf(wg, raw[b].v[e], acc.v[e]);
+            for (int e = 0; e < 8; ++e) acc.v[e] = fmaf(wg, raw[b].v[e], acc.v[e]);   // acc starts at 0: the first term is w_0 x_0
           }
         }
       }
@@ -332,7 +376,7 @@ __global__ void __launch_bounds__(kThreads) fedavg_kernel(const __grid_constant_
         float acc = 0.f;
         for (uint32_t g = 0; g < a.G; ++g) {
           const float x = a.x[g][s.a + e];
-          acc = (g == 0) ? a.w[g] * x : fmaf(a.w[g], x, acc);
+          acc = fmaf(a.w[g], x, acc);
         }
         for (uint32_t g = 0; g < a.G; ++g) a.x[g][s.a + e] = acc;
         if (a.write_bf16) {
@@ -346,21 +390,32 @@ __global__ void __launch_bounds__(kThreads) fedavg_kernel(const __grid_constant_
 
 }  // namespace
 
-cudaError_t launch_reduce(const ReduceArgs& a, bool f32, unsigned grid, cudaStream_t st) {
+template <bool F32>
+static void launch_reduce_t(const ReduceArgs& a, int sg, unsigned grid, cudaStream_t st) {
+  switch (sg) {
+    case 0: fls_reduce_kernel<F32, 0><<<grid, kThreads, 0, st>>>(a); break;
+    case 1: fls_reduce_kernel<F32, 1><<<grid, kThreads, 0, st>>>(a); break;
+    case 2: fls_reduce_kernel<F32, 2><<<grid, kThreads, 0, st>>>(a); break;
+    case 4: fls_reduce_kernel<F32, 4><<<grid, kThreads, 0, st>>>(a); break;
+    default: fls_reduce_kernel<F32, -1><<<grid, kThreads, 0, st>>>(a); break;
+  }
+}
+
+cudaError_t launch_reduce(const ReduceArgs& a, bool f32, int sg, unsigned grid, cudaStream_t st) {
   if (f32)
-    reduce_kernel<true><<<grid, kThreads, 0, st>>>(a);
+    launch_reduce_t<true>(a, sg, grid, st);
   else
-    reduce_kernel<false><<<grid, kThreads, 0, st>>>(a);
+    launch_reduce_t<false>(a, sg, grid, st);
   return cudaGetLastError();
 }
 
 cudaError_t launch_adamw(const AdamArgs& a, unsigned grid, cudaStream_t st) {
-  adamw_kernel<<<grid, kThreads, 0, st>>>(a);
+  fls_adamw_kernel<<<grid, kThreads, 0, st>>>(a);
   return cudaGetLastError();
 }
 
 cudaError_t launch_fedavg(const FedavgArgs& a, unsigned grid, cudaStream_t st) {
-  fedavg_kernel<<<grid, kThreads, 0, st>>>(a);
+  fls_fedavg_kernel<<<grid, kThreads, 0, st>>>(a);
   return cudaGetLastError();
 }
 

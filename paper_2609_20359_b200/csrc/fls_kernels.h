@@ -13,8 +13,10 @@ struct ReduceArgs {
   uint64_t n_tiles;
   uint32_t n_seg;
   uint32_t K, S;
-  float k_float;                           // K as float: the mean divides by it once
-  uint64_t start_mask, end_mask;           // bit k set: buffer k opens / closes a sharding group
+  float k_float, inv_k;                    // K and 1/K as float: the mean is scaled by 1/K once
+  uint32_t k_is_pow2;                      // 1/K exact: multiply; otherwise divide
+  uint32_t fold_mask;                      // bit i set: the i-th batch of 8 buffers closes a sharding group
+  uint64_t end_mask;                       // bit k set: buffer k closes a sharding group
   double* partials;                        // device, one per CTA
   uint32_t* ticket;                        // device, zero between launches
   float* norm_out;
@@ -49,7 +51,8 @@ struct FedavgArgs {
   int descending;
 };
 
-cudaError_t launch_reduce(const ReduceArgs& a, bool f32, unsigned grid, cudaStream_t st);
+// sg: level structure of the reduction (see reduce_elems): 0, 1, 2, 4 or -1 for the generic form
+cudaError_t launch_reduce(const ReduceArgs& a, bool f32, int sg, unsigned grid, cudaStream_t st);
 cudaError_t launch_adamw(const AdamArgs& a, unsigned grid, cudaStream_t st);
 cudaError_t launch_fedavg(const FedavgArgs& a, unsigned grid, cudaStream_t st);
 
