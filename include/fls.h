@@ -49,6 +49,7 @@ enum { FLS_STATUS_NONFINITE_NORM = 1 };             /* sticky bits of the device
 #define FLS_MAX_GROUPS 64        /* G <= 64 */
 #define FLS_MAX_GRAD_BUFFERS 64  /* K = shard_dim * replicate_dim <= 64 */
 #define FLS_BUFFER_ALIGN 32      /* every device buffer must start on a 32-byte boundary */
+#define FLS_NOALLOC_MAX_ELEMS 536870912ull /* 2^29: largest n_elems fls_reduce_norm_noalloc accepts */
 
 /* Problem statement.  One layout is shared by all groups (the paper's alignment constraint:
  * shards of different federation groups must correspond one to one). */
@@ -188,6 +189,28 @@ int fls_get_kernel_ms(fls_plan* plan, double* ms, uint64_t* launches);
 
 /* Number of kernels this plan has launched so far. */
 int fls_get_launch_count(const fls_plan* plan, uint64_t* launches);
+
+/* (No counterpart in the paper: this call exists for users of the library who are not allowed to allocate.)
+ * Gradient reduction + global norm of ONE group without a plan, a workspace or any allocation, for callers
+ * that must not call cudaMalloc: a plug-in inside an application whose pool already owns the device, a
+ * service that forbids allocation after start-up, a loop that cannot afford the device-wide stall an
+ * allocation can cause.  It computes what the first kernel of fls_sync_step computes for one group:
+ *   gbar_out[j] = mean over the K = shard_dim*replicate_dim buffers (same order: ascending inside a
+ *   sharding group, then ascending replicas; fp32), norm_coef_out[0] = L2 norm of gbar,
+ *   norm_coef_out[1] = min(1, max_grad_norm/(norm + 1e-6)) (1 if max_grad_norm <= 0).
+ * grads: host array of K device pointers (bf16 or fp32 per grad_dtype, n_elems each, 32-byte aligned);
+ * gbar_out: device, n_elems floats, 32-byte aligned; norm_coef_out: device, 2 floats, 8-byte aligned;
+ * all caller-owned.  The work is enqueued on cuda_stream; nothing is synchronised.
+ * Scratch (one double per 16384 elements and a counter) lives in a static device array of about 256 KiB
+ * that every GPU using the library holds until the process exits; hence n_elems <= FLS_NOALLOC_MAX_ELEMS,
+ * larger sizes are rejected with FLS_ESIZE and a message.  The first call on each device looks up the
+ * array's device address; make that first call outside any stream capture.  All calls share the array:
+ * calls that overlap on the same GPU (other streams or threads) race and must be serialised by the caller.
+ * No cudaMalloc/cudaFree or other allocating routine is called.
+ * Errors: FLS_EPTR, FLS_EALIGN, FLS_EINVAL (K > 64, n_elems = 0, bad dtype), FLS_ESIZE, FLS_ECUDA. */
+int fls_reduce_norm_noalloc(const void* const* grads, uint32_t shard_dim, uint32_t replicate_dim, uint32_t grad_dtype,
+                            uint64_t n_elems, double max_grad_norm, float* gbar_out, float* norm_coef_out,
+                            void* cuda_stream);
 
 /* Frees the plan and its events/stream.  Device buffers are the caller's and are not touched. */
 int fls_plan_destroy(fls_plan* plan);

@@ -17,12 +17,13 @@ FLS_STATUS_NONFINITE_NORM = 1
 FLS_MAX_GROUPS = 64
 FLS_MAX_GRAD_BUFFERS = 64
 FLS_BUFFER_ALIGN = 32
+FLS_NOALLOC_MAX_ELEMS = 1 << 29
 
 EXPORTS = [
     "fls_plan_create", "fls_plan_query", "fls_plan_bind", "fls_sync_step", "fls_sync_step_host", "fls_fedavg",
     "fls_get_norms", "fls_get_reduced_grad", "fls_get_status", "fls_get_step", "fls_set_step", "fls_comm_report",
     "fls_plan_tune", "fls_set_profiling", "fls_get_kernel_ms", "fls_get_launch_count", "fls_plan_destroy",
-    "fls_last_error",
+    "fls_last_error", "fls_reduce_norm_noalloc",
 ]
 
 
@@ -89,6 +90,7 @@ def _load() -> C.CDLL:
     lib.fls_get_kernel_ms.argtypes = [P, C.POINTER(C.c_double), C.POINTER(C.c_uint64)]
     lib.fls_get_launch_count.argtypes = [P, C.POINTER(C.c_uint64)]
     lib.fls_plan_destroy.argtypes = [P]
+    lib.fls_reduce_norm_noalloc.argtypes = [C.POINTER(C.c_void_p), C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint64, C.c_double, P, P, P]
     lib.fls_last_error.argtypes = []
     lib.fls_last_error.restype = C.c_char_p
     for name in EXPORTS:
@@ -242,6 +244,16 @@ def fls_get_launch_count(plan: int) -> int:
 
 def fls_plan_destroy(plan: int) -> None:
     _check(lib.fls_plan_destroy(plan))
+
+
+def fls_reduce_norm_noalloc(grads: Sequence, shard_dim: int, replicate_dim: int, grad_dtype: int, n_elems: int,
+                            max_grad_norm: float, gbar_out, norm_coef_out, stream=None) -> None:
+    """Mean gradient + norm + clip coefficient of one group without a plan or workspace, for callers that
+    may not allocate device memory (the scratch is a static array inside the library).  grads: K tensors;
+    gbar_out: float32 tensor of n_elems; norm_coef_out: float32 tensor of 2.  n_elems <= FLS_NOALLOC_MAX_ELEMS.
+    Calls share the static scratch: do not let two of them overlap on one GPU."""
+    _check(lib.fls_reduce_norm_noalloc(_ptr_array(grads), shard_dim, replicate_dim, grad_dtype, n_elems, max_grad_norm,
+                                       _ptr(gbar_out), _ptr(norm_coef_out), _stream_handle(stream)))
 
 
 def fls_last_error() -> str:

@@ -12,7 +12,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libfls.so")
-SOURCES = ["fls_api.cu", "fls_kernels.cu", "fls_layout.cpp", "fls_report.cpp"]
+SOURCES = ["fls_api.cu", "fls_kernels.cu", "fls_noalloc.cu", "fls_layout.cpp", "fls_report.cpp"]
 HEADERS = [os.path.join(CSRC, "fls_internal.h"), os.path.join(CSRC, "fls_kernels.h"), os.path.join(ROOT, "include", "fls.h")]
 
 

@@ -188,6 +188,10 @@ bool step_preamble(fls_plan* p, double* lr) {
 
 }  // namespace
 
+namespace fls {
+void set_last_error(const char* msg) { g_err = msg ? msg : ""; }
+}  // namespace fls
+
 extern "C" {
 
 const char* fls_last_error(void) { return g_err.c_str(); }

@@ -43,6 +43,9 @@ struct Layout {
 // Host planner: fills `out` from the unit table; returns an error message or "" on success.
 std::string build_layout(const std::vector<uint64_t>& unit_numel, uint32_t S, uint32_t Q, Layout* out);
 
+// Sets the calling thread's message returned by fls_last_error() (defined beside it).
+void set_last_error(const char* msg);
+
 void comm_report(const Layout& lay, const fls_plan_desc& d, const double* bw, fls_comm_costs* out);
 
 }  // namespace fls
