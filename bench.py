@@ -173,9 +173,12 @@ def run_ours(args, cfg):
     fill_session(sess, cfg)
     stream = torch.cuda.current_stream()
 
+    n_fedavg = [0]
+
     def one_step():
         if sess.step(stream=stream):
             sess.fedavg(counts, stream=stream)
+            n_fedavg[0] += 1
 
     def barrier():
         torch.cuda.synchronize()
@@ -187,6 +190,7 @@ def run_ours(args, cfg):
         fls.fls_set_profiling(sess.plan, profiling)
         barrier()
         l0 = fls.fls_get_launch_count(sess.plan)
+        n_fedavg[0] = 0
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
         for _ in range(n_steps):
@@ -206,6 +210,7 @@ def run_ours(args, cfg):
     if rank == 0:
         sampler.start()
     ms_total, launches = timed(args.steps, False)
+    fedavg_calls = n_fedavg[0]
     clocks = sampler.stop() if rank == 0 else None
     # second pass over the same number of steps with events around every kernel: per-kernel durations
     ms_prof, _ = timed(args.steps, True)
@@ -253,7 +258,8 @@ def run_ours(args, cfg):
                                  "share": kms[i] / sum(kms)}
         dom = max(kernels, key=lambda n: kernels[n]["share"])
         rep = fls.fls_comm_report(sess.plan)
-        step_bytes = rep["hbm_bytes_sync_step"] + rep["hbm_bytes_fedavg"] / cfg["sync_period"]
+        # bytes the timed steps had to move: every sync step, plus the FedAvg calls that fell inside the region
+        step_bytes = rep["hbm_bytes_sync_step"] + rep["hbm_bytes_fedavg"] * fedavg_calls / args.steps
         ms_step = ms_total / args.steps
         line = {
             "metric": METRIC, "value": world * G * P * args.steps / (ms_total / 1e3), "unit": UNIT, "n_gpus": world,
@@ -261,7 +267,7 @@ def run_ours(args, cfg):
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": cfg["name"], "n_params": P, "groups": G, "shard_dim": cfg["shard_dim"],
                        "replicate_dim": cfg["replicate_dim"], "sync_period": cfg["sync_period"], "grad_dtype": cfg["grad_dtype"],
-                       "fedavg_opt_state": bool(args.opt_state), "l2": "working set exceeds L2, no flush needed",
+                       "fedavg_opt_state": bool(args.opt_state), "fedavg_calls_in_timed_region": fedavg_calls, "l2": "working set exceeds L2, no flush needed",
                        "parallelism": "replicas only" if world > 1 else "1 gpu"},
             "hbm_gbs": step_bytes / ms_step / 1e6, "hbm_frac_of_measured_peak": step_bytes / ms_step / 1e6 / peak,
             "hbm_frac_of_8tbs": step_bytes / ms_step / 1e6 / 8000.0,
@@ -298,6 +304,10 @@ def main():
     ap.add_argument("--n-params", type=int, default=0, help="override P (single flat unit)")
     ap.add_argument("--groups", type=int, default=0, help="override G")
     ap.add_argument("--sync-period", type=int, default=0, help="override H")
+    ap.add_argument("--shard-dim", type=int, default=0, help="override S")
+    ap.add_argument("--replicate-dim", type=int, default=0, help="override R_rep")
+    ap.add_argument("--grad-dtype", default="", choices=["", "bf16", "f32"], help="override the gradient dtype")
+    ap.add_argument("--keep-units", action="store_true", help="with --n-params: keep the unit table's proportions")
     args = ap.parse_args()
     cfg = sy.config_by_name(args.config)
     if args.n_params:
@@ -306,6 +316,12 @@ def main():
         cfg.update(groups=args.groups, name=cfg["name"] + f"[G={args.groups}]")
     if args.sync_period:
         cfg.update(sync_period=args.sync_period, name=cfg["name"] + f"[H={args.sync_period}]")
+    if args.shard_dim:
+        cfg.update(shard_dim=args.shard_dim, name=cfg["name"] + f"[S={args.shard_dim}]")
+    if args.replicate_dim:
+        cfg.update(replicate_dim=args.replicate_dim, name=cfg["name"] + f"[R={args.replicate_dim}]")
+    if args.grad_dtype:
+        cfg.update(grad_dtype=args.grad_dtype, name=cfg["name"] + f"[{args.grad_dtype}]")
     if args.impl == "reference":
         run_reference(args, cfg)
     else:

@@ -177,8 +177,11 @@ int fls_set_step(fls_plan* plan, uint64_t t);
  * or NULL.  With R_rep = 1 the FL+HSDP entry equals the FL+FSDP one (the paper's fallback).  Host only. */
 int fls_comm_report(const fls_plan* plan, const double* bw_bytes_per_s, fls_comm_costs* out);
 
-/* Launch shape of one kernel (FLS_KERNEL_*): resident CTAs per SM used to size the persistent grid, and
- * whether the kernel walks the tiles in descending order.  0 / negative keep the current value. */
+/* Launch shape of one kernel (FLS_KERNEL_*).  By default the grid covers every tile once.  For the AdamW and
+ * FedAvg kernels ctas_per_sm > 0 switches to a persistent grid of ctas_per_sm * (number of SMs) CTAs that
+ * stride over the tiles; -2 restores the default; 0 and -1 keep the current value.  descending: 1 / 0 sets
+ * the direction in which those two kernels walk the tiles, negative keeps it.  The reduce kernel has one
+ * launch shape and ignores both. */
 int fls_plan_tune(fls_plan* plan, uint32_t kernel, int ctas_per_sm, int descending);
 
 /* Per-kernel timing with CUDA events recorded on the caller's stream around every launch.

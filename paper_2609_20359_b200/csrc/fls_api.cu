@@ -59,7 +59,7 @@ struct fls_plan {
 
   uint64_t step = 0;
   uint64_t launches = 0;
-  int ctas_per_sm[FLS_KERNEL_COUNT] = {2, 2, 2};
+  int ctas_per_sm[FLS_KERNEL_COUNT] = {0, 0, 0};   // 0: the grid covers every tile once (no grid-stride loop)
   int descending[FLS_KERNEL_COUNT] = {0, 0, 0};
 
   bool profiling = false;
@@ -75,14 +75,25 @@ struct fls_plan {
   float* d_norms() const { return reinterpret_cast<float*>(ws + kWsNorms); }
   float* d_coefs() const { return reinterpret_cast<float*>(ws + kWsCoefs); }
   double* d_normsq() const { return reinterpret_cast<double*>(ws + kWsNormSq); }
-  double* d_partials() const { return reinterpret_cast<double*>(ws + kWsPartials); }
+  double* d_partials() const { return reinterpret_cast<double*>(ws + lay.ws_partials_offset); }
   uint32_t* d_status() const { return reinterpret_cast<uint32_t*>(ws + kWsStatus); }
   uint32_t* d_ticket() const { return reinterpret_cast<uint32_t*>(ws + kWsStatus) + 1; }
 
+  SegIndex seg_index() const {
+    SegIndex ix{};
+    ix.segs = d_segs();
+    ix.n_seg = uint32_t(lay.segments.size());
+    ix.n_tiles = uint32_t(lay.n_tiles);
+    ix.in_params = ix.n_seg <= uint32_t(kParamSegs) ? 1u : 0u;
+    if (ix.in_params)
+      for (uint32_t i = 0; i < ix.n_seg; ++i) ix.tile_end[i] = uint32_t(lay.segments[i].tile_end);
+    return ix;
+  }
+
+  // grid of the AdamW / FedAvg kernels (the reduce kernel has a single launch shape of its own)
   unsigned grid_for(int kernel) const {
-    uint64_t g = uint64_t(sm_count) * uint64_t(ctas_per_sm[kernel]);
+    uint64_t g = ctas_per_sm[kernel] > 0 ? uint64_t(sm_count) * uint64_t(ctas_per_sm[kernel]) : lay.n_tiles;
     g = std::min<uint64_t>(g, lay.n_tiles);
-    g = std::min<uint64_t>(g, kMaxBlocks);
     return unsigned(std::max<uint64_t>(g, 1));
   }
 
@@ -131,9 +142,7 @@ int run_group(fls_plan* p, uint32_t g, double lr, uint64_t t_new, cudaStream_t s
   ReduceArgs ra{};
   for (uint32_t k = 0; k < p->K; ++k) ra.grad[k] = p->grads[size_t(g) * p->K + k];
   ra.gbar = p->d_gbar();
-  ra.segs = p->d_segs();
-  ra.n_tiles = p->lay.n_tiles;
-  ra.n_seg = uint32_t(p->lay.segments.size());
+  ra.idx = p->seg_index();
   ra.K = p->K;
   ra.S = d.shard_dim;
   ra.k_float = float(p->K);
@@ -148,10 +157,9 @@ int run_group(fls_plan* p, uint32_t g, double lr, uint64_t t_new, cudaStream_t s
   ra.normsq_out = p->d_normsq() + g;
   ra.status = p->d_status();
   ra.max_grad_norm = d.max_grad_norm;
-  ra.descending = p->descending[FLS_KERNEL_REDUCE];
   const bool f32 = d.grad_dtype == FLS_GRAD_F32;
   cudaError_t e = timed_launch(p, FLS_KERNEL_REDUCE, st,
-                               [&] { return launch_reduce(ra, f32, p->reduce_sg, p->grid_for(FLS_KERNEL_REDUCE), st); });
+                               [&] { return launch_reduce(ra, f32, p->reduce_sg, st); });
   if (e != cudaSuccess) return cuda_fail(e, "reduce kernel launch");
 
   // Scalars of the AdamW step, in double on the host, handed to the kernel as fp32.
@@ -163,9 +171,7 @@ int run_group(fls_plan* p, uint32_t g, double lr, uint64_t t_new, cudaStream_t s
   aa.m = p->m[g];
   aa.v = p->v[g];
   aa.pbf16 = p->pbf16[g];
-  aa.segs = p->d_segs();
-  aa.n_tiles = p->lay.n_tiles;
-  aa.n_seg = ra.n_seg;
+  aa.idx = ra.idx;
   aa.descending = p->descending[FLS_KERNEL_ADAMW];
   aa.coef = p->d_coefs() + g;
   aa.decay = float(1.0 - lr * d.weight_decay);
@@ -429,9 +435,7 @@ int fls_fedavg(fls_plan* p, const uint64_t* sample_counts, void* cuda_stream) {
     const double n = sample_counts ? double(sample_counts[g]) : 1.0;
     fa.w[g] = float(n / double(total));
   }
-  fa.segs = p->d_segs();
-  fa.n_tiles = p->lay.n_tiles;
-  fa.n_seg = uint32_t(p->lay.segments.size());
+  fa.idx = p->seg_index();
   fa.G = G;
   fa.descending = p->descending[FLS_KERNEL_FEDAVG];
   const int n_arrays = (p->desc.fedavg_what & FLS_AVG_OPT_STATE) ? 3 : 1;
@@ -492,7 +496,8 @@ int fls_comm_report(const fls_plan* p, const double* bw, fls_comm_costs* out) {
 
 int fls_plan_tune(fls_plan* p, uint32_t kernel, int ctas_per_sm, int descending) {
   if (!p || kernel >= FLS_KERNEL_COUNT) return fail(FLS_EINVAL, "fls_plan_tune: bad argument");
-  if (ctas_per_sm > 0) p->ctas_per_sm[kernel] = std::min(ctas_per_sm, 32);
+  if (ctas_per_sm > 0) p->ctas_per_sm[kernel] = std::min(ctas_per_sm, 1 << 16);
+  if (ctas_per_sm == -2) p->ctas_per_sm[kernel] = 0;   // back to the default: one pass, the grid covers every tile
   if (descending >= 0) p->descending[kernel] = descending ? 1 : 0;
   return FLS_OK;
 }

@@ -11,7 +11,7 @@ namespace fls {
 constexpr int kThreads = 256;            // threads per CTA, all kernels
 constexpr int kVec = 8;                  // elements per thread per tile
 constexpr int kTile = kThreads * kVec;   // 2048 elements per tile
-constexpr int kMaxBlocks = 4096;         // upper bound on any grid (size of the norm-partials array)
+constexpr int kParamSegs = 512;          // segment tables up to this size also travel in the kernel parameters
 
 // A run of elements that is contiguous in both the unsharded order (index j) and the shard order
 // (address a): one rank's slice of one unit, or several merged when they are adjacent in both.
@@ -29,14 +29,13 @@ constexpr uint64_t kWsStatus = 0;        // uint32 status, uint32 ticket counter
 constexpr uint64_t kWsNorms = 256;       // float[64]
 constexpr uint64_t kWsCoefs = 512;       // float[64]
 constexpr uint64_t kWsNormSq = 768;      // double[64]
-constexpr uint64_t kWsPartials = 1280;   // double[kMaxBlocks]
-constexpr uint64_t kWsSegments = kWsPartials + 8ull * kMaxBlocks;
+constexpr uint64_t kWsSegments = 1280;   // Segment[n_segments], then double[n_tiles] norm partials, then the scratch
 
 struct Layout {
   std::vector<uint64_t> unit_numel, unit_offset, unit_shard_numel, unit_shard_offset;
   std::vector<Segment> segments;
   uint64_t n_params = 0, n_padded = 0, shard_numel = 0, n_tiles = 0;
-  uint64_t ws_scratch_offset = 0, workspace_bytes = 0;
+  uint64_t ws_partials_offset = 0, ws_scratch_offset = 0, workspace_bytes = 0;
   bool vector_path = true;
 };
 

@@ -1,12 +1,17 @@
-// sm_100a kernels of libfls.  All three are HBM streams: persistent grids of 256-thread CTAs walk
-// 2048-element tiles; a thread owns 8 consecutive elements of a tile and moves them with 128-bit
-// (bf16) and 256-bit (fp32) global accesses.  No shared-memory staging and no tensor cores: nothing
-// here is a contraction, and each byte is touched once.
+// sm_100a kernels of libfls.  All three are HBM streams over 2048-element tiles; a group of 256
+// threads owns a tile, a thread owns 8 consecutive elements of it and moves them with 128-bit (bf16)
+// and 256-bit (fp32) global accesses.  By default the grid covers the whole buffer in one pass (no
+// grid-stride loop): the hardware scheduler hands out CTAs in order, so the tiles in flight form a
+// compact window that moves through memory and the SMs stay balanced, which measured 5-15 % faster
+// than persistent grid-stride CTAs.  The kernels are kept small in registers (32-66) so that 1024-2048
+// threads are resident per SM; that, not unrolling, is what keeps enough loads in flight.
+// No shared-memory staging and no tensor cores: nothing here is a contraction, and each byte is touched
+// once.
 //
 //   fls_reduce_kernel  : K gradient buffers -> mean gradient (fp32, shard order) + squared-norm partials;
-//                    the last CTA to finish adds the partials in index order and writes the group's
-//                    norm and clip coefficient (no floating-point atomics: the result does not depend
-//                    on which CTA is last).
+//                        the last CTA to finish adds the partials in index order and writes the group's
+//                        norm and clip coefficient (no floating-point atomics: the result does not depend
+//                        on which CTA is last).
 //   fls_adamw_kernel   : clip + AdamW on master/m/v in place + bf16 copy in unsharded order.
 //   fls_fedavg_kernel  : weighted average of G copies written back to all G (+ bf16 copies).
 #include <cuda_bf16.h>
@@ -24,6 +29,8 @@ namespace {
 struct alignas(32) F8 { float v[8]; };
 
 #define FLS_O8(r) "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+#define FLS_U8(r) "r"(__float_as_uint(r.v[0])), "r"(__float_as_uint(r.v[1])), "r"(__float_as_uint(r.v[2])), "r"(__float_as_uint(r.v[3])), \
+                  "r"(__float_as_uint(r.v[4])), "r"(__float_as_uint(r.v[5])), "r"(__float_as_uint(r.v[6])), "r"(__float_as_uint(r.v[7]))
 __device__ __forceinline__ F8 ld8_stream(const float* p) {
   uint32_t u[8];
   asm volatile("ld.global.L1::no_allocate.L2::evict_first.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];" : FLS_O8(u) : "l"(p));
@@ -40,17 +47,15 @@ __device__ __forceinline__ F8 ld8_keep(const float* p) {
   for (int e = 0; e < 8; ++e) r.v[e] = __uint_as_float(u[e]);
   return r;
 }
-#define FLS_U8(r) "r"(__float_as_uint(r.v[0])), "r"(__float_as_uint(r.v[1])), "r"(__float_as_uint(r.v[2])), "r"(__float_as_uint(r.v[3])), \
-                  "r"(__float_as_uint(r.v[4])), "r"(__float_as_uint(r.v[5])), "r"(__float_as_uint(r.v[6])), "r"(__float_as_uint(r.v[7]))
 __device__ __forceinline__ void st8_stream(float* p, const F8& r) {
   asm volatile("st.global.L1::no_allocate.L2::evict_first.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" :: "l"(p), FLS_U8(r) : "memory");
 }
 __device__ __forceinline__ void st8_keep(float* p, const F8& r) {
   asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" :: "l"(p), FLS_U8(r) : "memory");
 }
+// 128-bit accesses have no L2::evict_first form; .cs is the streaming (evict-first) cache operator
 __device__ __forceinline__ uint4 ld_b128_stream(const void* p) {
   uint4 r;
-  // 128-bit accesses have no L2::evict_first form; .cs is the streaming (evict-first) cache operator
   asm volatile("ld.global.cs.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
   return r;
 }
@@ -63,45 +68,74 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);   // round to nearest even
   return *reinterpret_cast<uint32_t*>(&h);
 }
+__device__ __forceinline__ uint4 pack_bf16x8(const F8& x) {
+  uint4 p;
+  p.x = pack_bf16x2(x.v[0], x.v[1]); p.y = pack_bf16x2(x.v[2], x.v[3]);
+  p.z = pack_bf16x2(x.v[4], x.v[5]); p.w = pack_bf16x2(x.v[6], x.v[7]);
+  return p;
+}
 __device__ __forceinline__ uint16_t to_bf16_bits(float x) {
   __nv_bfloat16 h = __float2bfloat16_rn(x);
   return *reinterpret_cast<uint16_t*>(&h);
 }
 
 // ------------------------------------------------------------------------------------------------
-// Tile -> segment walk.  A CTA visits tiles in monotone order, so it only ever steps to a
-// neighbouring segment; the current segment lives in registers.
+// Tile -> segment.  A segment is a run that is contiguous in both index orders.
 // ------------------------------------------------------------------------------------------------
-struct Walker {
-  const Segment* segs;
-  uint32_t i;
-  Segment cur;
-  __device__ __forceinline__ void init(const Segment* s, uint32_t n_seg, bool descending) {
-    segs = s;
-    i = descending ? n_seg - 1 : 0;
-    cur = segs[i];
+// Index of the segment that holds `tile`: bisection over the tile_end table, read from the kernel
+// parameters when the table is small enough to travel there, else from global memory.
+__device__ __forceinline__ uint32_t find_segment(const SegIndex& ix, uint32_t tile) {
+  uint32_t lo = 0, hi = ix.n_seg - 1;
+  if (ix.in_params) {
+    while (lo < hi) {
+      const uint32_t mid = (lo + hi) >> 1;
+      if (ix.tile_end[mid] <= tile) lo = mid + 1; else hi = mid;
+    }
+  } else {
+    while (lo < hi) {
+      const uint32_t mid = (lo + hi) >> 1;
+      if (__ldg(&ix.segs[mid].tile_end) <= uint64_t(tile)) lo = mid + 1; else hi = mid;
+    }
   }
-  __device__ __forceinline__ void seek(uint64_t tile) {
-    while (tile >= cur.tile_end) cur = segs[++i];
-    while (tile < cur.tile_begin) cur = segs[--i];
-  }
-};
+  return lo;
+}
 
 // Per-thread slice of a tile: n = number of valid elements (0..8), vec = whole 8 on the vector path.
+// `lane` is the thread's index inside the 256-thread group that owns the tile.
 struct Slice { uint64_t j, a; uint32_t n; bool vec; };
-__device__ __forceinline__ Slice slice_of(const Segment& s, uint64_t tile) {
+__device__ __forceinline__ Slice slice_of(const Segment* sg, uint32_t tile, uint32_t lane) {
   Slice r;
-  const uint64_t e0 = (tile - s.tile_begin) * kTile + threadIdx.x * kVec;
-  const uint64_t rem = e0 < s.len ? s.len - e0 : 0;
+  const uint64_t e0 = (uint64_t(tile) - __ldg(&sg->tile_begin)) * kTile + lane * kVec;
+  const uint64_t len = __ldg(&sg->len);
+  const uint64_t rem = e0 < len ? len - e0 : 0;
   r.n = rem < kVec ? uint32_t(rem) : kVec;
-  r.vec = s.aligned && r.n == kVec;
-  r.j = s.j0 + e0;
-  r.a = s.a0 + e0;
+  r.vec = __ldg(&sg->aligned) && r.n == kVec;
+  r.j = __ldg(&sg->j0) + e0;
+  r.a = __ldg(&sg->a0) + e0;
   return r;
 }
 
+// Segment cursor of a CTA that visits several tiles in monotone order (persistent launch shapes).
+struct Walker {
+  const Segment* segs;
+  uint32_t i;
+  uint64_t begin, end;
+  __device__ __forceinline__ void init(const SegIndex& ix, uint32_t tile) {
+    segs = ix.segs;
+    i = find_segment(ix, tile);
+    begin = __ldg(&segs[i].tile_begin);
+    end = __ldg(&segs[i].tile_end);
+  }
+  __device__ __forceinline__ const Segment* seek(uint32_t tile) {
+    while (uint64_t(tile) >= end) { ++i; begin = end; end = __ldg(&segs[i].tile_end); }
+    while (uint64_t(tile) < begin) { --i; end = begin; begin = __ldg(&segs[i].tile_begin); }
+    return segs + i;
+  }
+};
+
 // Fixed-shape block sum of one double per thread (shuffle tree inside a warp, then warp 0 over the
 // per-warp results): same order every run.  Result valid in thread 0.
+template <int THREADS>
 __device__ __forceinline__ double block_sum(double x, double* sh) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, o);
@@ -111,9 +145,9 @@ __device__ __forceinline__ double block_sum(double x, double* sh) {
   __syncthreads();
   double t = 0.0;
   if (warp == 0) {
-    t = lane < kThreads / 32 ? sh[lane] : 0.0;
+    t = lane < THREADS / 32 ? sh[lane] : 0.0;
 #pragma unroll
-    for (int o = 4; o > 0; o >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, o);
+    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, o);
   }
   return t;
 }
@@ -154,40 +188,45 @@ __device__ __forceinline__ void unpack(const Raw<1, true>& x, float (&f)[1]) { f
 // sigma, eight loads in flight at a time.  `inner` is the running sum of the current sharding group
 // (the reduce-scatter level); when the group's last buffer has been added it is folded into `outer`
 // (the all-reduce level across replicas).  Both start at zero, so every level is a plain ascending
-// sum (0 + x is exact).  SG fixes the level structure at compile time so the hot loop holds only
-// unpack + add:
+// sum (0 + x is exact).  KT and SG fix the shape at compile time so the hot path holds only
+// load + unpack + add:
+//   KT = K for K in {1, 2, 4, 8} (the buffer loop is unrolled and the pointers are read straight from
+//        the kernel parameters), 0 for any other K (batches of 8 with a run-time bound);
 //   SG =  0 : every batch of 8 lies inside one sharding group (FSDP, or S a multiple of 8); bit i of
 //             fold_mask says that batch i closes a group.
-//   SG = 1, 2, 4 : S == SG, a batch holds 8/SG whole groups.
+//   SG = 1, 2, 4 : S == SG, a batch holds whole groups of SG buffers.
 //   SG = -1 : any other shape; bit k of end_mask says that buffer k closes a group.
-template <int N, bool F32, int SG>
+template <int N, bool F32, int KT, int SG>
 __device__ __forceinline__ void reduce_elems(const ReduceArgs& a, uint64_t j, float (&mean)[N]) {
+  constexpr int B = KT ? KT : 8;            // buffers per batch
+  const uint32_t K = KT ? uint32_t(KT) : a.K;
   float inner[N], outer[N];
 #pragma unroll
   for (int e = 0; e < N; ++e) inner[e] = outer[e] = 0.f;
-  for (uint32_t k0 = 0; k0 < a.K; k0 += 8) {
-    Raw<N, F32> raw[8];
+#pragma unroll 1
+  for (uint32_t k0 = 0; k0 < K; k0 += B) {
+    Raw<N, F32> raw[B];
 #pragma unroll
-    for (int b = 0; b < 8; ++b)
-      if (k0 + b < a.K) load_raw(raw[b], a.grad[k0 + b], j);
+    for (int b = 0; b < B; ++b)
+      if (KT || k0 + b < K) load_raw(raw[b], a.grad[KT ? b : k0 + b], j);
     if constexpr (SG == 0) {
 #pragma unroll
-      for (int b = 0; b < 8; ++b) {
-        if (k0 + b < a.K) {
+      for (int b = 0; b < B; ++b) {
+        if (KT || k0 + b < K) {
           float x[N];
           unpack(raw[b], x);
 #pragma unroll
           for (int e = 0; e < N; ++e) inner[e] += x[e];
         }
       }
-      if ((a.fold_mask >> (k0 >> 3)) & 1u) {
+      if (KT || ((a.fold_mask >> (k0 >> 3)) & 1u)) {
 #pragma unroll
         for (int e = 0; e < N; ++e) { outer[e] += inner[e]; inner[e] = 0.f; }
       }
     } else if constexpr (SG > 0) {
 #pragma unroll
-      for (int g0 = 0; g0 < 8; g0 += SG) {
-        if (k0 + g0 < a.K) {
+      for (int g0 = 0; g0 < B; g0 += SG) {
+        if (KT || k0 + g0 < K) {
           float s[N];
           unpack(raw[g0], s);
 #pragma unroll
@@ -203,9 +242,9 @@ __device__ __forceinline__ void reduce_elems(const ReduceArgs& a, uint64_t j, fl
       }
     } else {
 #pragma unroll
-      for (int b = 0; b < 8; ++b) {
+      for (int b = 0; b < B; ++b) {
         const uint32_t k = k0 + b;
-        if (k < a.K) {
+        if (k < K) {
           float x[N];
           unpack(raw[b], x);
 #pragma unroll
@@ -228,39 +267,46 @@ __device__ __forceinline__ void reduce_elems(const ReduceArgs& a, uint64_t j, fl
   }
 }
 
-template <bool F32, int SG>
-__global__ void __launch_bounds__(kThreads, 2) fls_reduce_kernel(const __grid_constant__ ReduceArgs a) {
-  __shared__ double sh[kThreads / 32];
+// element-wise path of one thread's slice (unaligned runs and ragged tails); kept out of line so that
+// it does not cost the vector path registers
+template <bool F32>
+__device__ __noinline__ float reduce_slice_scalar(const ReduceArgs& a, uint64_t j, uint64_t addr, uint32_t n) {
+  float sq = 0.f;
+  for (uint32_t e = 0; e < n; ++e) {
+    float g[1];
+    reduce_elems<1, F32, 0, -1>(a, j + e, g);
+    a.gbar[addr + e] = g[0];
+    sq = fmaf(g[0], g[0], sq);
+  }
+  return sq;
+}
+
+// One pass, no loop: a CTA of THREADS threads owns THREADS/256 consecutive tiles, one per group of 256
+// threads, and the grid covers the whole buffer.  MINB resident CTAs per SM fix the register budget:
+// 1024 x 2 (32 registers) for the flat order, 512 x 3 (42 registers) for the two-level orders, which
+// carry a second set of accumulators, 256 x 2 for a run-time K.
+template <bool F32, int KT, int SG, int THREADS, int MINB>
+__global__ void __launch_bounds__(THREADS, MINB) fls_reduce_kernel(const __grid_constant__ ReduceArgs a) {
+  __shared__ double sh[THREADS / 32];
   __shared__ bool is_last;
-  double dsum = 0.0;
-  if (blockIdx.x < a.n_tiles) {
-    Walker w;
-    w.init(a.segs, a.n_seg, a.descending);
-    for (uint64_t lin = blockIdx.x; lin < a.n_tiles; lin += gridDim.x) {
-      const uint64_t tile = a.descending ? a.n_tiles - 1 - lin : lin;
-      w.seek(tile);
-      const Slice s = slice_of(w.cur, tile);
-      if (s.vec) {
-        float g[8];
-        reduce_elems<8, F32, SG>(a, s.j, g);
-        F8 o;
-        float sq = 0.f;
+  float sq = 0.f;
+  const uint32_t tile = blockIdx.x * (THREADS / kThreads) + threadIdx.x / kThreads;
+  if (tile < a.idx.n_tiles) {
+    const Slice s = slice_of(a.idx.segs + find_segment(a.idx, tile), tile, threadIdx.x % kThreads);
+    if (s.vec) {
+      float g[8];
+      reduce_elems<8, F32, KT, SG>(a, s.j, g);
+      F8 o;
 #pragma unroll
-        for (int e = 0; e < 8; ++e) { o.v[e] = g[e]; sq = fmaf(g[e], g[e], sq); }
-        st8_keep(a.gbar + s.a, o);
-        dsum += double(sq);
-      } else {
-        for (uint32_t e = 0; e < s.n; ++e) {
-          float g[1];
-          reduce_elems<1, F32, -1>(a, s.j + e, g);
-          a.gbar[s.a + e] = g[0];
-          dsum += double(g[0] * g[0]);
-        }
-      }
+      for (int e = 0; e < 8; ++e) { o.v[e] = g[e]; sq = fmaf(g[e], g[e], sq); }
+      st8_keep(a.gbar + s.a, o);
+    } else if (s.n) {
+      sq = reduce_slice_scalar<F32>(a, s.j, s.a, s.n);
     }
   }
-  // CTA partial -> workspace; the CTA that takes the last ticket adds all partials in index order.
-  double total = block_sum(dsum, sh);
+  // CTA partial -> workspace; the CTA that takes the last ticket adds all partials in index order, so
+  // the norm does not depend on the order in which CTAs finish.
+  double total = block_sum<THREADS>(double(sq), sh);
   if (threadIdx.x == 0) {
     a.partials[blockIdx.x] = total;
     __threadfence();
@@ -271,8 +317,8 @@ __global__ void __launch_bounds__(kThreads, 2) fls_reduce_kernel(const __grid_co
   if (!is_last) return;
   __threadfence();
   double s = 0.0;
-  for (uint32_t i = threadIdx.x; i < gridDim.x; i += kThreads) s += __ldcg(a.partials + i);
-  total = block_sum(s, sh);
+  for (uint32_t i = threadIdx.x; i < gridDim.x; i += THREADS) s += __ldcg(a.partials + i);
+  total = block_sum<THREADS>(s, sh);
   if (threadIdx.x == 0) {
     const double nrm = sqrt(total);
     double c = 1.0;
@@ -300,15 +346,24 @@ __device__ __forceinline__ void adamw_one(const AdamArgs& a, float c, float gbar
   th = fmaf(-a.step_size, __fdiv_rn(m, denom), th);         // step_size = lr / (1 - beta1^t)
 }
 
+__device__ __noinline__ void adamw_slice_scalar(const AdamArgs& a, float c, uint64_t j, uint64_t addr, uint32_t n) {
+  for (uint32_t e = 0; e < n; ++e) {
+    float th = a.theta[addr + e], m = a.m[addr + e], v = a.v[addr + e];
+    adamw_one(a, c, a.gbar[addr + e], th, m, v);
+    a.theta[addr + e] = th; a.m[addr + e] = m; a.v[addr + e] = v;
+    a.pbf16[j + e] = to_bf16_bits(th);
+  }
+}
+
 __global__ void __launch_bounds__(kThreads, 3) fls_adamw_kernel(const __grid_constant__ AdamArgs a) {
-  if (blockIdx.x >= a.n_tiles) return;
+  const uint32_t n_tiles = a.idx.n_tiles;
+  if (blockIdx.x >= n_tiles) return;
   const float c = __ldcg(a.coef);
   Walker w;
-  w.init(a.segs, a.n_seg, a.descending);
-  for (uint64_t lin = blockIdx.x; lin < a.n_tiles; lin += gridDim.x) {
-    const uint64_t tile = a.descending ? a.n_tiles - 1 - lin : lin;
-    w.seek(tile);
-    const Slice s = slice_of(w.cur, tile);
+  w.init(a.idx, a.descending ? n_tiles - 1 - blockIdx.x : blockIdx.x);
+  for (uint32_t lin = blockIdx.x; lin < n_tiles; lin += gridDim.x) {
+    const uint32_t tile = a.descending ? n_tiles - 1 - lin : lin;
+    const Slice s = slice_of(w.seek(tile), tile, threadIdx.x);
     if (s.vec) {
       const F8 g = ld8_keep(a.gbar + s.a);
       F8 th = ld8_stream(a.theta + s.a);
@@ -319,89 +374,135 @@ __global__ void __launch_bounds__(kThreads, 3) fls_adamw_kernel(const __grid_con
       st8_stream(a.theta + s.a, th);
       st8_stream(a.m + s.a, m);
       st8_stream(a.v + s.a, v);
-      uint4 p;
-      p.x = pack_bf16x2(th.v[0], th.v[1]); p.y = pack_bf16x2(th.v[2], th.v[3]);
-      p.z = pack_bf16x2(th.v[4], th.v[5]); p.w = pack_bf16x2(th.v[6], th.v[7]);
-      st_b128_stream(a.pbf16 + s.j, p);
-    } else {
-      for (uint32_t e = 0; e < s.n; ++e) {
-        float th = a.theta[s.a + e], m = a.m[s.a + e], v = a.v[s.a + e];
-        adamw_one(a, c, a.gbar[s.a + e], th, m, v);
-        a.theta[s.a + e] = th; a.m[s.a + e] = m; a.v[s.a + e] = v;
-        a.pbf16[s.j + e] = to_bf16_bits(th);
-      }
+      st_b128_stream(a.pbf16 + s.j, pack_bf16x8(th));
+    } else if (s.n) {
+      adamw_slice_scalar(a, c, s.j, s.a, s.n);
     }
   }
 }
 
 // ------------------------------------------------------------------------------------------------
-// K3: FedAvg.  x_bar = sum_g w_g x_g, ascending g, written to all G copies.
+// K3: FedAvg.  x_bar = sum_g w_g x_g, ascending g from zero, written to all G copies.
+// GT = G for G in {1, 2, 4, 8} (unrolled, pointers straight from the kernel parameters), else 0.
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kThreads, 2) fls_fedavg_kernel(const __grid_constant__ FedavgArgs a) {
-  if (blockIdx.x >= a.n_tiles) return;
+__device__ __noinline__ void fedavg_slice_scalar(const FedavgArgs& a, uint64_t j, uint64_t addr, uint32_t n) {
+  for (uint32_t e = 0; e < n; ++e) {
+    float acc = 0.f;
+    for (uint32_t g = 0; g < a.G; ++g) acc = fmaf(a.w[g], a.x[g][addr + e], acc);
+    for (uint32_t g = 0; g < a.G; ++g) a.x[g][addr + e] = acc;
+    if (a.write_bf16) {
+      const uint16_t b = to_bf16_bits(acc);
+      for (uint32_t g = 0; g < a.G; ++g) a.pbf16[g][j + e] = b;
+    }
+  }
+}
+
+template <int GT, int MINB>
+__global__ void __launch_bounds__(kThreads, MINB) fls_fedavg_kernel(const __grid_constant__ FedavgArgs a) {
+  constexpr int B = GT ? GT : 8;
+  const uint32_t G = GT ? uint32_t(GT) : a.G;
+  const uint32_t n_tiles = a.idx.n_tiles;
+  if (blockIdx.x >= n_tiles) return;
   Walker w;
-  w.init(a.segs, a.n_seg, a.descending);
-  for (uint64_t lin = blockIdx.x; lin < a.n_tiles; lin += gridDim.x) {
-    const uint64_t tile = a.descending ? a.n_tiles - 1 - lin : lin;
-    w.seek(tile);
-    const Slice s = slice_of(w.cur, tile);
+  w.init(a.idx, a.descending ? n_tiles - 1 - blockIdx.x : blockIdx.x);
+  for (uint32_t lin = blockIdx.x; lin < n_tiles; lin += gridDim.x) {
+    const uint32_t tile = a.descending ? n_tiles - 1 - lin : lin;
+    const Slice s = slice_of(w.seek(tile), tile, threadIdx.x);
     if (s.vec) {
       F8 acc;
 #pragma unroll
       for (int e = 0; e < 8; ++e) acc.v[e] = 0.f;
-      for (uint32_t g0 = 0; g0 < a.G; g0 += 8) {
-        F8 raw[8];
+#pragma unroll 1
+      for (uint32_t g0 = 0; g0 < G; g0 += B) {
+        F8 raw[B];
 #pragma unroll
-        for (int b = 0; b < 8; ++b)
-          if (g0 + b < a.G) raw[b] = ld8_stream(a.x[g0 + b] + s.a);
+        for (int b = 0; b < B; ++b)
+          if (GT || g0 + b < G) raw[b] = ld8_stream(a.x[GT ? b : g0 + b] + s.a);
 #pragma unroll
-        for (int b = 0; b < 8; ++b) {
-          const uint32_t g = g0 + b;
-          if (g < a.G) {
-            const float wg = a.w[g];
+        for (int b = 0; b < B; ++b) {
+          if (GT || g0 + b < G) {
+            const float wg = a.w[GT ? b : g0 + b];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) acc.v[e] = fmaf(wg, raw[b].v[e], acc.v[e]);   // acc starts at 0: the first term is w_0 x_0
+            for (int e = 0; e < 8; ++e) acc.v[e] = fmaf(wg, raw[b].v[e], acc.v[e]);   // acc starts at 0: first term w_0 x_0
           }
         }
       }
-      for (uint32_t g = 0; g < a.G; ++g) st8_stream(a.x[g] + s.a, acc);
+      if constexpr (GT != 0) {
+#pragma unroll
+        for (int g = 0; g < GT; ++g) st8_stream(a.x[g] + s.a, acc);
+      } else {
+        for (uint32_t g = 0; g < G; ++g) st8_stream(a.x[g] + s.a, acc);
+      }
       if (a.write_bf16) {
-        uint4 p;
-        p.x = pack_bf16x2(acc.v[0], acc.v[1]); p.y = pack_bf16x2(acc.v[2], acc.v[3]);
-        p.z = pack_bf16x2(acc.v[4], acc.v[5]); p.w = pack_bf16x2(acc.v[6], acc.v[7]);
-        for (uint32_t g = 0; g < a.G; ++g) st_b128_stream(a.pbf16[g] + s.j, p);
-      }
-    } else {
-      for (uint32_t e = 0; e < s.n; ++e) {
-        float acc = 0.f;
-        for (uint32_t g = 0; g < a.G; ++g) {
-          const float x = a.x[g][s.a + e];
-          acc = fmaf(a.w[g], x, acc);
-        }
-        for (uint32_t g = 0; g < a.G; ++g) a.x[g][s.a + e] = acc;
-        if (a.write_bf16) {
-          const uint16_t b = to_bf16_bits(acc);
-          for (uint32_t g = 0; g < a.G; ++g) a.pbf16[g][s.j + e] = b;
+        const uint4 p = pack_bf16x8(acc);
+        if constexpr (GT != 0) {
+#pragma unroll
+          for (int g = 0; g < GT; ++g) st_b128_stream(a.pbf16[g] + s.j, p);
+        } else {
+          for (uint32_t g = 0; g < G; ++g) st_b128_stream(a.pbf16[g] + s.j, p);
         }
       }
+    } else if (s.n) {
+      fedavg_slice_scalar(a, s.j, s.a, s.n);
     }
   }
 }
 
-}  // namespace
+// ------------------------------------------------------------------------------------------------
+// Launchers.
+// ------------------------------------------------------------------------------------------------
+constexpr int kFlatThreads = 1024, kFlatMinB = 2;      // SG == 0 with a static K
+constexpr int kLevelThreads = 512, kLevelMinB = 3;     // two-level orders with a static K
+constexpr int kAnyThreads = 256, kAnyMinB = 2;         // run-time K: batches of 8 loads need the registers
 
-template <bool F32>
-static void launch_reduce_t(const ReduceArgs& a, int sg, unsigned grid, cudaStream_t st) {
-  switch (sg) {
-    case 0: fls_reduce_kernel<F32, 0><<<grid, kThreads, 0, st>>>(a); break;
-    case 1: fls_reduce_kernel<F32, 1><<<grid, kThreads, 0, st>>>(a); break;
-    case 2: fls_reduce_kernel<F32, 2><<<grid, kThreads, 0, st>>>(a); break;
-    case 4: fls_reduce_kernel<F32, 4><<<grid, kThreads, 0, st>>>(a); break;
-    default: fls_reduce_kernel<F32, -1><<<grid, kThreads, 0, st>>>(a); break;
-  }
+inline int reduce_threads(const ReduceArgs& a, int sg) {
+  const bool static_k = sg >= 0 && (a.K == 1 || a.K == 2 || a.K == 4 || a.K == 8);
+  return !static_k ? kAnyThreads : (sg == 0 ? kFlatThreads : kLevelThreads);
 }
 
-cudaError_t launch_reduce(const ReduceArgs& a, bool f32, int sg, unsigned grid, cudaStream_t st) {
+template <bool F32, int KT, int SG>
+void launch_reduce_shape(const ReduceArgs& a, unsigned grid, cudaStream_t st) {
+  if constexpr (KT == 0)
+    fls_reduce_kernel<F32, KT, SG, kAnyThreads, kAnyMinB><<<grid, kAnyThreads, 0, st>>>(a);
+  else if constexpr (SG == 0)
+    fls_reduce_kernel<F32, KT, SG, kFlatThreads, kFlatMinB><<<grid, kFlatThreads, 0, st>>>(a);
+  else
+    fls_reduce_kernel<F32, KT, SG, kLevelThreads, kLevelMinB><<<grid, kLevelThreads, 0, st>>>(a);
+}
+
+template <bool F32, int KT>
+void launch_reduce_k(const ReduceArgs& a, int sg, unsigned grid, cudaStream_t st) {
+  // only the level structures that can occur with KT buffers are instantiated (SG divides KT)
+  if (sg == 0) { launch_reduce_shape<F32, KT, 0>(a, grid, st); return; }
+  if constexpr (KT == 0 || KT >= 2) { if (sg == 1) { launch_reduce_shape<F32, KT, 1>(a, grid, st); return; } }
+  if constexpr (KT == 0 || KT >= 4) { if (sg == 2) { launch_reduce_shape<F32, KT, 2>(a, grid, st); return; } }
+  if constexpr (KT == 0 || KT == 8) { if (sg == 4) { launch_reduce_shape<F32, KT, 4>(a, grid, st); return; } }
+  launch_reduce_shape<F32, 0, -1>(a, grid, st);
+}
+
+template <bool F32>
+void launch_reduce_t(const ReduceArgs& a, int sg, unsigned grid, cudaStream_t st) {
+  if (sg >= 0) {
+    switch (a.K) {
+      case 1: launch_reduce_k<F32, 1>(a, sg, grid, st); return;
+      case 2: launch_reduce_k<F32, 2>(a, sg, grid, st); return;
+      case 4: launch_reduce_k<F32, 4>(a, sg, grid, st); return;
+      case 8: launch_reduce_k<F32, 8>(a, sg, grid, st); return;
+      default: break;
+    }
+  }
+  launch_reduce_k<F32, 0>(a, sg, grid, st);
+}
+
+}  // namespace
+
+unsigned reduce_grid(const ReduceArgs& a, int sg) {
+  const unsigned tiles_per_cta = reduce_threads(a, sg) / kThreads;
+  return (a.idx.n_tiles + tiles_per_cta - 1) / tiles_per_cta;
+}
+
+cudaError_t launch_reduce(const ReduceArgs& a, bool f32, int sg, cudaStream_t st) {
+  const unsigned grid = reduce_grid(a, sg);
   if (f32)
     launch_reduce_t<true>(a, sg, grid, st);
   else
@@ -415,7 +516,13 @@ cudaError_t launch_adamw(const AdamArgs& a, unsigned grid, cudaStream_t st) {
 }
 
 cudaError_t launch_fedavg(const FedavgArgs& a, unsigned grid, cudaStream_t st) {
-  fls_fedavg_kernel<<<grid, kThreads, 0, st>>>(a);
+  switch (a.G) {
+    case 1: fls_fedavg_kernel<1, 6><<<grid, kThreads, 0, st>>>(a); break;
+    case 2: fls_fedavg_kernel<2, 5><<<grid, kThreads, 0, st>>>(a); break;
+    case 4: fls_fedavg_kernel<4, 4><<<grid, kThreads, 0, st>>>(a); break;
+    case 8: fls_fedavg_kernel<8, 2><<<grid, kThreads, 0, st>>>(a); break;
+    default: fls_fedavg_kernel<0, 2><<<grid, kThreads, 0, st>>>(a); break;
+  }
   return cudaGetLastError();
 }
 

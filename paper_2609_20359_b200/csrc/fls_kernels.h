@@ -6,12 +6,21 @@
 
 namespace fls {
 
+// Where the tiles of each segment end, for the tile -> segment search.  Small tables (the usual case)
+// are also copied here so that the search runs out of the kernel parameters (constant bank) instead of
+// global memory; the segment record itself is then one global load.
+struct SegIndex {
+  const Segment* segs;                     // device
+  uint32_t n_seg;
+  uint32_t n_tiles;
+  uint32_t in_params;                      // 1: tile_end[] below is filled
+  uint32_t tile_end[kParamSegs];
+};
+
 struct ReduceArgs {
   const void* grad[FLS_MAX_GRAD_BUFFERS];  // device, K buffers of this group, index rho*S + sigma
   float* gbar;                             // device, reduced gradient (shard order)
-  const Segment* segs;                     // device
-  uint64_t n_tiles;
-  uint32_t n_seg;
+  SegIndex idx;
   uint32_t K, S;
   float k_float, inv_k;                    // K and 1/K as float: the mean is scaled by 1/K once
   uint32_t k_is_pow2;                      // 1/K exact: multiply; otherwise divide
@@ -24,16 +33,13 @@ struct ReduceArgs {
   double* normsq_out;
   uint32_t* status;
   double max_grad_norm;
-  int descending;
 };
 
 struct AdamArgs {
   const float* gbar;
   float *theta, *m, *v;
   uint16_t* pbf16;
-  const Segment* segs;
-  uint64_t n_tiles;
-  uint32_t n_seg;
+  SegIndex idx;
   int descending;
   const float* coef;                       // device, written by the reduce kernel of the same group
   float decay, beta1, omb1, beta2, omb2, step_size, inv_sqrt_bc2, eps;
@@ -43,16 +49,16 @@ struct FedavgArgs {
   float* x[FLS_MAX_GROUPS];                // device, the G copies (in/out)
   uint16_t* pbf16[FLS_MAX_GROUPS];         // device, the G bf16 copies (out), used if write_bf16
   float w[FLS_MAX_GROUPS];
-  const Segment* segs;
-  uint64_t n_tiles;
-  uint32_t n_seg;
+  SegIndex idx;
   uint32_t G;
   int write_bf16;
   int descending;
 };
 
-// sg: level structure of the reduction (see reduce_elems): 0, 1, 2, 4 or -1 for the generic form
-cudaError_t launch_reduce(const ReduceArgs& a, bool f32, int sg, unsigned grid, cudaStream_t st);
+// sg: level structure of the reduction (see reduce_elems): 0, 1, 2, 4 or -1 for the generic form.
+// The reduce kernel has one launch shape; reduce_grid() is its grid (= number of norm partials it writes).
+unsigned reduce_grid(const ReduceArgs& a, int sg);
+cudaError_t launch_reduce(const ReduceArgs& a, bool f32, int sg, cudaStream_t st);
 cudaError_t launch_adamw(const AdamArgs& a, unsigned grid, cudaStream_t st);
 cudaError_t launch_fedavg(const FedavgArgs& a, unsigned grid, cudaStream_t st);
 

@@ -67,7 +67,9 @@ std::string build_layout(const std::vector<uint64_t>& unit_numel, uint32_t S, ui
     if (g.len % kVec != 0) L.vector_path = false;
   L.n_tiles = tile;
   const uint64_t seg_bytes = L.segments.size() * sizeof(Segment);
-  L.ws_scratch_offset = (kWsSegments + seg_bytes + 255) / 256 * 256;
+  if (L.n_tiles >= (1ull << 32)) return "plan too large";
+  L.ws_partials_offset = (kWsSegments + seg_bytes + 255) / 256 * 256;
+  L.ws_scratch_offset = (L.ws_partials_offset + 8 * L.n_tiles + 255) / 256 * 256;   // at most one partial per tile
   L.workspace_bytes = L.ws_scratch_offset + 4ull * L.n_padded;
   return "";
 }
