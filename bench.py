@@ -31,9 +31,9 @@ import synthetic as sy
 METRIC = "synced_params_per_s"
 UNIT = "params/s"
 DEFAULT_CONFIG = "gpt2_small_fl_fsdp"
-# DRAM bytes per launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
-# dram__bytes_write.sum), per config; None until a capture of that workload exists under profiles/.
-NCU_TRAFFIC_BYTES = {}
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture summarised in
+# profiles/dram_traffic_gpt2_small.md; None for workloads that have no capture.
+NCU_TRAFFIC_BYTES = {("gpt2_small_fl_fsdp", "adamw"): 3673.2e6, ("gpt2_small_fl_fsdp", "reduce"): 2444.6e6}
 
 
 def measured_peak_gbs():
@@ -46,86 +46,140 @@ def measured_peak_gbs():
 
 # --------------------------------------------------------------------------------------- clocks
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """Samples the SM clock and the throttle reasons of one GPU while the timed region runs.  Reads NVML
+    directly every few milliseconds (the timed region of a small workload lasts only tens of ms); falls
+    back to one nvidia-smi query if the NVML binding is missing.  Nothing is ever set, only read."""
+    REASONS = (("hw_slowdown", 0x8), ("hw_thermal_slowdown", 0x40), ("sw_thermal_slowdown", 0x20), ("sw_power_cap", 0x4),
+               ("hw_power_brake_slowdown", 0x80))
 
     def __init__(self, index: int):
-        self.index, self.rows, self.proc = index, [], None
+        self.index, self.sm, self.reason_bits, self.power = index, [], 0, []
+        self.max_sm, self._stop, self._thread, self._nvml = None, threading.Event(), None, None
 
     def start(self):
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            threading.Thread(target=self._read, daemon=True).start()
+            import pynvml
+            pynvml.nvmlInit()
+            self._nvml = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(self._physical_index())
+            self.max_sm = float(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+            self._thread = threading.Thread(target=self._poll, daemon=True)
+            self._thread.start()
         except Exception:
-            self.proc = None
+            self._nvml = None
 
-    def _read(self):
-        for line in self.proc.stdout:
-            self.rows.append([x.strip() for x in line.split(",")])
+    def _physical_index(self) -> int:
+        vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+        ids = [v for v in vis.split(",") if v.strip() != ""]
+        if ids and all(v.strip().isdigit() for v in ids) and self.index < len(ids):
+            return int(ids[self.index])
+        return self.index
+
+    def _poll(self):
+        nv = self._nvml
+        while not self._stop.is_set():
+            try:
+                self.sm.append(float(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                self.reason_bits |= int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h)) if hasattr(nv, "nvmlDeviceGetCurrentClocksEventReasons") \
+                    else int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                self.power.append(nv.nvmlDeviceGetPowerUsage(self._h) / 1000.0)
+            except Exception:
+                pass
+            time.sleep(0.002)
 
     def stop(self) -> dict:
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
-        self.proc.terminate()
-        sm, mx, reasons = [], [], set()
-        for r in self.rows:
-            try:
-                sm.append(float(r[0])); mx.append(float(r[1]))
-            except Exception:
-                continue
-            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
-        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+        if self._nvml is None:
+            return self._smi_once()
+        self._stop.set()
+        self._thread.join(timeout=1.0)
+        reasons = [name for name, bit in self.REASONS if self.reason_bits & bit]
+        return {"sm_mhz": float(np.median(self.sm)) if self.sm else None, "sm_max_mhz": self.max_sm, "reasons": reasons,
+                "samples": len(self.sm), "power_w_max": max(self.power) if self.power else None, "source": "nvml"}
+
+    def _smi_once(self) -> dict:
+        try:
+            out = subprocess.run(["nvidia-smi", f"--id={self.index}", "--query-gpu=clocks.sm,clocks.max.sm", "--format=csv,noheader,nounits"],
+                                 capture_output=True, text=True, timeout=10).stdout.strip().split(",")
+            return {"sm_mhz": float(out[0]), "sm_max_mhz": float(out[1]), "reasons": [], "samples": 1, "source": "nvidia-smi after the region"}
+        except Exception:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["clock query unavailable"], "samples": 0}
+
+
+def max_over_ranks(value: float, world: int, device=None) -> float:
+    """Largest `value` over all ranks of the default process group (the job's time is its slowest rank's)."""
+    if world <= 1:
+        return value
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
 
 
 # --------------------------------------------------------------------------------------- CPU oracle leg
 def oracle_sample(cfg: dict, sample_params: int):
-    """One oracle step of all G groups (+ FedAvg/H) on the first `sample_params` parameters.
-    Returns (params/s, seconds, threads)."""
+    """One oracle step of all G groups and one FedAvg on the first `sample_params` parameters of every
+    buffer, as the oracle stands, on one host thread.  The sample's inputs come from the shared generator
+    (filled on the GPU when there is one, since the fill is not what is being timed, then copied to the
+    host).  Returns (params/s with FedAvg counted once per H steps, seconds of oracle work, threads)."""
     from oracle import fls_oracle as orc
+    try:
+        from threadpoolctl import threadpool_limits
+    except Exception:                                   # pragma: no cover
+        import contextlib
+        threadpool_limits = lambda limits: contextlib.nullcontext()
     G, S, R = cfg["groups"], cfg["shard_dim"], cfg["replicate_dim"]
     K = S * R
     P = min(sample_params, cfg["n_params"])
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    f32 = cfg["grad_dtype"] == "f32"
     hp = orc.Hyper(cfg["lr"], cfg["beta1"], cfg["beta2"], cfg["eps"], cfg["weight_decay"], cfg["max_grad_norm"])
-    th0 = sy.normal_fill_(torch.empty(P), sy.stream_key(cfg["seed"], sy.KIND_MASTER), cfg["master_sigma"]).numpy()
+    th0 = sy.normal_fill_(torch.empty(P, device=dev), sy.stream_key(cfg["seed"], sy.KIND_MASTER), cfg["master_sigma"]).cpu().numpy()
     states = [orc.GroupState(th0.copy(), np.zeros(P, np.float32), np.zeros(P, np.float32), None) for _ in range(G)]
-    bits = [[sy.normal_fill_(torch.empty(P, dtype=torch.bfloat16), sy.stream_key(cfg["seed"], sy.KIND_GRAD, 1, g, k), cfg["grad_sigma"])
-             .view(torch.int16).numpy().view(np.uint16) for k in range(K)] for g in range(G)]
-    t0 = time.perf_counter()
+    raw = []
     for g in range(G):
-        grads = [orc.bf16_bits_to_f64(b) for b in bits[g]]
-        orc.sync_step_group(states[g], grads, S, R, 1, hp)
-    t_step = time.perf_counter() - t0
-    t0 = time.perf_counter()
-    orc.fedavg(states, [sy.sample_count(cfg["seed"], g) for g in range(G)] if cfg["weights"] == "counts" else None)
-    t_avg = time.perf_counter() - t0
+        row = []
+        for k in range(K):
+            scale = sy.uniform_scale(cfg["seed"], g, k) if cfg["per_buffer_scale"] else 1.0
+            t = sy.normal_fill_(torch.empty(P, dtype=torch.float32 if f32 else torch.bfloat16, device=dev),
+                                sy.stream_key(cfg["seed"], sy.KIND_GRAD, 1, g, k), cfg["grad_sigma"], scale).cpu()
+            row.append(t.numpy() if f32 else t.view(torch.int16).numpy().view(np.uint16))
+        raw.append(row)
+    counts = [sy.sample_count(cfg["seed"], g) for g in range(G)] if cfg["weights"] == "counts" else None
+    with threadpool_limits(limits=1):
+        t0 = time.perf_counter()
+        for g in range(G):
+            grads = [x.astype(np.float64) if f32 else orc.bf16_bits_to_f64(x) for x in raw[g]]
+            orc.sync_step_group(states[g], grads, S, R, 1, hp)
+            del grads
+        t_step = time.perf_counter() - t0
+        t0 = time.perf_counter()
+        orc.fedavg(states, counts)
+        t_avg = time.perf_counter() - t0
     sec = t_step + t_avg / cfg["sync_period"]
     return G * P / sec, t_step + t_avg, 1
 
 
 def run_reference(args, cfg):
+    """The reference arm of this build is the CPU oracle (the paper ships no code): every "step" is one
+    oracle step + FedAvg/H on a bounded sample of the workload.  Rank 0 only."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    sample = 1 << 22
+    sample = 1 << 24
     vals, secs = [], []
-    for _ in range(args.warmup and 1):
+    if args.warmup:
         oracle_sample(cfg, 1 << 18)
-    for _ in range(max(1, min(args.steps, 3))):
+    n = max(1, min(args.steps, 3))
+    for _ in range(n):
         v, s, cores = oracle_sample(cfg, sample)
         vals.append(v); secs.append(s)
     value = float(np.mean(vals))
-    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": len(vals),
+    what = f"one oracle step of all {cfg['groups']} groups + FedAvg/H on the first {min(sample, cfg['n_params'])} params of every buffer"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": n,
             "warmup": 1 if args.warmup else 0, "ms_per_step": 1e3 * float(np.mean(secs)), "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": cfg["name"], "sample": f"first {sample} params of each of {cfg['groups']} groups"},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
-                             "sample": f"one oracle step (+FedAvg/H) on the first {sample} params of each group"},
+            "config": {"workload": cfg["name"], "sample": what},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": what},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
 
@@ -197,11 +251,7 @@ def run_ours(args, cfg):
             one_step()
         e1.record(stream)
         barrier()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        ms = max_over_ranks(e0.elapsed_time(e1), world, "cuda")
         return ms, fls.fls_get_launch_count(sess.plan) - l0
 
     for _ in range(args.warmup):
@@ -219,7 +269,10 @@ def run_ours(args, cfg):
 
     # end to end: gradients start in pinned host memory, norms come back to the host, every step
     e2e = None
-    if not args.no_e2e:
+    eg_bytes = 4 if cfg["grad_dtype"] == "f32" else 2
+    if not args.no_e2e and G * sess.K * sess.n_padded * eg_bytes > args.e2e_max_gb * 2 ** 30:
+        e2e = {"value": None, "unit": UNIT, "skipped": f"pinned staging above --e2e-max-gb {args.e2e_max_gb}"}
+    elif not args.no_e2e:
         host = [[torch.empty(sess.n_padded, dtype=sess.grad_torch_dtype).pin_memory() for _ in range(sess.K)] for _ in range(G)]
         for g in range(G):
             for k in range(sess.K):
@@ -236,9 +289,7 @@ def run_ours(args, cfg):
         for _ in range(n_e2e):
             e2e_step()
         torch.cuda.synchronize()
-        dt = time.perf_counter() - t0
-        if world > 1:
-            t = torch.tensor([dt], device="cuda"); dist.all_reduce(t, op=dist.ReduceOp.MAX); dt = float(t.item())
+        dt = max_over_ranks(time.perf_counter() - t0, world, "cuda")
         eg = 4 if cfg["grad_dtype"] == "f32" else 2
         e2e = {"value": world * G * P * n_e2e / dt, "unit": UNIT, "h2d_bytes_per_step": G * sess.K * sess.n_padded * eg,
                "d2h_bytes_per_step": 4 * G, "steps": n_e2e, "ms_per_step": 1e3 * dt / n_e2e}
@@ -276,12 +327,15 @@ def run_ours(args, cfg):
             "kernels": kernels, "ms_per_step_profiled": ms_prof / args.steps,
             "gpu_launches": launches, "clocks": clocks, "e2e": e2e,
         }
-        if world == 1 and not args.no_cpu_baseline:
-            v, s, cores = oracle_sample(cfg, 1 << 22)
-            line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "seconds": s,
-                                    "sample": f"one oracle step (+FedAvg/H) on the first {1 << 22} params of each of {G} groups"}
-        print(json.dumps(line), flush=True)
     sess.close()
+    if rank == 0:
+        if world == 1 and not args.no_cpu_baseline:
+            torch.cuda.empty_cache()
+            n_s = min(1 << 25, P)
+            v, s, cores = oracle_sample(cfg, n_s)
+            line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "seconds": s,
+                                    "sample": f"one oracle step of all {G} groups + FedAvg/H on the first {n_s} params of every buffer"}
+        print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
 
@@ -295,6 +349,7 @@ def main():
     ap.add_argument("--config", default=DEFAULT_CONFIG, choices=[c["name"] for c in sy.CONFIGS])
     ap.add_argument("--opt-state", action="store_true", help="FedAvg also averages m and v")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--e2e-max-gb", type=float, default=48.0, help="skip the end-to-end pass if its pinned host staging would exceed this")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ctas-reduce", type=int, default=0)
     ap.add_argument("--ctas-adamw", type=int, default=0)

@@ -7,7 +7,8 @@ import os
 from typing import Optional, Sequence
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libfls.so")
+# FLS_LIBRARY points the binding at another build of the same ABI (e.g. one compiled with other tuning flags)
+LIB_PATH = os.environ.get("FLS_LIBRARY") or os.path.join(_PKG, "libfls.so")
 
 FLS_OK, FLS_EINVAL, FLS_EALIGN, FLS_EPTR, FLS_ESIZE, FLS_ECUDA, FLS_ESTATE = range(7)
 FLS_GRAD_BF16, FLS_GRAD_F32 = 0, 1

@@ -451,8 +451,16 @@ __global__ void __launch_bounds__(kThreads, MINB) fls_fedavg_kernel(const __grid
 // ------------------------------------------------------------------------------------------------
 // Launchers.
 // ------------------------------------------------------------------------------------------------
-constexpr int kFlatThreads = 1024, kFlatMinB = 2;      // SG == 0 with a static K
-constexpr int kLevelThreads = 512, kLevelMinB = 3;     // two-level orders with a static K
+#ifndef FLS_FLAT_THREADS
+#define FLS_FLAT_THREADS 1024
+#define FLS_FLAT_MINB 2
+#endif
+#ifndef FLS_LEVEL_THREADS
+#define FLS_LEVEL_THREADS 512
+#define FLS_LEVEL_MINB 3
+#endif
+constexpr int kFlatThreads = FLS_FLAT_THREADS, kFlatMinB = FLS_FLAT_MINB;       // SG == 0 with a static K
+constexpr int kLevelThreads = FLS_LEVEL_THREADS, kLevelMinB = FLS_LEVEL_MINB;   // two-level orders with a static K
 constexpr int kAnyThreads = 256, kAnyMinB = 2;         // run-time K: batches of 8 loads need the registers
 
 inline int reduce_threads(const ReduceArgs& a, int sg) {
