@@ -16,7 +16,6 @@ import json
 import os
 import subprocess
 import sys
-import threading
 import time
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
@@ -46,15 +45,16 @@ def measured_peak_gbs():
 
 # --------------------------------------------------------------------------------------- clocks
 class ClockSampler:
-    """Samples the SM clock and the throttle reasons of one GPU while the timed region runs.  Reads NVML
-    directly every few milliseconds (the timed region of a small workload lasts only tens of ms); falls
-    back to one nvidia-smi query if the NVML binding is missing.  Nothing is ever set, only read."""
+    """Samples the SM clock and the throttle reasons of one GPU while the timed region runs: the main thread
+    reads NVML about once a millisecond while it waits for the region's end event (the region of a small
+    workload lasts only tens of ms, too short for nvidia-smi's loop mode).  Falls back to one nvidia-smi
+    query if the NVML binding is missing.  Nothing is ever set, only read."""
     REASONS = (("hw_slowdown", 0x8), ("hw_thermal_slowdown", 0x40), ("sw_thermal_slowdown", 0x20), ("sw_power_cap", 0x4),
                ("hw_power_brake_slowdown", 0x80))
 
     def __init__(self, index: int):
         self.index, self.sm, self.reason_bits, self.power = index, [], 0, []
-        self.max_sm, self._stop, self._thread, self._nvml = None, threading.Event(), None, None
+        self.max_sm, self._nvml = None, None
 
     def start(self):
         try:
@@ -63,8 +63,6 @@ class ClockSampler:
             self._nvml = pynvml
             self._h = pynvml.nvmlDeviceGetHandleByIndex(self._physical_index())
             self.max_sm = float(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
-            self._thread = threading.Thread(target=self._poll, daemon=True)
-            self._thread.start()
         except Exception:
             self._nvml = None
 
@@ -75,23 +73,28 @@ class ClockSampler:
             return int(ids[self.index])
         return self.index
 
-    def _poll(self):
+    def sample(self):
+        """One reading; called from the main thread while it waits for the timed region's end event."""
         nv = self._nvml
-        while not self._stop.is_set():
-            try:
-                self.sm.append(float(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
-                self.reason_bits |= int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h)) if hasattr(nv, "nvmlDeviceGetCurrentClocksEventReasons") \
-                    else int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
-                self.power.append(nv.nvmlDeviceGetPowerUsage(self._h) / 1000.0)
-            except Exception:
-                pass
-            time.sleep(0.002)
+        if nv is None:
+            return
+        try:
+            self.sm.append(float(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+            self.reason_bits |= int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h)) if hasattr(nv, "nvmlDeviceGetCurrentClocksEventReasons") \
+                else int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+            self.power.append(nv.nvmlDeviceGetPowerUsage(self._h) / 1000.0)
+        except Exception:
+            pass
+
+    def wait_for(self, event):
+        """Waits for a CUDA event, sampling the clocks every millisecond or so meanwhile."""
+        while not event.query():
+            self.sample()
+            time.sleep(0.001)
 
     def stop(self) -> dict:
         if self._nvml is None:
             return self._smi_once()
-        self._stop.set()
-        self._thread.join(timeout=1.0)
         reasons = [name for name, bit in self.REASONS if self.reason_bits & bit]
         return {"sm_mhz": float(np.median(self.sm)) if self.sm else None, "sm_max_mhz": self.max_sm, "reasons": reasons,
                 "samples": len(self.sm), "power_w_max": max(self.power) if self.power else None, "source": "nvml"}
@@ -240,7 +243,7 @@ def run_ours(args, cfg):
             dist.barrier()
             torch.cuda.synchronize()
 
-    def timed(n_steps, profiling):
+    def timed(n_steps, profiling, sampler=None):
         fls.fls_set_profiling(sess.plan, profiling)
         barrier()
         l0 = fls.fls_get_launch_count(sess.plan)
@@ -250,6 +253,8 @@ def run_ours(args, cfg):
         for _ in range(n_steps):
             one_step()
         e1.record(stream)
+        if sampler is not None:
+            sampler.wait_for(e1)
         barrier()
         ms = max_over_ranks(e0.elapsed_time(e1), world, "cuda")
         return ms, fls.fls_get_launch_count(sess.plan) - l0
@@ -259,7 +264,7 @@ def run_ours(args, cfg):
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    ms_total, launches = timed(args.steps, False)
+    ms_total, launches = timed(args.steps, False, sampler if rank == 0 else None)
     fedavg_calls = n_fedavg[0]
     clocks = sampler.stop() if rank == 0 else None
     # second pass over the same number of steps with events around every kernel: per-kernel durations
@@ -299,7 +304,9 @@ def run_ours(args, cfg):
         peak, peak_kind = measured_peak_gbs()
         N = sess.n_padded
         eg = 4 if cfg["grad_dtype"] == "f32" else 2
-        per_launch = {"reduce": N * (sess.K * eg + 4), "adamw": N * 30, "fedavg": N * G * 10}
+        # FedAvg runs one launch per averaged array: parameters move 10 B per group-element (4 read, 4 + 2
+        # written), m and v 8 B each; the figure is the mean over the launches of one call
+        per_launch = {"reduce": N * (sess.K * eg + 4), "adamw": N * 30, "fedavg": N * G * (26 / 3 if args.opt_state else 10)}
         kernels = {}
         for i, name in enumerate(("reduce", "adamw", "fedavg")):
             if kn[i]:
@@ -340,6 +347,88 @@ def run_ours(args, cfg):
         dist.destroy_process_group()
 
 
+# --------------------------------------------------------------------------------------- bandwidth sweep
+SWEEP_SPLITS = [(2, 1), (2, 2), (2, 4), (4, 4), (4, 8), (8, 8)]       # (G, K): R*G = 2, 4, 8, 16, 32, 64
+
+
+def sweep_points(p_exps=(20, 22, 24, 26, 28, 30)):
+    for e in p_exps:
+        for G, K in SWEEP_SPLITS:
+            for order in ("fsdp", "hsdp"):
+                if order == "hsdp" and K < 2:
+                    continue
+                for dt in ("bf16", "f32"):
+                    S, R = (K, 1) if order == "fsdp" else (K // 2, 2)
+                    yield dict(P=1 << e, G=G, K=K, S=S, R=R, order=order, dtype=dt)
+
+
+def run_sweep(args):
+    """HBM GB/s of the fused reduce+AdamW step and of FedAvg over flat P = 2^20 .. 2^30, R*G in 2..64,
+    FL+FSDP vs FL+HSDP order, bf16 vs fp32 gradients.  One JSON line per point into --sweep-out.  Points whose
+    buffers would not fit in 90 % of the free HBM are reported as skipped; points whose working set is below
+    twice the L2 get an L2 flush (a 512 MB write) before every timed call."""
+    from paper_2609_20359_b200 import build
+    from paper_2609_20359_b200 import _binding as fls
+    from paper_2609_20359_b200.session import Session
+    build.build()
+    torch.cuda.set_device(0)
+    peak, peak_kind = measured_peak_gbs()
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    block = 1 << 22
+    seedbuf = {dt: sy.normal_fill_(torch.empty(block, dtype=torch.float32 if dt == "f32" else torch.bfloat16, device="cuda"),
+                                   sy.stream_key(5, sy.KIND_GRAD, 1, 0, 0), 1e-3) for dt in ("bf16", "f32")}
+    seedth = sy.normal_fill_(torch.empty(block, device="cuda"), sy.stream_key(5, sy.KIND_MASTER), 0.02)
+    out = open(args.sweep_out, "w")
+    exps = [int(x) for x in args.sweep_exps.split(",")]
+    for pt in sweep_points(exps):
+        P, G, K = pt["P"], pt["G"], pt["K"]
+        eg = 4 if pt["dtype"] == "f32" else 2
+        need = G * K * P * eg + G * 14 * P + 4 * P + (64 << 20)
+        free, _ = torch.cuda.mem_get_info()
+        rec = dict(pt, bytes_needed=need)
+        if need > 0.9 * free:
+            rec["skipped"] = "exceeds HBM"
+            out.write(json.dumps(rec) + "\n"); out.flush()
+            continue
+        sess = Session(P, None, G, pt["S"], pt["R"], 1, pt["dtype"], 8, False)
+        for g in range(G):
+            # the fill repeats a 4 Mi-element generator block (bandwidth does not depend on the values)
+            for buf, src in [(sess.master[g], seedth)] + [(b, seedbuf[pt["dtype"]]) for b in sess.grads[g]]:
+                n = buf.numel()
+                if n >= block:
+                    buf[: n // block * block].view(-1, block).copy_(src.expand(n // block, block))
+                buf[n // block * block:].copy_(src[: n % block])
+        torch.cuda.synchronize()
+        resident = need < 2 * 126e6
+        stream = torch.cuda.current_stream()
+        def timed(call, reps):
+            ts = []
+            for i in range(reps + 3):
+                if resident:
+                    flush.fill_(i & 0xFF)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream); call(); e1.record(stream)
+                torch.cuda.synchronize()
+                if i >= 3:
+                    ts.append(e0.elapsed_time(e1))
+            return float(np.median(ts))
+        ms_step = timed(lambda: sess.step(stream=stream), 5)
+        ms_avg = timed(lambda: sess.fedavg(None, stream=stream), 3)
+        rep = fls.fls_comm_report(sess.plan)
+        rec.update(ms_sync_step=ms_step, ms_fedavg=ms_avg, l2_flush=resident,
+                   sync_step_gbs=rep["hbm_bytes_sync_step"] / ms_step / 1e6, fedavg_gbs=rep["hbm_bytes_fedavg"] / ms_avg / 1e6,
+                   synced_params_per_s=G * P / (ms_step / 1e3))
+        rec["sync_step_frac_of_8tbs"] = rec["sync_step_gbs"] / 8000.0
+        rec["fedavg_frac_of_8tbs"] = rec["fedavg_gbs"] / 8000.0
+        rec["peak_gbs"], rec["peak_kind"] = peak, peak_kind
+        out.write(json.dumps(rec) + "\n"); out.flush()
+        sess.close()
+        del sess
+        torch.cuda.empty_cache()
+    out.close()
+    print(json.dumps({"sweep": args.sweep_out}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -363,7 +452,14 @@ def main():
     ap.add_argument("--replicate-dim", type=int, default=0, help="override R_rep")
     ap.add_argument("--grad-dtype", default="", choices=["", "bf16", "f32"], help="override the gradient dtype")
     ap.add_argument("--keep-units", action="store_true", help="with --n-params: keep the unit table's proportions")
+    ap.add_argument("--sweep", action="store_true", help="run the bandwidth sweep instead of the benchmark")
+    ap.add_argument("--sweep-out", default="gpurun_out/sweep.jsonl")
+    ap.add_argument("--sweep-exps", default="20,22,24,26,28,30", help="log2 of the parameter counts to sweep")
     args = ap.parse_args()
+    if args.sweep:
+        os.makedirs(os.path.dirname(args.sweep_out) or ".", exist_ok=True)
+        run_sweep(args)
+        return
     cfg = sy.config_by_name(args.config)
     if args.n_params:
         cfg.update(n_params=args.n_params, unit_numel=[args.n_params], name=cfg["name"] + f"[P={args.n_params}]")

@@ -114,6 +114,25 @@ def test_two_level_order_differs_from_flat_where_fp32_rounds(fls):
     assert not np.array_equal(res[(8, 1)], res[(4, 2)])
 
 
+def _sweep_shapes():
+    import bench
+    seen = set()
+    for pt in bench.sweep_points((17,)):
+        key = (pt["G"], pt["S"], pt["R"], pt["dtype"])
+        if key not in seen:
+            seen.add(key)
+            yield key
+
+
+@pytest.mark.parametrize("G,S,R_rep,dtype", list(_sweep_shapes()))
+def test_bandwidth_sweep_shapes(fls, G, S, R_rep, dtype):
+    """Every (groups, buffers, order, gradient dtype) point of the bandwidth sweep, at P = 2^17 + a step and a FedAvg."""
+    c = Case([1 << 17], G, S, R_rep, H=1, Q=8, grad_dtype=dtype, hp=orc.Hyper(max_grad_norm=0.05))
+    c.step()
+    c.compare()
+    c.close()
+
+
 # ------------------------------------------------------------------ FedAvg
 @pytest.mark.parametrize("G,opt_state,counts", [(1, True, [9]), (3, False, [1, 2, 5]), (8, True, None), (9, True, "rand"), (64, False, "rand")])
 def test_fedavg(fls, G, opt_state, counts):
