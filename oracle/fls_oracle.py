@@ -96,19 +96,23 @@ def plan(unit_numel: Sequence[int], S: int, Q: int = 1) -> Layout:
     return Layout(list(unit_numel), S, Q, M, padded, off, soff, int(sum(unit_numel)), o, so)
 
 
+def addresses_of(L: Layout, logical_index) -> tuple:
+    """For logical elements (index into the concatenation of all units): their index in the unsharded
+    order and their address in the rank-major shard order [S][shard_numel]."""
+    p = np.asarray(logical_index, dtype=np.int64)
+    starts = np.concatenate([[0], np.cumsum(L.unit_numel)]).astype(np.int64)
+    u = np.searchsorted(starts, p, side="right") - 1                 # unit of each element
+    i = p - starts[u]                                                # index inside the unit
+    M = np.asarray(L.unit_shard_numel, dtype=np.int64)[u]
+    j = np.asarray(L.unit_offset, dtype=np.int64)[u] + i
+    a = (i // M) * L.shard_numel + np.asarray(L.unit_shard_offset, dtype=np.int64)[u] + i % M
+    return j, a
+
+
 def _addresses(L: Layout):
-    """For every logical element: its index in the unsharded order and its address
-    in the rank-major shard order [S][shard_numel]."""
+    """addresses_of every logical element, cached."""
     if L._addr_unsharded is None:
-        ju, ja = [], []
-        for u, n in enumerate(L.unit_numel):
-            i = np.arange(n, dtype=np.int64)
-            ju.append(L.unit_offset[u] + i)
-            s = i // L.unit_shard_numel[u]
-            k = L.unit_shard_offset[u] + i % L.unit_shard_numel[u]
-            ja.append(s * L.shard_numel + k)
-        L._addr_unsharded = np.concatenate(ju)
-        L._addr_sharded = np.concatenate(ja)
+        L._addr_unsharded, L._addr_sharded = addresses_of(L, np.arange(L.n_params, dtype=np.int64))
     return L._addr_unsharded, L._addr_sharded
 
 

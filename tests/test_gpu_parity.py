@@ -305,49 +305,82 @@ def test_bind_rejects_bad_buffers(fls):
 
 
 # ------------------------------------------------------------------ full size, in the benchmark's launch configuration
-def test_full_size_gpt2_small_sampled(fls):
-    """P = 124,439,808, G = 4, K = 8 (the benchmark workload).  The oracle computes every group's
-    norm over the full gradient (chunked), then the step and FedAvg at sampled positions: first and
-    last tiles, tile and shard boundaries, and random indices."""
-    from paper_2609_20359_b200.session import Session
-    cfg = sy.CONFIGS[1]
-    P, G, K = cfg["n_params"], cfg["groups"], cfg["shard_dim"]
-    hp = orc.Hyper()
-    s = Session(P, cfg["unit_numel"], G, K, 1, cfg["sync_period"], "bf16", 8, False)
+def _fill_full_size(s, cfg, L):
+    """Fills a Session's device buffers from the generator by LOGICAL index (what the oracle samples)."""
     th_key = sy.stream_key(cfg["seed"], sy.KIND_MASTER)
-    for g in range(G):
-        sy.normal_fill_(s.master[g], th_key, cfg["master_sigma"])
-        for k in range(K):
-            sy.normal_fill_(s.grads[g][k], sy.stream_key(cfg["seed"], sy.KIND_GRAD, 1, g, k), cfg["grad_sigma"],
-                            sy.uniform_scale(cfg["seed"], g, k))
-    counts = [sy.sample_count(cfg["seed"], g) for g in range(G)]
+    starts = np.concatenate([[0], np.cumsum(L.unit_numel)])
+    for g in range(cfg["groups"]):
+        for u, n in enumerate(L.unit_numel):
+            M = L.unit_shard_numel[u]
+            for sh in range(L.S):
+                ln = min(M, n - sh * M)
+                if ln > 0:
+                    a0 = sh * L.shard_numel + L.unit_shard_offset[u]
+                    sy.normal_fill_(s.master[g][a0:a0 + ln], th_key, cfg["master_sigma"], start=int(starts[u]) + sh * M)
+            for k in range(s.K):
+                scale = sy.uniform_scale(cfg["seed"], g, k) if cfg["per_buffer_scale"] else 1.0
+                sy.normal_fill_(s.grads[g][k][L.unit_offset[u]:L.unit_offset[u] + n], sy.stream_key(cfg["seed"], sy.KIND_GRAD, 1, g, k),
+                                cfg["grad_sigma"], scale, start=int(starts[u]))
+    torch.cuda.synchronize()
+
+
+def _oracle_norm_full(grads, S, R_rep, chunk=1 << 22, threads=16):
+    """Norm of one group's mean gradient over the whole (padded, unsharded) buffers: the oracle's reduce_mean
+    and grad_norm on chunks copied to the host, chunks spread over host threads, partial sums added in order."""
+    from concurrent.futures import ThreadPoolExecutor
+    n = grads[0].numel()
+    def one(lo):
+        part = [orc.bf16_bits_to_f64(bf16_bits(g[lo:lo + chunk])) for g in grads]
+        return orc.grad_norm(orc.reduce_mean(part, S, R_rep)) ** 2
+    with ThreadPoolExecutor(threads) as ex:
+        parts = list(ex.map(one, range(0, n, chunk)))
+    return math.sqrt(math.fsum(parts))
+
+
+@pytest.mark.parametrize("cfg_index", [1, 2, 3])
+def test_full_size_workloads_sampled(fls, cfg_index):
+    """The GPT-2-small, Llama-3.2-1B (18 units, two-level order) and Llama-3.1-8B-block (9 tensors) workloads at
+    full size, launched as the benchmark launches them.  The oracle computes every group's norm over the full
+    gradient, then the step and FedAvg at sampled logical positions: the first and last 4096 parameters, 16
+    around every unit and shard boundary, and 200,000 random ones."""
+    from paper_2609_20359_b200.session import Session
+    cfg = sy.CONFIGS[cfg_index]
+    P, G, S, R_rep = cfg["n_params"], cfg["groups"], cfg["shard_dim"], cfg["replicate_dim"]
+    K = S * R_rep
+    hp = orc.Hyper()
+    L = orc.plan(cfg["unit_numel"], S, 8)
+    s = Session(P, cfg["unit_numel"], G, S, R_rep, cfg["sync_period"], "bf16", 8, False)
+    assert s.n_padded == L.n_padded
+    _fill_full_size(s, cfg, L)
+    counts = [sy.sample_count(cfg["seed"], g) for g in range(G)] if cfg["weights"] == "counts" else None
     rng = np.random.default_rng(3)
-    idx = np.unique(np.concatenate([np.arange(0, 4096), np.arange(P - 4096, P), rng.integers(0, P, 200_000),
-                                    (np.arange(1, K)[:, None] * (P // K) + np.arange(-8, 8)[None, :]).ravel()]))
+    starts = np.concatenate([[0], np.cumsum(L.unit_numel)])
+    edges = [starts[u] + sh * L.unit_shard_numel[u] for u in range(len(L.unit_numel)) for sh in range(S)]
+    idx = np.concatenate([np.arange(0, 4096), np.arange(P - 4096, P), rng.integers(0, P, 200_000),
+                          (np.asarray(edges)[:, None] + np.arange(-8, 8)[None, :]).ravel()])
+    idx = np.unique(idx[(idx >= 0) & (idx < P)])
     tidx = torch.from_numpy(idx)
-    th0 = sy.normal_at(tidx, th_key, cfg["master_sigma"]).numpy()
-    # oracle norms over the full buffers (gradients come from the generator, copied to the host)
-    norms, gbar_s = [], []
-    CH = 1 << 23
+    j_np, a_np = orc.addresses_of(L, idx)
+    jt, at = torch.from_numpy(j_np).cuda(), torch.from_numpy(a_np).cuda()
+    th0 = sy.normal_at(tidx, sy.stream_key(cfg["seed"], sy.KIND_MASTER), cfg["master_sigma"]).numpy()
+    assert np.array_equal(s.master[0][at].cpu().numpy(), th0)            # the fill put every sample where the oracle's planner says
+    norms, gbar_s, samp_last = [], [], None
     for g in range(G):
-        tot = 0.0
-        for lo in range(0, P, CH):
-            chunk = [orc.bf16_bits_to_f64(bf16_bits(s.grads[g][k][lo:lo + CH])) for k in range(K)]
-            gb = orc.reduce_mean(chunk, K, 1)
-            tot += orc.grad_norm(gb) ** 2
-        norms.append(math.sqrt(tot))
+        norms.append(_oracle_norm_full(s.grads[g], S, R_rep))
         samp = [orc.bf16_bits_to_f64(bf16_bits(sy.normal_at(tidx, sy.stream_key(cfg["seed"], sy.KIND_GRAD, 1, g, k), cfg["grad_sigma"],
-                                                             sy.uniform_scale(cfg["seed"], g, k), torch.bfloat16))) for k in range(K)]
-        gbar_s.append(orc.reduce_mean(samp, K, 1))
+                                                             sy.uniform_scale(cfg["seed"], g, k) if cfg["per_buffer_scale"] else 1.0,
+                                                             torch.bfloat16))) for k in range(K)]
+        gbar_s.append(orc.reduce_mean(samp, S, R_rep))
+        samp_last = samp
     due = s.step()
     torch.cuda.synchronize()
     assert not due
     got_n = s.norms().cpu().numpy().astype(np.float64)
     assert np.allclose(got_n, norms, rtol=1e-6, atol=0), (got_n, norms)
     # fp32 running sum against the exactly rounded mean: identical except where a tiny addend loses bits
-    got_g = s.reduced_grad()[tidx.cuda()].cpu().numpy()
+    got_g = s.reduced_grad()[at].cpu().numpy()
     assert np.mean(got_g == gbar_s[G - 1]) > 0.999
-    assert np.all(np.abs(got_g.astype(np.float64) - gbar_s[G - 1]) <= 2.0 ** -24 * np.sum(np.abs(samp), axis=0))
+    assert np.all(np.abs(got_g.astype(np.float64) - gbar_s[G - 1]) <= 2.0 ** -24 * np.sum(np.abs(samp_last), axis=0))
     states = []
     for g in range(G):
         c = orc.clip_coef(norms[g], hp.max_grad_norm)
@@ -355,15 +388,16 @@ def test_full_size_gpt2_small_sampled(fls):
         z = np.zeros(idx.size, np.float32)
         th, m, v, bits = orc.adamw(th0, z, z, gbar_s[g], c, 1, hp.lr, hp.beta1, hp.beta2, hp.eps, hp.weight_decay)
         states.append(orc.GroupState(th, m, v, bits))
-        assert_state_close(s.master[g][tidx.cuda()].cpu().numpy(), th, f"master[{g}]")
-        assert_state_close(s.m[g][tidx.cuda()].cpu().numpy(), m, f"m[{g}]", 1e-5, "rms")
-        assert_state_close(s.v[g][tidx.cuda()].cpu().numpy(), v, f"v[{g}]", 1e-5, "rms")
-        assert_bf16_close(bf16_bits(s.param_bf16[g][tidx.cuda()]), bits, f"bf16[{g}]")
+        assert_state_close(s.master[g][at].cpu().numpy(), th, f"master[{g}]")
+        assert_state_close(s.m[g][at].cpu().numpy(), m, f"m[{g}]", 1e-5, "rms")
+        assert_state_close(s.v[g][at].cpu().numpy(), v, f"v[{g}]", 1e-5, "rms")
+        assert_bf16_close(bf16_bits(s.param_bf16[g][jt]), bits, f"bf16[{g}]")
     orc.fedavg(states, counts)
     s.fedavg(counts)
     torch.cuda.synchronize()
     for g in range(G):
-        assert_state_close(s.master[g][tidx.cuda()].cpu().numpy(), states[g].theta, f"fedavg master[{g}]")
-        assert_bf16_close(bf16_bits(s.param_bf16[g][tidx.cuda()]), states[g].param_bf16, f"fedavg bf16[{g}]")
-    assert torch.equal(s.master[0], s.master[G - 1])
+        assert_state_close(s.master[g][at].cpu().numpy(), states[g].theta, f"fedavg master[{g}]")
+        assert_bf16_close(bf16_bits(s.param_bf16[g][jt]), states[g].param_bf16, f"fedavg bf16[{g}]")
+    assert torch.equal(s.master[0], s.master[G - 1]) and torch.equal(s.param_bf16[0], s.param_bf16[G - 1])
+    assert s.status() == 0
     s.close()

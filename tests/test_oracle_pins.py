@@ -103,6 +103,21 @@ def test_planner_brute_force(units, S, Q):
         p += n
 
 
+def test_addresses_of_matches_elementwise_definition():
+    units, S, Q = [5, 1, 12, 7], 3, 4
+    L = orc.plan(units, S, Q)
+    j, a = orc.addresses_of(L, np.arange(sum(units)))
+    p = 0
+    for u, n in enumerate(units):
+        for i in range(n):
+            s_, k = divmod(i, L.unit_shard_numel[u])
+            assert j[p] == sum(L.unit_padded[:u]) + i
+            assert a[p] == s_ * L.shard_numel + sum(L.unit_shard_numel[:u]) + k
+            p += 1
+    jj, aa = orc.addresses_of(L, [24, 0, 17])
+    assert list(jj) == [j[24], j[0], j[17]] and list(aa) == [a[24], a[0], a[17]]
+
+
 def test_planner_p17_numbers():
     L = orc.plan([17], 4, 1)
     assert (L.n_padded, L.shard_numel, L.unit_shard_numel) == (20, 5, [5])
