@@ -79,6 +79,37 @@ def test_layouts_and_orders(fls, units, G, S, R_rep, Q, dtype):
     c.close()
 
 
+def test_large_segment_table_uses_global_lookup(fls):
+    """200 units x 4 shards = 800 segments: above the 512 that travel in the kernel parameters, so the kernels
+    bisect the table in global memory."""
+    rng = np.random.default_rng(8)
+    units = [int(x) for x in rng.integers(1, 3000, 200)]
+    c = Case(units, 2, 4, 2, H=1, Q=8, opt_state=True, hp=orc.Hyper(max_grad_norm=0.05))
+    assert c.sess.layout["n_segments"] == 800
+    for _ in range(2):
+        c.step([3, 1])
+        c.compare()
+    c.close()
+
+
+@pytest.mark.parametrize("ctas,descending", [(1, 0), (3, 1), (0, 1), (64, 0)])
+def test_tuned_launch_shapes_give_identical_results(fls, ctas, descending):
+    """Persistent / descending launch shapes of the AdamW and FedAvg kernels change scheduling only: the
+    results are bit-identical to the default one-pass shape."""
+    def run(tune):
+        c = Case([40000, 30011, 5000], 3, 4, 1, H=1, Q=8, opt_state=True, hp=orc.Hyper(max_grad_norm=0.05))
+        if tune:
+            for kern in (fls.FLS_KERNEL_REDUCE, fls.FLS_KERNEL_ADAMW, fls.FLS_KERNEL_FEDAVG):
+                fls.fls_plan_tune(c.sess.plan, kern, ctas, descending)
+        for _ in range(2):
+            c.step([1, 2, 3])
+        c.compare()
+        out = [x.clone() for x in c.sess.master + c.sess.m + c.sess.v + c.sess.param_bf16]
+        c.close()
+        return out
+    assert all(torch.equal(x, y) for x, y in zip(run(False), run(True)))
+
+
 def test_reduced_gradient_matches_oracle_exactly_for_bf16(fls):
     """With bf16 inputs of similar magnitude the fp32 running sum is exact, so the mean gradient is
     bit-identical to the oracle's (this case is small enough that no element loses bits)."""
