@@ -227,6 +227,10 @@ def run_ours(args, cfg):
             fls.fls_plan_tune(sess.plan, {"reduce": 0, "adamw": 1, "fedavg": 2}[kern], val, -1)
     if args.descending_adamw:
         fls.fls_plan_tune(sess.plan, fls.FLS_KERNEL_ADAMW, 0, 1)
+    if args.ascending_adamw:
+        fls.fls_plan_tune(sess.plan, fls.FLS_KERNEL_ADAMW, 0, 0)
+    if args.no_overlap:
+        fls.fls_plan_tune(sess.plan, fls.FLS_KERNEL_ADAMW, -3, -1)
     fill_session(sess, cfg)
     stream = torch.cuda.current_stream()
 
@@ -444,6 +448,8 @@ def main():
     ap.add_argument("--ctas-adamw", type=int, default=0)
     ap.add_argument("--ctas-fedavg", type=int, default=0)
     ap.add_argument("--descending-adamw", action="store_true")
+    ap.add_argument("--ascending-adamw", action="store_true")
+    ap.add_argument("--no-overlap", action="store_true", help="plain launches instead of programmatic dependent launch")
     # slices of a workload, for profiler captures that must stay small (same kernels, fewer bytes)
     ap.add_argument("--n-params", type=int, default=0, help="override P (single flat unit)")
     ap.add_argument("--groups", type=int, default=0, help="override G")

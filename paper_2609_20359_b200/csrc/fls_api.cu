@@ -60,8 +60,9 @@ struct fls_plan {
   uint64_t step = 0;
   uint64_t launches = 0;
   int ctas_per_sm[FLS_KERNEL_COUNT] = {0, 0, 0};   // 0: the grid covers every tile once (no grid-stride loop)
-  int descending[FLS_KERNEL_COUNT] = {0, 0, 0};
+  int descending[FLS_KERNEL_COUNT] = {0, 1, 0};   // AdamW starts where the reduce kernel stopped: those lines are still in L2
 
+  bool overlap = true;     // programmatic dependent launch between the kernels of one call
   bool profiling = false;
   std::vector<TimedLaunch> timed;
   std::vector<cudaEvent_t> event_pool;
@@ -137,7 +138,9 @@ cudaError_t timed_launch(fls_plan* p, int kernel, cudaStream_t st, F&& launch) {
   return e;
 }
 
-int run_group(fls_plan* p, uint32_t g, double lr, uint64_t t_new, cudaStream_t st) {
+// chain: the previous operation on `st` is a kernel of this same call, so this group's first kernel may
+// overlap its tail
+int run_group(fls_plan* p, uint32_t g, double lr, uint64_t t_new, cudaStream_t st, bool chain) {
   const fls_plan_desc& d = p->desc;
   ReduceArgs ra{};
   for (uint32_t k = 0; k < p->K; ++k) ra.grad[k] = p->grads[size_t(g) * p->K + k];
@@ -158,8 +161,9 @@ int run_group(fls_plan* p, uint32_t g, double lr, uint64_t t_new, cudaStream_t s
   ra.status = p->d_status();
   ra.max_grad_norm = d.max_grad_norm;
   const bool f32 = d.grad_dtype == FLS_GRAD_F32;
+  const bool overlap = p->overlap && !p->profiling;   // event records between kernels would serialise anyway
   cudaError_t e = timed_launch(p, FLS_KERNEL_REDUCE, st,
-                               [&] { return launch_reduce(ra, f32, p->reduce_sg, st); });
+                               [&] { return launch_reduce(ra, f32, p->reduce_sg, st, overlap && chain); });
   if (e != cudaSuccess) return cuda_fail(e, "reduce kernel launch");
 
   // Scalars of the AdamW step, in double on the host, handed to the kernel as fp32.
@@ -182,7 +186,7 @@ int run_group(fls_plan* p, uint32_t g, double lr, uint64_t t_new, cudaStream_t s
   aa.step_size = float(lr / bc1);
   aa.inv_sqrt_bc2 = float(1.0 / std::sqrt(bc2));
   aa.eps = float(d.eps);
-  e = timed_launch(p, FLS_KERNEL_ADAMW, st, [&] { return launch_adamw(aa, p->grid_for(FLS_KERNEL_ADAMW), st); });
+  e = timed_launch(p, FLS_KERNEL_ADAMW, st, [&] { return launch_adamw(aa, p->grid_for(FLS_KERNEL_ADAMW), st, overlap); });
   if (e != cudaSuccess) return cuda_fail(e, "adamw kernel launch");
   return FLS_OK;
 }
@@ -374,7 +378,7 @@ int fls_sync_step(fls_plan* p, double lr, void* cuda_stream, int* fedavg_due) {
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const uint64_t t_new = p->step + 1;
   for (uint32_t g = 0; g < p->desc.groups; ++g) {
-    const int rc = run_group(p, g, lr, t_new, st);
+    const int rc = run_group(p, g, lr, t_new, st, g > 0);
     if (rc != FLS_OK) return rc;
   }
   p->step = t_new;
@@ -408,7 +412,7 @@ int fls_sync_step_host(fls_plan* p, const void* const* host_grads, double lr, vo
     if (e != cudaSuccess) return cuda_fail(e, "cudaEventRecord");
     e = cudaStreamWaitEvent(st, p->ev_copied[g], 0);
     if (e != cudaSuccess) return cuda_fail(e, "cudaStreamWaitEvent");
-    const int rc = run_group(p, g, lr, t_new, st);
+    const int rc = run_group(p, g, lr, t_new, st, false);   // an event wait precedes every group here
     if (rc != FLS_OK) return rc;
   }
   if (host_norms) {
@@ -445,7 +449,8 @@ int fls_fedavg(fls_plan* p, const uint64_t* sample_counts, void* cuda_stream) {
       fa.pbf16[g] = p->pbf16[g];
     }
     fa.write_bf16 = arr == 0 ? 1 : 0;
-    cudaError_t e = timed_launch(p, FLS_KERNEL_FEDAVG, st, [&] { return launch_fedavg(fa, p->grid_for(FLS_KERNEL_FEDAVG), st); });
+    const bool overlap = p->overlap && !p->profiling && arr > 0;
+    cudaError_t e = timed_launch(p, FLS_KERNEL_FEDAVG, st, [&] { return launch_fedavg(fa, p->grid_for(FLS_KERNEL_FEDAVG), st, overlap); });
     if (e != cudaSuccess) return cuda_fail(e, "fedavg kernel launch");
   }
   return FLS_OK;
@@ -498,6 +503,8 @@ int fls_plan_tune(fls_plan* p, uint32_t kernel, int ctas_per_sm, int descending)
   if (!p || kernel >= FLS_KERNEL_COUNT) return fail(FLS_EINVAL, "fls_plan_tune: bad argument");
   if (ctas_per_sm > 0) p->ctas_per_sm[kernel] = std::min(ctas_per_sm, 1 << 16);
   if (ctas_per_sm == -2) p->ctas_per_sm[kernel] = 0;   // back to the default: one pass, the grid covers every tile
+  if (ctas_per_sm == -3) p->overlap = false;            // plain launches: no kernel overlaps its predecessor
+  if (ctas_per_sm == -4) p->overlap = true;
   if (descending >= 0) p->descending[kernel] = descending ? 1 : 0;
   return FLS_OK;
 }

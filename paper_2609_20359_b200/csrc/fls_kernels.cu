@@ -24,7 +24,7 @@ namespace {
 
 // ------------------------------------------------------------------------------------------------
 // Global-memory accessors.  "stream": data touched once (evict-first, no L1 allocation).
-// "keep": default policy, used for the reduced gradient that the next kernel reads back.
+// "keep": the reduced gradient, written by one kernel and read back by the next.
 // ------------------------------------------------------------------------------------------------
 struct alignas(32) F8 { float v[8]; };
 
@@ -50,8 +50,9 @@ __device__ __forceinline__ F8 ld8_keep(const float* p) {
 __device__ __forceinline__ void st8_stream(float* p, const F8& r) {
   asm volatile("st.global.L1::no_allocate.L2::evict_first.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" :: "l"(p), FLS_U8(r) : "memory");
 }
+// the reduced gradient is the one stream that is read again (by the next kernel): ask L2 to evict it last
 __device__ __forceinline__ void st8_keep(float* p, const F8& r) {
-  asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" :: "l"(p), FLS_U8(r) : "memory");
+  asm volatile("st.global.L2::evict_last.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" :: "l"(p), FLS_U8(r) : "memory");
 }
 // 128-bit accesses have no L2::evict_first form; .cs is the streaming (evict-first) cache operator
 __device__ __forceinline__ uint4 ld_b128_stream(const void* p) {
@@ -78,6 +79,20 @@ __device__ __forceinline__ uint16_t to_bf16_bits(float x) {
   __nv_bfloat16 h = __float2bfloat16_rn(x);
   return *reinterpret_cast<uint16_t*>(&h);
 }
+
+// ------------------------------------------------------------------------------------------------
+// Programmatic dependent launch.  Inside one API call every kernel but the first is launched with
+// programmatic stream serialization: its CTAs may start while the previous kernel's last CTAs are still
+// running.  A kernel first issues the loads that its direct predecessor does not write, then waits
+// (dep_wait) for that predecessor to have completed and flushed, and only then touches what the
+// predecessor wrote or still reads.  A thread lets its successor go (dep_launch) only AFTER its own
+// dep_wait: "the successor has started" then implies "my predecessor has completed", so at most two
+// kernels of the chain ever overlap and the early loads can only race with the direct predecessor.  The
+// first kernel of a call is launched normally and is therefore ordered after everything the caller
+// enqueued before.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // ------------------------------------------------------------------------------------------------
 // Tile -> segment.  A segment is a run that is contiguous in both index orders.
@@ -292,6 +307,7 @@ __global__ void __launch_bounds__(THREADS, MINB) fls_reduce_kernel(const __grid_
   float sq = 0.f;
   const uint32_t tile = blockIdx.x * (THREADS / kThreads) + threadIdx.x / kThreads;
   if (tile < a.idx.n_tiles) {
+    // the segment table and the gradients are not written by any kernel of the step: read them at once
     const Slice s = slice_of(a.idx.segs + find_segment(a.idx, tile), tile, threadIdx.x % kThreads);
     if (s.vec) {
       float g[8];
@@ -299,11 +315,15 @@ __global__ void __launch_bounds__(THREADS, MINB) fls_reduce_kernel(const __grid_
       F8 o;
 #pragma unroll
       for (int e = 0; e < 8; ++e) { o.v[e] = g[e]; sq = fmaf(g[e], g[e], sq); }
+      dep_wait();                        // the previous group's AdamW kernel may still be reading the scratch
       st8_keep(a.gbar + s.a, o);
     } else if (s.n) {
+      dep_wait();
       sq = reduce_slice_scalar<F32>(a, s.j, s.a, s.n);
     }
   }
+  dep_wait();                            // partials, ticket and the norm slots belong to the predecessor until now
+  dep_launch();
   // CTA partial -> workspace; the CTA that takes the last ticket adds all partials in index order, so
   // the norm does not depend on the order in which CTAs finish.
   double total = block_sum<THREADS>(double(sq), sh);
@@ -357,18 +377,21 @@ __device__ __noinline__ void adamw_slice_scalar(const AdamArgs& a, float c, uint
 
 __global__ void __launch_bounds__(kThreads, 3) fls_adamw_kernel(const __grid_constant__ AdamArgs a) {
   const uint32_t n_tiles = a.idx.n_tiles;
-  if (blockIdx.x >= n_tiles) return;
-  const float c = __ldcg(a.coef);
+  if (blockIdx.x >= n_tiles) { dep_wait(); dep_launch(); return; }
+  float c = 0.f;
+  bool waited = false;
   Walker w;
   w.init(a.idx, a.descending ? n_tiles - 1 - blockIdx.x : blockIdx.x);
   for (uint32_t lin = blockIdx.x; lin < n_tiles; lin += gridDim.x) {
     const uint32_t tile = a.descending ? n_tiles - 1 - lin : lin;
     const Slice s = slice_of(w.seek(tile), tile, threadIdx.x);
     if (s.vec) {
-      const F8 g = ld8_keep(a.gbar + s.a);
+      // theta, m and v of this group are not touched by the reduce kernel: fetch them before waiting for it
       F8 th = ld8_stream(a.theta + s.a);
       F8 m = ld8_stream(a.m + s.a);
       F8 v = ld8_stream(a.v + s.a);
+      if (!waited) { dep_wait(); dep_launch(); c = __ldcg(a.coef); waited = true; }
+      const F8 g = ld8_keep(a.gbar + s.a);
 #pragma unroll
       for (int e = 0; e < 8; ++e) adamw_one(a, c, g.v[e], th.v[e], m.v[e], v.v[e]);
       st8_stream(a.theta + s.a, th);
@@ -376,9 +399,11 @@ __global__ void __launch_bounds__(kThreads, 3) fls_adamw_kernel(const __grid_con
       st8_stream(a.v + s.a, v);
       st_b128_stream(a.pbf16 + s.j, pack_bf16x8(th));
     } else if (s.n) {
+      if (!waited) { dep_wait(); dep_launch(); c = __ldcg(a.coef); waited = true; }
       adamw_slice_scalar(a, c, s.j, s.a, s.n);
     }
   }
+  if (!waited) { dep_wait(); dep_launch(); }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -402,6 +427,8 @@ __global__ void __launch_bounds__(kThreads, MINB) fls_fedavg_kernel(const __grid
   constexpr int B = GT ? GT : 8;
   const uint32_t G = GT ? uint32_t(GT) : a.G;
   const uint32_t n_tiles = a.idx.n_tiles;
+  dep_wait();                            // the copies being averaged were just written by the predecessor
+  dep_launch();
   if (blockIdx.x >= n_tiles) return;
   Walker w;
   w.init(a.idx, a.descending ? n_tiles - 1 - blockIdx.x : blockIdx.x);
@@ -463,43 +490,59 @@ constexpr int kFlatThreads = FLS_FLAT_THREADS, kFlatMinB = FLS_FLAT_MINB;       
 constexpr int kLevelThreads = FLS_LEVEL_THREADS, kLevelMinB = FLS_LEVEL_MINB;   // two-level orders with a static K
 constexpr int kAnyThreads = 256, kAnyMinB = 2;         // run-time K: batches of 8 loads need the registers
 
+// Launch, with programmatic stream serialization if `overlap` (see dep_wait / dep_launch above).
+template <typename Args>
+void launch_k(void (*kernel)(Args), const Args& a, unsigned grid, unsigned threads, cudaStream_t st, bool overlap) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(threads);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = overlap ? 1 : 0;
+  cudaLaunchKernelEx(&cfg, kernel, a);
+}
+
 inline int reduce_threads(const ReduceArgs& a, int sg) {
   const bool static_k = sg >= 0 && (a.K == 1 || a.K == 2 || a.K == 4 || a.K == 8);
   return !static_k ? kAnyThreads : (sg == 0 ? kFlatThreads : kLevelThreads);
 }
 
 template <bool F32, int KT, int SG>
-void launch_reduce_shape(const ReduceArgs& a, unsigned grid, cudaStream_t st) {
+void launch_reduce_shape(const ReduceArgs& a, unsigned grid, cudaStream_t st, bool ov) {
   if constexpr (KT == 0)
-    fls_reduce_kernel<F32, KT, SG, kAnyThreads, kAnyMinB><<<grid, kAnyThreads, 0, st>>>(a);
+    launch_k(fls_reduce_kernel<F32, KT, SG, kAnyThreads, kAnyMinB>, a, grid, kAnyThreads, st, ov);
   else if constexpr (SG == 0)
-    fls_reduce_kernel<F32, KT, SG, kFlatThreads, kFlatMinB><<<grid, kFlatThreads, 0, st>>>(a);
+    launch_k(fls_reduce_kernel<F32, KT, SG, kFlatThreads, kFlatMinB>, a, grid, kFlatThreads, st, ov);
   else
-    fls_reduce_kernel<F32, KT, SG, kLevelThreads, kLevelMinB><<<grid, kLevelThreads, 0, st>>>(a);
+    launch_k(fls_reduce_kernel<F32, KT, SG, kLevelThreads, kLevelMinB>, a, grid, kLevelThreads, st, ov);
 }
 
 template <bool F32, int KT>
-void launch_reduce_k(const ReduceArgs& a, int sg, unsigned grid, cudaStream_t st) {
+void launch_reduce_k(const ReduceArgs& a, int sg, unsigned grid, cudaStream_t st, bool ov) {
   // only the level structures that can occur with KT buffers are instantiated (SG divides KT)
-  if (sg == 0) { launch_reduce_shape<F32, KT, 0>(a, grid, st); return; }
-  if constexpr (KT == 0 || KT >= 2) { if (sg == 1) { launch_reduce_shape<F32, KT, 1>(a, grid, st); return; } }
-  if constexpr (KT == 0 || KT >= 4) { if (sg == 2) { launch_reduce_shape<F32, KT, 2>(a, grid, st); return; } }
-  if constexpr (KT == 0 || KT == 8) { if (sg == 4) { launch_reduce_shape<F32, KT, 4>(a, grid, st); return; } }
-  launch_reduce_shape<F32, 0, -1>(a, grid, st);
+  if (sg == 0) { launch_reduce_shape<F32, KT, 0>(a, grid, st, ov); return; }
+  if constexpr (KT == 0 || KT >= 2) { if (sg == 1) { launch_reduce_shape<F32, KT, 1>(a, grid, st, ov); return; } }
+  if constexpr (KT == 0 || KT >= 4) { if (sg == 2) { launch_reduce_shape<F32, KT, 2>(a, grid, st, ov); return; } }
+  if constexpr (KT == 0 || KT == 8) { if (sg == 4) { launch_reduce_shape<F32, KT, 4>(a, grid, st, ov); return; } }
+  launch_reduce_shape<F32, 0, -1>(a, grid, st, ov);
 }
 
 template <bool F32>
-void launch_reduce_t(const ReduceArgs& a, int sg, unsigned grid, cudaStream_t st) {
+void launch_reduce_t(const ReduceArgs& a, int sg, unsigned grid, cudaStream_t st, bool ov) {
   if (sg >= 0) {
     switch (a.K) {
-      case 1: launch_reduce_k<F32, 1>(a, sg, grid, st); return;
-      case 2: launch_reduce_k<F32, 2>(a, sg, grid, st); return;
-      case 4: launch_reduce_k<F32, 4>(a, sg, grid, st); return;
-      case 8: launch_reduce_k<F32, 8>(a, sg, grid, st); return;
+      case 1: launch_reduce_k<F32, 1>(a, sg, grid, st, ov); return;
+      case 2: launch_reduce_k<F32, 2>(a, sg, grid, st, ov); return;
+      case 4: launch_reduce_k<F32, 4>(a, sg, grid, st, ov); return;
+      case 8: launch_reduce_k<F32, 8>(a, sg, grid, st, ov); return;
       default: break;
     }
   }
-  launch_reduce_k<F32, 0>(a, sg, grid, st);
+  launch_reduce_k<F32, 0>(a, sg, grid, st, ov);
 }
 
 }  // namespace
@@ -509,27 +552,27 @@ unsigned reduce_grid(const ReduceArgs& a, int sg) {
   return (a.idx.n_tiles + tiles_per_cta - 1) / tiles_per_cta;
 }
 
-cudaError_t launch_reduce(const ReduceArgs& a, bool f32, int sg, cudaStream_t st) {
+cudaError_t launch_reduce(const ReduceArgs& a, bool f32, int sg, cudaStream_t st, bool overlap) {
   const unsigned grid = reduce_grid(a, sg);
   if (f32)
-    launch_reduce_t<true>(a, sg, grid, st);
+    launch_reduce_t<true>(a, sg, grid, st, overlap);
   else
-    launch_reduce_t<false>(a, sg, grid, st);
+    launch_reduce_t<false>(a, sg, grid, st, overlap);
   return cudaGetLastError();
 }
 
-cudaError_t launch_adamw(const AdamArgs& a, unsigned grid, cudaStream_t st) {
-  fls_adamw_kernel<<<grid, kThreads, 0, st>>>(a);
+cudaError_t launch_adamw(const AdamArgs& a, unsigned grid, cudaStream_t st, bool overlap) {
+  launch_k(fls_adamw_kernel, a, grid, kThreads, st, overlap);
   return cudaGetLastError();
 }
 
-cudaError_t launch_fedavg(const FedavgArgs& a, unsigned grid, cudaStream_t st) {
+cudaError_t launch_fedavg(const FedavgArgs& a, unsigned grid, cudaStream_t st, bool overlap) {
   switch (a.G) {
-    case 1: fls_fedavg_kernel<1, 6><<<grid, kThreads, 0, st>>>(a); break;
-    case 2: fls_fedavg_kernel<2, 5><<<grid, kThreads, 0, st>>>(a); break;
-    case 4: fls_fedavg_kernel<4, 4><<<grid, kThreads, 0, st>>>(a); break;
-    case 8: fls_fedavg_kernel<8, 2><<<grid, kThreads, 0, st>>>(a); break;
-    default: fls_fedavg_kernel<0, 2><<<grid, kThreads, 0, st>>>(a); break;
+    case 1: launch_k(fls_fedavg_kernel<1, 6>, a, grid, kThreads, st, overlap); break;
+    case 2: launch_k(fls_fedavg_kernel<2, 5>, a, grid, kThreads, st, overlap); break;
+    case 4: launch_k(fls_fedavg_kernel<4, 4>, a, grid, kThreads, st, overlap); break;
+    case 8: launch_k(fls_fedavg_kernel<8, 2>, a, grid, kThreads, st, overlap); break;
+    default: launch_k(fls_fedavg_kernel<0, 2>, a, grid, kThreads, st, overlap); break;
   }
   return cudaGetLastError();
 }

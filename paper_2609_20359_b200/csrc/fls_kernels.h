@@ -58,8 +58,10 @@ struct FedavgArgs {
 // sg: level structure of the reduction (see reduce_elems): 0, 1, 2, 4 or -1 for the generic form.
 // The reduce kernel has one launch shape; reduce_grid() is its grid (= number of norm partials it writes).
 unsigned reduce_grid(const ReduceArgs& a, int sg);
-cudaError_t launch_reduce(const ReduceArgs& a, bool f32, int sg, cudaStream_t st);
-cudaError_t launch_adamw(const AdamArgs& a, unsigned grid, cudaStream_t st);
-cudaError_t launch_fedavg(const FedavgArgs& a, unsigned grid, cudaStream_t st);
+// overlap: launch with programmatic stream serialization, so that the kernel's first CTAs may start during
+// the tail of the kernel launched just before it on the same stream (which must be one of these three).
+cudaError_t launch_reduce(const ReduceArgs& a, bool f32, int sg, cudaStream_t st, bool overlap);
+cudaError_t launch_adamw(const AdamArgs& a, unsigned grid, cudaStream_t st, bool overlap);
+cudaError_t launch_fedavg(const FedavgArgs& a, unsigned grid, cudaStream_t st, bool overlap);
 
 }  // namespace fls
