@@ -219,9 +219,11 @@ def run_ours(args, cfg):
 
     G, P = cfg["groups"], cfg["n_params"]
     counts = [sy.sample_count(cfg["seed"], g) for g in range(G)] if cfg["weights"] == "counts" else None
+    fused = not args.unfused and G <= fls.FLS_MAX_FUSED_GROUPS
     sess = Session(P, cfg["unit_numel"], G, cfg["shard_dim"], cfg["replicate_dim"], cfg["sync_period"], cfg["grad_dtype"], 8,
                    args.opt_state, cfg["lr"], cfg["beta1"], cfg["beta2"], cfg["eps"], cfg["weight_decay"], cfg["max_grad_norm"],
-                   device=f"cuda:{local}")
+                   device=f"cuda:{local}", fused=fused)
+    H = cfg["sync_period"]
     for kern, val in (("reduce", args.ctas_reduce), ("adamw", args.ctas_adamw), ("fedavg", args.ctas_fedavg)):
         if val:
             fls.fls_plan_tune(sess.plan, {"reduce": 0, "adamw": 1, "fedavg": 2}[kern], val, -1)
@@ -237,7 +239,11 @@ def run_ours(args, cfg):
     n_fedavg = [0]
 
     def one_step():
-        if sess.step(stream=stream):
+        # on the steps where aggregation is due, the fused call does the step and FedAvg in one go
+        if fused and (sess.t + 1) % H == 0:
+            sess.step_fedavg(counts, stream=stream)
+            n_fedavg[0] += 1
+        elif sess.step(stream=stream):
             sess.fedavg(counts, stream=stream)
             n_fedavg[0] += 1
 
@@ -310,9 +316,10 @@ def run_ours(args, cfg):
         eg = 4 if cfg["grad_dtype"] == "f32" else 2
         # FedAvg runs one launch per averaged array: parameters move 10 B per group-element (4 read, 4 + 2
         # written), m and v 8 B each; the figure is the mean over the launches of one call
-        per_launch = {"reduce": N * (sess.K * eg + 4), "adamw": N * 30, "fedavg": N * G * (26 / 3 if args.opt_state else 10)}
+        per_launch = {"reduce": N * (sess.K * eg + 4), "adamw": N * 30, "fedavg": N * G * (26 / 3 if args.opt_state else 10),
+                      "adamw_fedavg": N * G * 30}
         kernels = {}
-        for i, name in enumerate(("reduce", "adamw", "fedavg")):
+        for i, name in enumerate(("reduce", "adamw", "fedavg", "adamw_fedavg")):
             if kn[i]:
                 avg_ms = kms[i] / kn[i]
                 kernels[name] = {"launches": kn[i], "avg_ms": avg_ms, "bytes_per_launch": per_launch[name],
@@ -321,7 +328,8 @@ def run_ours(args, cfg):
         dom = max(kernels, key=lambda n: kernels[n]["share"])
         rep = fls.fls_comm_report(sess.plan)
         # bytes the timed steps had to move: every sync step, plus the FedAvg calls that fell inside the region
-        step_bytes = rep["hbm_bytes_sync_step"] + rep["hbm_bytes_fedavg"] * fedavg_calls / args.steps
+        # (the fused aggregation moves no bytes of its own: an aggregation step costs what a plain step costs)
+        step_bytes = rep["hbm_bytes_sync_step"] + (0 if fused else rep["hbm_bytes_fedavg"] * fedavg_calls / args.steps)
         ms_step = ms_total / args.steps
         line = {
             "metric": METRIC, "value": world * G * P * args.steps / (ms_total / 1e3), "unit": UNIT, "n_gpus": world,
@@ -329,7 +337,7 @@ def run_ours(args, cfg):
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": cfg["name"], "n_params": P, "groups": G, "shard_dim": cfg["shard_dim"],
                        "replicate_dim": cfg["replicate_dim"], "sync_period": cfg["sync_period"], "grad_dtype": cfg["grad_dtype"],
-                       "fedavg_opt_state": bool(args.opt_state), "fedavg_calls_in_timed_region": fedavg_calls, "l2": "working set exceeds L2, no flush needed",
+                       "fedavg_opt_state": bool(args.opt_state), "fused_aggregation": bool(fused), "fedavg_calls_in_timed_region": fedavg_calls, "l2": "working set exceeds L2, no flush needed",
                        "parallelism": "replicas only" if world > 1 else "1 gpu"},
             "hbm_gbs": step_bytes / ms_step / 1e6, "hbm_frac_of_measured_peak": step_bytes / ms_step / 1e6 / peak,
             "hbm_frac_of_8tbs": step_bytes / ms_step / 1e6 / 8000.0,
@@ -441,6 +449,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default=DEFAULT_CONFIG, choices=[c["name"] for c in sy.CONFIGS])
     ap.add_argument("--opt-state", action="store_true", help="FedAvg also averages m and v")
+    ap.add_argument("--unfused", action="store_true", help="aggregation steps call fls_sync_step + fls_fedavg instead of fls_sync_step_fedavg")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-max-gb", type=float, default=48.0, help="skip the end-to-end pass if its pinned host staging would exceed this")
     ap.add_argument("--no-cpu-baseline", action="store_true")

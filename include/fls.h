@@ -42,12 +42,13 @@ typedef struct fls_plan fls_plan; /* opaque, created by fls_plan_create, freed b
 
 enum { FLS_OK = 0, FLS_EINVAL = 1, FLS_EALIGN = 2, FLS_EPTR = 3, FLS_ESIZE = 4, FLS_ECUDA = 5, FLS_ESTATE = 6 };
 enum { FLS_GRAD_BF16 = 0, FLS_GRAD_F32 = 1 };
-enum { FLS_AVG_PARAMS = 1, FLS_AVG_OPT_STATE = 2 }; /* fedavg_what bit mask */
-enum { FLS_KERNEL_REDUCE = 0, FLS_KERNEL_ADAMW = 1, FLS_KERNEL_FEDAVG = 2, FLS_KERNEL_COUNT = 3 };
+enum { FLS_AVG_PARAMS = 1, FLS_AVG_OPT_STATE = 2, FLS_AVG_FUSED = 4 }; /* fedavg_what bit mask */
+enum { FLS_KERNEL_REDUCE = 0, FLS_KERNEL_ADAMW = 1, FLS_KERNEL_FEDAVG = 2, FLS_KERNEL_ADAMW_FEDAVG = 3, FLS_KERNEL_COUNT = 4 };
 enum { FLS_STATUS_NONFINITE_NORM = 1 };             /* sticky bits of the device status word */
 
 #define FLS_MAX_GROUPS 64        /* G <= 64 */
 #define FLS_MAX_GRAD_BUFFERS 64  /* K = shard_dim * replicate_dim <= 64 */
+#define FLS_MAX_FUSED_GROUPS 16  /* fls_sync_step_fedavg fuses the aggregation for G up to this */
 #define FLS_BUFFER_ALIGN 32      /* every device buffer must start on a 32-byte boundary */
 #define FLS_NOALLOC_MAX_ELEMS 536870912ull /* 2^29: largest n_elems fls_reduce_norm_noalloc accepts */
 
@@ -65,7 +66,9 @@ typedef struct {
   uint32_t align_elems;       /* Q >= 1: every unit's shard length is rounded up to a multiple of Q.
                                  Q = 1 pads a unit to a multiple of S exactly; multiples of 8 keep every
                                  shard on the vector path (otherwise element-wise loads are used)      */
-  uint32_t fedavg_what;       /* FLS_AVG_PARAMS, optionally | FLS_AVG_OPT_STATE (m and v averaged too)  */
+  uint32_t fedavg_what;       /* FLS_AVG_PARAMS, optionally | FLS_AVG_OPT_STATE (m and v averaged too),
+                                 optionally | FLS_AVG_FUSED (workspace holds one reduced gradient per group
+                                 so that fls_sync_step_fedavg can fuse the aggregation into the step)      */
   uint32_t reserved;          /* must be 0                                                              */
   double lr, beta1, beta2, eps, weight_decay;
   double max_grad_norm;       /* <= 0 disables clipping (the norm is still computed)                    */
@@ -157,6 +160,15 @@ int fls_sync_step_host(fls_plan* plan, const void* const* host_grads, double lr,
  * Errors: FLS_EINVAL if all counts are zero, FLS_ESTATE, FLS_ECUDA. */
 int fls_fedavg(fls_plan* plan, const uint64_t* sample_counts, void* cuda_stream);
 
+/* One local step of all groups immediately followed by FedAvg, i.e. exactly fls_sync_step then fls_fedavg
+ * (same results bit for bit), for the steps on which aggregation is due ("after the local update every A
+ * training steps").  With FLS_AVG_FUSED in the plan and G <= FLS_MAX_FUSED_GROUPS the aggregation is fused
+ * into the optimizer kernel: after the G reductions one kernel applies AdamW to every group's element,
+ * averages the G results in registers and writes the average to all G copies, which saves FedAvg's own
+ * read and write of the parameters (10*G bytes per parameter).  Otherwise it runs the two calls one after the
+ * other.  sample_counts: host, G entries, NULL = equal weights.  Errors: as fls_sync_step and fls_fedavg. */
+int fls_sync_step_fedavg(fls_plan* plan, double lr, const uint64_t* sample_counts, void* cuda_stream);
+
 /* Device pointers (inside the workspace) to G floats each: the gradient norm and the clip coefficient of
  * the last step, valid once that step has completed on its stream.  Either output may be NULL. */
 int fls_get_norms(const fls_plan* plan, const float** dev_norms, const float** dev_coefs);
@@ -188,7 +200,8 @@ int fls_plan_tune(fls_plan* plan, uint32_t kernel, int ctas_per_sm, int descendi
 
 /* Per-kernel timing with CUDA events recorded on the caller's stream around every launch.
  * fls_set_profiling(plan, 1) turns it on; fls_get_kernel_ms waits for the recorded events, adds their
- * durations into ms[FLS_KERNEL_COUNT] / launches[FLS_KERNEL_COUNT] (host) and clears the record. */
+ * durations into ms[FLS_KERNEL_COUNT] / launches[FLS_KERNEL_COUNT] (host, indexed by FLS_KERNEL_*) and clears
+ * the record. */
 int fls_set_profiling(fls_plan* plan, int enabled);
 int fls_get_kernel_ms(fls_plan* plan, double* ms, uint64_t* launches);
 

@@ -12,16 +12,18 @@ LIB_PATH = os.environ.get("FLS_LIBRARY") or os.path.join(_PKG, "libfls.so")
 
 FLS_OK, FLS_EINVAL, FLS_EALIGN, FLS_EPTR, FLS_ESIZE, FLS_ECUDA, FLS_ESTATE = range(7)
 FLS_GRAD_BF16, FLS_GRAD_F32 = 0, 1
-FLS_AVG_PARAMS, FLS_AVG_OPT_STATE = 1, 2
-FLS_KERNEL_REDUCE, FLS_KERNEL_ADAMW, FLS_KERNEL_FEDAVG, FLS_KERNEL_COUNT = 0, 1, 2, 3
+FLS_AVG_PARAMS, FLS_AVG_OPT_STATE, FLS_AVG_FUSED = 1, 2, 4
+FLS_KERNEL_REDUCE, FLS_KERNEL_ADAMW, FLS_KERNEL_FEDAVG, FLS_KERNEL_ADAMW_FEDAVG, FLS_KERNEL_COUNT = 0, 1, 2, 3, 4
 FLS_STATUS_NONFINITE_NORM = 1
 FLS_MAX_GROUPS = 64
 FLS_MAX_GRAD_BUFFERS = 64
+FLS_MAX_FUSED_GROUPS = 16
 FLS_BUFFER_ALIGN = 32
 FLS_NOALLOC_MAX_ELEMS = 1 << 29
 
 EXPORTS = [
     "fls_plan_create", "fls_plan_query", "fls_plan_bind", "fls_sync_step", "fls_sync_step_host", "fls_fedavg",
+    "fls_sync_step_fedavg",
     "fls_get_norms", "fls_get_reduced_grad", "fls_get_status", "fls_get_step", "fls_set_step", "fls_comm_report",
     "fls_plan_tune", "fls_set_profiling", "fls_get_kernel_ms", "fls_get_launch_count", "fls_plan_destroy",
     "fls_last_error", "fls_reduce_norm_noalloc",
@@ -80,6 +82,7 @@ def _load() -> C.CDLL:
     lib.fls_sync_step.argtypes = [P, C.c_double, P, C.POINTER(C.c_int)]
     lib.fls_sync_step_host.argtypes = [P, C.POINTER(C.c_void_p), C.c_double, P, C.POINTER(C.c_float), C.POINTER(C.c_int)]
     lib.fls_fedavg.argtypes = [P, C.POINTER(C.c_uint64), P]
+    lib.fls_sync_step_fedavg.argtypes = [P, C.c_double, C.POINTER(C.c_uint64), P]
     lib.fls_get_norms.argtypes = [P, C.POINTER(P), C.POINTER(P)]
     lib.fls_get_reduced_grad.argtypes = [P, C.POINTER(P)]
     lib.fls_get_status.argtypes = [P, C.POINTER(P)]
@@ -183,6 +186,12 @@ def fls_sync_step_host(plan: int, host_grads: Sequence, lr: float = math.nan, st
 def fls_fedavg(plan: int, sample_counts: Optional[Sequence[int]] = None, stream=None) -> None:
     arr = (C.c_uint64 * len(sample_counts))(*sample_counts) if sample_counts is not None else None
     _check(lib.fls_fedavg(plan, arr, _stream_handle(stream)))
+
+
+def fls_sync_step_fedavg(plan: int, lr: float = math.nan, sample_counts: Optional[Sequence[int]] = None, stream=None) -> None:
+    """fls_sync_step followed by fls_fedavg, fused into the optimizer kernel when the plan has FLS_AVG_FUSED."""
+    arr = (C.c_uint64 * len(sample_counts))(*sample_counts) if sample_counts is not None else None
+    _check(lib.fls_sync_step_fedavg(plan, lr, arr, _stream_handle(stream)))
 
 
 def fls_get_norms(plan: int):

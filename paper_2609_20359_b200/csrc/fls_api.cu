@@ -59,8 +59,8 @@ struct fls_plan {
 
   uint64_t step = 0;
   uint64_t launches = 0;
-  int ctas_per_sm[FLS_KERNEL_COUNT] = {0, 0, 0};   // 0: the grid covers every tile once (no grid-stride loop)
-  int descending[FLS_KERNEL_COUNT] = {0, 1, 0};   // AdamW starts where the reduce kernel stopped: those lines are still in L2
+  int ctas_per_sm[FLS_KERNEL_COUNT] = {0, 0, 0, 0};   // 0: the grid covers every tile once (no grid-stride loop)
+  int descending[FLS_KERNEL_COUNT] = {0, 1, 0, 1};   // AdamW starts where the reduce kernel stopped: those lines are still in L2
 
   bool overlap = true;     // programmatic dependent launch between the kernels of one call
   bool profiling = false;
@@ -72,7 +72,8 @@ struct fls_plan {
   std::vector<cudaEvent_t> ev_copied;
 
   const Segment* d_segs() const { return reinterpret_cast<const Segment*>(ws + kWsSegments); }
-  float* d_gbar() const { return reinterpret_cast<float*>(ws + lay.ws_scratch_offset); }
+  float* d_gbar(uint32_t slot = 0) const { return reinterpret_cast<float*>(ws + lay.ws_scratch_offset + lay.scratch_stride * slot); }
+  uint32_t last_slot = 0;   // where the last processed group's reduced gradient lives
   float* d_norms() const { return reinterpret_cast<float*>(ws + kWsNorms); }
   float* d_coefs() const { return reinterpret_cast<float*>(ws + kWsCoefs); }
   double* d_normsq() const { return reinterpret_cast<double*>(ws + kWsNormSq); }
@@ -140,11 +141,33 @@ cudaError_t timed_launch(fls_plan* p, int kernel, cudaStream_t st, F&& launch) {
 
 // chain: the previous operation on `st` is a kernel of this same call, so this group's first kernel may
 // overlap its tail
-int run_group(fls_plan* p, uint32_t g, double lr, uint64_t t_new, cudaStream_t st, bool chain) {
+struct AdamScalars { float decay, beta1, omb1, beta2, omb2, step_size, inv_sqrt_bc2, eps; };
+
+// Scalars of the AdamW step, in double on the host, handed to the kernels as fp32.
+AdamScalars adam_scalars(const fls_plan_desc& d, double lr, uint64_t t_new) {
+  const double bc1 = 1.0 - std::pow(d.beta1, double(t_new));
+  const double bc2 = 1.0 - std::pow(d.beta2, double(t_new));
+  AdamScalars s;
+  s.decay = float(1.0 - lr * d.weight_decay);
+  s.beta1 = float(d.beta1);
+  s.omb1 = float(1.0 - d.beta1);
+  s.beta2 = float(d.beta2);
+  s.omb2 = float(1.0 - d.beta2);
+  s.step_size = float(lr / bc1);
+  s.inv_sqrt_bc2 = float(1.0 / std::sqrt(bc2));
+  s.eps = float(d.eps);
+  return s;
+}
+
+// slot: which reduced-gradient buffer of the workspace receives the mean gradient; with_adamw = false stops
+// after the reduction (the fused aggregation applies AdamW to all groups afterwards)
+int run_group(fls_plan* p, uint32_t g, double lr, uint64_t t_new, cudaStream_t st, bool chain, uint32_t slot = 0,
+              bool with_adamw = true) {
   const fls_plan_desc& d = p->desc;
   ReduceArgs ra{};
   for (uint32_t k = 0; k < p->K; ++k) ra.grad[k] = p->grads[size_t(g) * p->K + k];
-  ra.gbar = p->d_gbar();
+  ra.gbar = p->d_gbar(slot);
+  p->last_slot = slot;
   ra.idx = p->seg_index();
   ra.K = p->K;
   ra.S = d.shard_dim;
@@ -165,12 +188,11 @@ int run_group(fls_plan* p, uint32_t g, double lr, uint64_t t_new, cudaStream_t s
   cudaError_t e = timed_launch(p, FLS_KERNEL_REDUCE, st,
                                [&] { return launch_reduce(ra, f32, p->reduce_sg, st, overlap && chain); });
   if (e != cudaSuccess) return cuda_fail(e, "reduce kernel launch");
+  if (!with_adamw) return FLS_OK;
 
-  // Scalars of the AdamW step, in double on the host, handed to the kernel as fp32.
-  const double bc1 = 1.0 - std::pow(d.beta1, double(t_new));
-  const double bc2 = 1.0 - std::pow(d.beta2, double(t_new));
+  const AdamScalars sc = adam_scalars(d, lr, t_new);
   AdamArgs aa{};
-  aa.gbar = p->d_gbar();
+  aa.gbar = p->d_gbar(slot);
   aa.theta = p->master[g];
   aa.m = p->m[g];
   aa.v = p->v[g];
@@ -178,14 +200,8 @@ int run_group(fls_plan* p, uint32_t g, double lr, uint64_t t_new, cudaStream_t s
   aa.idx = ra.idx;
   aa.descending = p->descending[FLS_KERNEL_ADAMW];
   aa.coef = p->d_coefs() + g;
-  aa.decay = float(1.0 - lr * d.weight_decay);
-  aa.beta1 = float(d.beta1);
-  aa.omb1 = float(1.0 - d.beta1);
-  aa.beta2 = float(d.beta2);
-  aa.omb2 = float(1.0 - d.beta2);
-  aa.step_size = float(lr / bc1);
-  aa.inv_sqrt_bc2 = float(1.0 / std::sqrt(bc2));
-  aa.eps = float(d.eps);
+  aa.decay = sc.decay; aa.beta1 = sc.beta1; aa.omb1 = sc.omb1; aa.beta2 = sc.beta2; aa.omb2 = sc.omb2;
+  aa.step_size = sc.step_size; aa.inv_sqrt_bc2 = sc.inv_sqrt_bc2; aa.eps = sc.eps;
   e = timed_launch(p, FLS_KERNEL_ADAMW, st, [&] { return launch_adamw(aa, p->grid_for(FLS_KERNEL_ADAMW), st, overlap); });
   if (e != cudaSuccess) return cuda_fail(e, "adamw kernel launch");
   return FLS_OK;
@@ -217,8 +233,8 @@ int fls_plan_create(const fls_plan_desc* desc, fls_plan** out) {
   if (K > FLS_MAX_GRAD_BUFFERS)
     return fail(FLS_EINVAL, "shard_dim*replicate_dim = %llu exceeds %d", (unsigned long long)K, FLS_MAX_GRAD_BUFFERS);
   if (d.grad_dtype != FLS_GRAD_BF16 && d.grad_dtype != FLS_GRAD_F32) return fail(FLS_EINVAL, "unknown grad_dtype %u", d.grad_dtype);
-  if (!(d.fedavg_what & FLS_AVG_PARAMS) || (d.fedavg_what & ~uint32_t(FLS_AVG_PARAMS | FLS_AVG_OPT_STATE)))
-    return fail(FLS_EINVAL, "fedavg_what must be FLS_AVG_PARAMS, optionally | FLS_AVG_OPT_STATE");
+  if (!(d.fedavg_what & FLS_AVG_PARAMS) || (d.fedavg_what & ~uint32_t(FLS_AVG_PARAMS | FLS_AVG_OPT_STATE | FLS_AVG_FUSED)))
+    return fail(FLS_EINVAL, "fedavg_what must be FLS_AVG_PARAMS, optionally | FLS_AVG_OPT_STATE | FLS_AVG_FUSED");
   if (d.reserved != 0) return fail(FLS_EINVAL, "reserved must be 0");
   if (!(d.beta1 >= 0.0 && d.beta1 < 1.0) || !(d.beta2 >= 0.0 && d.beta2 < 1.0)) return fail(FLS_EINVAL, "betas must lie in [0, 1)");
   if (!(d.eps > 0.0) || !std::isfinite(d.eps)) return fail(FLS_EINVAL, "eps must be positive");
@@ -244,7 +260,8 @@ int fls_plan_create(const fls_plan_desc* desc, fls_plan** out) {
   p->units = units;
   p->desc.unit_numel = nullptr;   // the caller's table is not kept; p->units is the copy
   p->desc.n_units = uint32_t(units.size());
-  const std::string msg = build_layout(units, d.shard_dim, d.align_elems, &p->lay);
+  const bool fused = (d.fedavg_what & FLS_AVG_FUSED) && d.groups <= FLS_MAX_FUSED_GROUPS;
+  const std::string msg = build_layout(units, d.shard_dim, d.align_elems, fused ? d.groups : 1, &p->lay);
   if (!msg.empty()) {
     delete p;
     return fail(FLS_EINVAL, "layout: %s", msg.c_str());
@@ -456,6 +473,49 @@ int fls_fedavg(fls_plan* p, const uint64_t* sample_counts, void* cuda_stream) {
   return FLS_OK;
 }
 
+int fls_sync_step_fedavg(fls_plan* p, double lr, const uint64_t* sample_counts, void* cuda_stream) {
+  if (!p) return fail(FLS_EINVAL, "fls_sync_step_fedavg: null plan");
+  if (!p->bound) return fail(FLS_ESTATE, "fls_sync_step_fedavg: plan has no buffers bound");
+  const uint32_t G = p->desc.groups;
+  if (p->lay.scratch_slots < G) {   // not planned for fusion: the two calls in sequence give the same result
+    const int rc = fls_sync_step(p, lr, cuda_stream, nullptr);
+    return rc != FLS_OK ? rc : fls_fedavg(p, sample_counts, cuda_stream);
+  }
+  if (!step_preamble(p, &lr)) return fail(FLS_EINVAL, "fls_sync_step_fedavg: lr must be finite and >= 0");
+  long double total = 0;
+  for (uint32_t g = 0; g < G; ++g) total += sample_counts ? (long double)sample_counts[g] : 1.0L;
+  if (!(total > 0)) return fail(FLS_EINVAL, "fls_sync_step_fedavg: all sample counts are zero");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const uint64_t t_new = p->step + 1;
+  for (uint32_t g = 0; g < G; ++g) {
+    const int rc = run_group(p, g, lr, t_new, st, g > 0, g, false);
+    if (rc != FLS_OK) return rc;
+  }
+  const AdamScalars sc = adam_scalars(p->desc, lr, t_new);
+  FusedArgs fa{};
+  for (uint32_t g = 0; g < G; ++g) {
+    fa.gbar[g] = p->d_gbar(g);
+    fa.theta[g] = p->master[g];
+    fa.m[g] = p->m[g];
+    fa.v[g] = p->v[g];
+    fa.pbf16[g] = p->pbf16[g];
+    fa.w[g] = float((sample_counts ? double(sample_counts[g]) : 1.0) / double(total));
+  }
+  fa.coefs = p->d_coefs();
+  fa.idx = p->seg_index();
+  fa.G = G;
+  fa.avg_opt_state = (p->desc.fedavg_what & FLS_AVG_OPT_STATE) ? 1 : 0;
+  fa.descending = p->descending[FLS_KERNEL_ADAMW_FEDAVG];
+  fa.decay = sc.decay; fa.beta1 = sc.beta1; fa.omb1 = sc.omb1; fa.beta2 = sc.beta2; fa.omb2 = sc.omb2;
+  fa.step_size = sc.step_size; fa.inv_sqrt_bc2 = sc.inv_sqrt_bc2; fa.eps = sc.eps;
+  const bool overlap = p->overlap && !p->profiling;
+  cudaError_t e = timed_launch(p, FLS_KERNEL_ADAMW_FEDAVG, st,
+                               [&] { return launch_adamw_fedavg(fa, p->grid_for(FLS_KERNEL_ADAMW_FEDAVG), st, overlap); });
+  if (e != cudaSuccess) return cuda_fail(e, "fused adamw+fedavg kernel launch");
+  p->step = t_new;
+  return FLS_OK;
+}
+
 int fls_get_norms(const fls_plan* p, const float** dev_norms, const float** dev_coefs) {
   if (!p) return fail(FLS_EINVAL, "fls_get_norms: null plan");
   if (!p->bound) return fail(FLS_ESTATE, "fls_get_norms: plan has no buffers bound");
@@ -467,7 +527,7 @@ int fls_get_norms(const fls_plan* p, const float** dev_norms, const float** dev_
 int fls_get_reduced_grad(const fls_plan* p, const float** dev_gbar) {
   if (!p || !dev_gbar) return fail(FLS_EINVAL, "fls_get_reduced_grad: null argument");
   if (!p->bound) return fail(FLS_ESTATE, "fls_get_reduced_grad: plan has no buffers bound");
-  *dev_gbar = p->d_gbar();
+  *dev_gbar = p->d_gbar(p->last_slot);
   return FLS_OK;
 }
 

@@ -37,10 +37,13 @@ struct Layout {
   uint64_t n_params = 0, n_padded = 0, shard_numel = 0, n_tiles = 0;
   uint64_t ws_partials_offset = 0, ws_scratch_offset = 0, workspace_bytes = 0;
   bool vector_path = true;
+  uint32_t scratch_slots = 1;              // reduced-gradient buffers in the workspace, each 4*n_padded bytes (256-byte aligned)
+  uint64_t scratch_stride = 0;             // bytes between two of them
 };
 
 // Host planner: fills `out` from the unit table; returns an error message or "" on success.
-std::string build_layout(const std::vector<uint64_t>& unit_numel, uint32_t S, uint32_t Q, Layout* out);
+// scratch_slots: how many reduced-gradient buffers the workspace holds (1, or G for the fused aggregation).
+std::string build_layout(const std::vector<uint64_t>& unit_numel, uint32_t S, uint32_t Q, uint32_t scratch_slots, Layout* out);
 
 // Sets the calling thread's message returned by fls_last_error() (defined beside it).
 void set_last_error(const char* msg);

@@ -476,6 +476,86 @@ __global__ void __launch_bounds__(kThreads, MINB) fls_fedavg_kernel(const __grid
 }
 
 // ------------------------------------------------------------------------------------------------
+// K2+K3 fused for aggregation steps: AdamW on every group's element, then the weighted average of the G
+// results, written to all G copies.  The arithmetic and its order are those of fls_adamw_kernel followed by
+// fls_fedavg_kernel (each group's new theta is rounded to fp32 before it enters the fma chain), so the
+// results are bit-identical to the two-kernel sequence; what is saved is FedAvg's own pass over the
+// parameters.  m and v stay per group unless the plan averages the optimizer state.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void adamw_one_f(const FusedArgs& a, float c, float gbar, float& th, float& m, float& v) {
+  const float g = c * gbar;
+  th = th * a.decay;
+  m = fmaf(a.beta1, m, a.omb1 * g);
+  v = fmaf(a.beta2, v, a.omb2 * (g * g));
+  const float denom = fmaf(sqrtf(v), a.inv_sqrt_bc2, a.eps);
+  th = fmaf(-a.step_size, __fdiv_rn(m, denom), th);
+}
+
+__device__ __noinline__ void fused_slice_scalar(const FusedArgs& a, uint64_t j, uint64_t addr, uint32_t n) {
+  for (uint32_t e = 0; e < n; ++e) {
+    float ath = 0.f, am = 0.f, av = 0.f;
+    for (uint32_t g = 0; g < a.G; ++g) {
+      float th = a.theta[g][addr + e], m = a.m[g][addr + e], v = a.v[g][addr + e];
+      adamw_one_f(a, __ldcg(a.coefs + g), a.gbar[g][addr + e], th, m, v);
+      ath = fmaf(a.w[g], th, ath);
+      if (a.avg_opt_state) { am = fmaf(a.w[g], m, am); av = fmaf(a.w[g], v, av); }
+      else { a.m[g][addr + e] = m; a.v[g][addr + e] = v; }
+    }
+    const uint16_t b = to_bf16_bits(ath);
+    for (uint32_t g = 0; g < a.G; ++g) {
+      a.theta[g][addr + e] = ath;
+      a.pbf16[g][j + e] = b;
+      if (a.avg_opt_state) { a.m[g][addr + e] = am; a.v[g][addr + e] = av; }
+    }
+  }
+}
+
+template <bool OPT>
+__global__ void __launch_bounds__(kThreads, 3) fls_adamw_fedavg_kernel(const __grid_constant__ FusedArgs a) {
+  const uint32_t n_tiles = a.idx.n_tiles;
+  if (blockIdx.x >= n_tiles) { dep_wait(); dep_launch(); return; }
+  bool waited = false;
+  Walker w;
+  w.init(a.idx, a.descending ? n_tiles - 1 - blockIdx.x : blockIdx.x);
+  for (uint32_t lin = blockIdx.x; lin < n_tiles; lin += gridDim.x) {
+    const uint32_t tile = a.descending ? n_tiles - 1 - lin : lin;
+    const Slice s = slice_of(w.seek(tile), tile, threadIdx.x);
+    if (s.vec) {
+      F8 ath, am, av;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) ath.v[e] = am.v[e] = av.v[e] = 0.f;
+#pragma unroll 1
+      for (uint32_t g = 0; g < a.G; ++g) {
+        // theta, m, v are not written by the reduce kernels: group 0's can be fetched before the wait
+        F8 th = ld8_stream(a.theta[g] + s.a);
+        F8 m = ld8_stream(a.m[g] + s.a);
+        F8 v = ld8_stream(a.v[g] + s.a);
+        if (!waited) { dep_wait(); dep_launch(); waited = true; }
+        const F8 gb = ld8_keep(a.gbar[g] + s.a);
+        const float c = __ldcg(a.coefs + g), wg = a.w[g];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          adamw_one_f(a, c, gb.v[e], th.v[e], m.v[e], v.v[e]);
+          ath.v[e] = fmaf(wg, th.v[e], ath.v[e]);
+          if (OPT) { am.v[e] = fmaf(wg, m.v[e], am.v[e]); av.v[e] = fmaf(wg, v.v[e], av.v[e]); }
+        }
+        if (!OPT) { st8_stream(a.m[g] + s.a, m); st8_stream(a.v[g] + s.a, v); }
+      }
+      const uint4 p = pack_bf16x8(ath);
+      for (uint32_t g = 0; g < a.G; ++g) {
+        st8_stream(a.theta[g] + s.a, ath);
+        st_b128_stream(a.pbf16[g] + s.j, p);
+        if (OPT) { st8_stream(a.m[g] + s.a, am); st8_stream(a.v[g] + s.a, av); }
+      }
+    } else if (s.n) {
+      if (!waited) { dep_wait(); dep_launch(); waited = true; }
+      fused_slice_scalar(a, s.j, s.a, s.n);
+    }
+  }
+  if (!waited) { dep_wait(); dep_launch(); }
+}
+
+// ------------------------------------------------------------------------------------------------
 // Launchers.
 // ------------------------------------------------------------------------------------------------
 #ifndef FLS_FLAT_THREADS
@@ -574,6 +654,14 @@ cudaError_t launch_fedavg(const FedavgArgs& a, unsigned grid, cudaStream_t st, b
     case 8: launch_k(fls_fedavg_kernel<8, 2>, a, grid, kThreads, st, overlap); break;
     default: launch_k(fls_fedavg_kernel<0, 2>, a, grid, kThreads, st, overlap); break;
   }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_adamw_fedavg(const FusedArgs& a, unsigned grid, cudaStream_t st, bool overlap) {
+  if (a.avg_opt_state)
+    launch_k(fls_adamw_fedavg_kernel<true>, a, grid, kThreads, st, overlap);
+  else
+    launch_k(fls_adamw_fedavg_kernel<false>, a, grid, kThreads, st, overlap);
   return cudaGetLastError();
 }
 

@@ -55,6 +55,22 @@ struct FedavgArgs {
   int descending;
 };
 
+// AdamW of all G groups + FedAvg of the results in one pass (G <= FLS_MAX_FUSED_GROUPS).
+struct FusedArgs {
+  const float* gbar[FLS_MAX_FUSED_GROUPS];  // device, one reduced gradient per group
+  float* theta[FLS_MAX_FUSED_GROUPS];
+  float* m[FLS_MAX_FUSED_GROUPS];
+  float* v[FLS_MAX_FUSED_GROUPS];
+  uint16_t* pbf16[FLS_MAX_FUSED_GROUPS];
+  float w[FLS_MAX_FUSED_GROUPS];
+  const float* coefs;                      // device, G clip coefficients written by the reduce kernels
+  SegIndex idx;
+  uint32_t G;
+  int avg_opt_state;                       // m and v are averaged too
+  int descending;
+  float decay, beta1, omb1, beta2, omb2, step_size, inv_sqrt_bc2, eps;
+};
+
 // sg: level structure of the reduction (see reduce_elems): 0, 1, 2, 4 or -1 for the generic form.
 // The reduce kernel has one launch shape; reduce_grid() is its grid (= number of norm partials it writes).
 unsigned reduce_grid(const ReduceArgs& a, int sg);
@@ -63,5 +79,6 @@ unsigned reduce_grid(const ReduceArgs& a, int sg);
 cudaError_t launch_reduce(const ReduceArgs& a, bool f32, int sg, cudaStream_t st, bool overlap);
 cudaError_t launch_adamw(const AdamArgs& a, unsigned grid, cudaStream_t st, bool overlap);
 cudaError_t launch_fedavg(const FedavgArgs& a, unsigned grid, cudaStream_t st, bool overlap);
+cudaError_t launch_adamw_fedavg(const FusedArgs& a, unsigned grid, cudaStream_t st, bool overlap);
 
 }  // namespace fls

@@ -9,7 +9,7 @@
 
 namespace fls {
 
-std::string build_layout(const std::vector<uint64_t>& unit_numel, uint32_t S, uint32_t Q, Layout* out) {
+std::string build_layout(const std::vector<uint64_t>& unit_numel, uint32_t S, uint32_t Q, uint32_t scratch_slots, Layout* out) {
   if (unit_numel.empty()) return "empty unit table";
   if (S == 0 || Q == 0) return "shard_dim and align_elems must be >= 1";
   Layout& L = *out;
@@ -70,7 +70,9 @@ std::string build_layout(const std::vector<uint64_t>& unit_numel, uint32_t S, ui
   if (L.n_tiles >= (1ull << 32)) return "plan too large";
   L.ws_partials_offset = (kWsSegments + seg_bytes + 255) / 256 * 256;
   L.ws_scratch_offset = (L.ws_partials_offset + 8 * L.n_tiles + 255) / 256 * 256;   // at most one partial per tile
-  L.workspace_bytes = L.ws_scratch_offset + 4ull * L.n_padded;
+  L.scratch_slots = scratch_slots ? scratch_slots : 1;
+  L.scratch_stride = (4ull * L.n_padded + 255) / 256 * 256;
+  L.workspace_bytes = L.ws_scratch_offset + L.scratch_stride * L.scratch_slots;
   return "";
 }
 

@@ -65,7 +65,7 @@ class Case:
 
     def __init__(self, units, G, S, R_rep=1, H=1, Q=8, grad_dtype="bf16", opt_state=False, seed=1234,
                  grad_sigma=1e-3, master_sigma=0.02, per_buffer_scale=False, hp: orc.Hyper = None, guard=4096,
-                 same_grads_all_groups=False):
+                 same_grads_all_groups=False, fused=False):
         from paper_2609_20359_b200.session import Session
         self.units, self.G, self.S, self.R_rep, self.H, self.Q = list(units), G, S, R_rep, H, Q
         self.K = S * R_rep
@@ -79,7 +79,8 @@ class Case:
         z = np.zeros(self.P, np.float32)
         self.states = [orc.GroupState(th0.copy(), z.copy(), z.copy(), orc.f32_to_bf16_bits(th0)) for _ in range(G)]
         self.sess = Session(self.P, units, G, S, R_rep, H, grad_dtype, Q, opt_state, self.hp.lr, self.hp.beta1,
-                            self.hp.beta2, self.hp.eps, self.hp.weight_decay, self.hp.max_grad_norm, guard_bytes=guard)
+                            self.hp.beta2, self.hp.eps, self.hp.weight_decay, self.hp.max_grad_norm, guard_bytes=guard, fused=fused)
+        self.fused = fused
         lay = self.sess.layout
         assert lay["n_padded"] == self.L.n_padded and lay["shard_numel"] == self.L.shard_numel
         for g in range(G):
@@ -124,11 +125,16 @@ class Case:
             nrm, c, _ = orc.sync_step_group(self.states[g], grads[g], self.S, self.R_rep, self.t, self.hp, lr)
             row.append((nrm, c))
         self.norms.append(row)
-        due = self.sess.step(float("nan") if lr is None else lr)
-        assert due == (self.t % self.H == 0)
-        if due and fedavg:
+        due = self.t % self.H == 0
+        if due and fedavg and self.fused:
+            # the single call that does the step and the aggregation
             orc.fedavg(self.states, counts, self.opt_state)
-            self.sess.fedavg(counts)
+            self.sess.step_fedavg(counts, float("nan") if lr is None else lr)
+        else:
+            assert self.sess.step(float("nan") if lr is None else lr) == due
+            if due and fedavg:
+                orc.fedavg(self.states, counts, self.opt_state)
+                self.sess.fedavg(counts)
         torch.cuda.synchronize()
         return row
 

@@ -189,6 +189,30 @@ def test_fedavg(fls, G, opt_state, counts):
     c.close()
 
 
+@pytest.mark.parametrize("units,G,S,R_rep,Q,dtype,opt_state", [
+    ([50000, 1234, 4096], 2, 2, 2, 8, "bf16", False),
+    ([50000, 1234, 4096], 4, 4, 1, 8, "bf16", True),
+    ([70001], 3, 2, 1, 1, "f32", True),                 # unaligned tail, G = 3
+    ([30000, 517], 16, 2, 1, 8, "bf16", False),         # the largest fused G
+    ([30000, 517], 17, 2, 1, 8, "bf16", True),          # above it: the call falls back to the two-kernel sequence
+    ([17], 2, 4, 1, 1, "bf16", False),
+])
+def test_fused_step_fedavg_matches_oracle_and_unfused(fls, units, G, S, R_rep, Q, dtype, opt_state):
+    """fls_sync_step_fedavg = fls_sync_step + fls_fedavg: against the oracle, and bit for bit against the
+    two separate calls on the same inputs (H = 2: steps 1 and 3 are plain, 2 and 4 aggregate)."""
+    counts = [sy.sample_count(21, g) for g in range(G)]
+    outs = []
+    for fused in (True, False):
+        c = Case(units, G, S, R_rep, H=2, Q=Q, grad_dtype=dtype, opt_state=opt_state, hp=orc.Hyper(max_grad_norm=0.05), fused=fused)
+        for _ in range(4):
+            c.step(counts)
+            c.compare()
+        assert c.sess.t == 4
+        outs.append([x.clone() for x in c.sess.master + c.sess.m + c.sess.v + c.sess.param_bf16])
+        c.close()
+    assert all(torch.equal(x, y) for x, y in zip(*outs))
+
+
 def test_fedavg_g1_is_bit_exact_identity_and_idempotent(fls):
     c = Case([5000], 1, 2, 1, H=1, Q=8, opt_state=True)
     c.step(fedavg=False)
