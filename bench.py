@@ -88,9 +88,10 @@ class ClockSampler:
 
     def wait_for(self, event):
         """Waits for a CUDA event, sampling the clocks every millisecond or so meanwhile."""
+        self.sample()                      # at least one reading, taken while the region is (still) running
         while not event.query():
-            self.sample()
             time.sleep(0.001)
+            self.sample()
 
     def stop(self) -> dict:
         if self._nvml is None:
