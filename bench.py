@@ -203,8 +203,6 @@ def fill_session(sess, cfg):
 def run_ours(args, cfg):
     import torch.distributed as dist
     from paper_2609_20359_b200 import build
-    from paper_2609_20359_b200 import _binding as fls
-    from paper_2609_20359_b200.session import Session
 
     rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -217,6 +215,9 @@ def run_ours(args, cfg):
         build.build()
     if world > 1:
         dist.barrier()
+    # only now: importing the binding loads libfls.so, which rank 0 may just have built
+    from paper_2609_20359_b200 import _binding as fls
+    from paper_2609_20359_b200.session import Session
 
     G, P = cfg["groups"], cfg["n_params"]
     counts = [sy.sample_count(cfg["seed"], g) for g in range(G)] if cfg["weights"] == "counts" else None

@@ -42,6 +42,7 @@ typedef struct fls_plan fls_plan; /* opaque, created by fls_plan_create, freed b
 
 enum { FLS_OK = 0, FLS_EINVAL = 1, FLS_EALIGN = 2, FLS_EPTR = 3, FLS_ESIZE = 4, FLS_ECUDA = 5, FLS_ESTATE = 6 };
 enum { FLS_GRAD_BF16 = 0, FLS_GRAD_F32 = 1 };
+enum { FLS_WIRE_F32 = 0, FLS_WIRE_BF16 = 1 };          /* reduce_wire */
 enum { FLS_AVG_PARAMS = 1, FLS_AVG_OPT_STATE = 2, FLS_AVG_FUSED = 4 }; /* fedavg_what bit mask */
 enum { FLS_KERNEL_REDUCE = 0, FLS_KERNEL_ADAMW = 1, FLS_KERNEL_FEDAVG = 2, FLS_KERNEL_ADAMW_FEDAVG = 3, FLS_KERNEL_COUNT = 4 };
 enum { FLS_STATUS_NONFINITE_NORM = 1 };             /* sticky bits of the device status word */
@@ -69,7 +70,11 @@ typedef struct {
   uint32_t fedavg_what;       /* FLS_AVG_PARAMS, optionally | FLS_AVG_OPT_STATE (m and v averaged too),
                                  optionally | FLS_AVG_FUSED (workspace holds one reduced gradient per group
                                  so that fls_sync_step_fedavg can fuse the aggregation into the step)      */
-  uint32_t reserved;          /* must be 0                                                              */
+  uint32_t reduce_wire;       /* FLS_WIRE_F32 (default): fp32 partial sums.  FLS_WIRE_BF16 (bf16 gradients only):
+                                 every partial sum of both reduction levels and the final mean are rounded
+                                 to bf16, emulating collectives that run in bf16 -- the setting in which the
+                                 paper observes that the FSDP and HSDP orders give different numbers.  Slower
+                                 (generic kernel); meant for numerical experiments                         */
   double lr, beta1, beta2, eps, weight_decay;
   double max_grad_norm;       /* <= 0 disables clipping (the norm is still computed)                    */
 } fls_plan_desc;
@@ -121,7 +126,7 @@ typedef struct {
 /* Layout planner + validation (flat-buffer layout: padding to the shard multiple, per-unit offsets).
  * Host only: touches no GPU.  Errors: FLS_EINVAL for a null argument, G, S, R_rep, H or Q = 0, G or K
  * above the maxima, sum(unit_numel) != n_params, a zero-length unit, beta outside [0,1), eps <= 0, lr < 0,
- * an unknown dtype or fedavg_what without FLS_AVG_PARAMS.  On error *out is NULL. */
+ * an unknown dtype, FLS_WIRE_BF16 with fp32 gradients, or fedavg_what without FLS_AVG_PARAMS.  On error *out is NULL. */
 int fls_plan_create(const fls_plan_desc* desc, fls_plan** out);
 
 /* Copies the layout summary into *out (host). */

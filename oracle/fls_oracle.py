@@ -141,7 +141,12 @@ def unpack_sharded(L: Layout, buf: np.ndarray) -> np.ndarray:
 
 
 # --------------------------------------------------------------------------- one local step
-def reduce_mean(grads: Sequence[np.ndarray], S: int, R_rep: int = 1) -> np.ndarray:
+def round_to_bf16(x: np.ndarray) -> np.ndarray:
+    """Values rounded to bf16 (via the stored-fp32 rounding above), returned as float64."""
+    return bf16_bits_to_f64(f32_to_bf16_bits(np.asarray(x, dtype=np.float64).astype(np.float32)))
+
+
+def reduce_mean(grads: Sequence[np.ndarray], S: int, R_rep: int = 1, wire_bf16: bool = False) -> np.ndarray:
     """Mean gradient of one group, stored as fp32.
 
     grads: K = R_rep*S float64 arrays (exact input values), buffer rho*S+sigma.
@@ -150,9 +155,22 @@ def reduce_mean(grads: Sequence[np.ndarray], S: int, R_rep: int = 1) -> np.ndarr
     the all-reduce across the R_rep replicas (over rho) -- shard level first,
     replicate level second.  Reading: the reduction is a mean (sum, then one
     division by K after the last level), kept in fp32 afterwards.
+
+    wire_bf16: emulation of collectives that run in bf16 (the paper's runs are in
+    bfloat16 and it attributes HSDP's different result to the order of floating-point
+    operations): every partial sum and the final mean are rounded to bf16, so the
+    two orders give different numbers.  Both levels start from zero, as on the GPU.
     """
     K = len(grads)
     assert K == S * R_rep and K >= 1
+    if wire_bf16:
+        outer = np.zeros_like(np.asarray(grads[0], dtype=np.float64))
+        for rho in range(R_rep):
+            inner = np.zeros_like(outer)
+            for sigma in range(S):
+                inner = round_to_bf16((inner + np.asarray(grads[rho * S + sigma], dtype=np.float64)).astype(np.float32))
+            outer = round_to_bf16((outer + inner).astype(np.float32))
+        return round_to_bf16((outer / K).astype(np.float32)).astype(np.float32)
     outer = None
     for rho in range(R_rep):
         inner = None
@@ -219,6 +237,7 @@ class Hyper:
     eps: float = 1e-8
     weight_decay: float = 0.1
     max_grad_norm: float = 1.0
+    wire_bf16: bool = False        # bf16 emulation of the two reduction levels (see reduce_mean)
 
 
 def sync_step_group(st: GroupState, grads: Sequence[np.ndarray], S: int, R_rep: int, t_new: int,
@@ -226,7 +245,7 @@ def sync_step_group(st: GroupState, grads: Sequence[np.ndarray], S: int, R_rep: 
     """One local step of one group: reduce -> norm -> clip -> AdamW.  Returns
     (norm, coef, gbar).  Each group "proceeds independently of the others"
     (Section FL+FSDP)."""
-    gbar = reduce_mean(grads, S, R_rep)
+    gbar = reduce_mean(grads, S, R_rep, hp.wire_bf16)
     nrm = grad_norm(gbar)
     c = clip_coef(nrm, hp.max_grad_norm)
     st.theta, st.m, st.v, st.param_bf16 = adamw(

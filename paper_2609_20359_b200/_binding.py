@@ -12,6 +12,7 @@ LIB_PATH = os.environ.get("FLS_LIBRARY") or os.path.join(_PKG, "libfls.so")
 
 FLS_OK, FLS_EINVAL, FLS_EALIGN, FLS_EPTR, FLS_ESIZE, FLS_ECUDA, FLS_ESTATE = range(7)
 FLS_GRAD_BF16, FLS_GRAD_F32 = 0, 1
+FLS_WIRE_F32, FLS_WIRE_BF16 = 0, 1
 FLS_AVG_PARAMS, FLS_AVG_OPT_STATE, FLS_AVG_FUSED = 1, 2, 4
 FLS_KERNEL_REDUCE, FLS_KERNEL_ADAMW, FLS_KERNEL_FEDAVG, FLS_KERNEL_ADAMW_FEDAVG, FLS_KERNEL_COUNT = 0, 1, 2, 3, 4
 FLS_STATUS_NONFINITE_NORM = 1
@@ -40,7 +41,7 @@ class fls_plan_desc(C.Structure):
     _fields_ = [("n_params", C.c_uint64), ("n_units", C.c_uint32), ("unit_numel", C.POINTER(C.c_uint64)),
                 ("groups", C.c_uint32), ("shard_dim", C.c_uint32), ("replicate_dim", C.c_uint32),
                 ("sync_period", C.c_uint32), ("grad_dtype", C.c_uint32), ("align_elems", C.c_uint32),
-                ("fedavg_what", C.c_uint32), ("reserved", C.c_uint32),
+                ("fedavg_what", C.c_uint32), ("reduce_wire", C.c_uint32),
                 ("lr", C.c_double), ("beta1", C.c_double), ("beta2", C.c_double), ("eps", C.c_double),
                 ("weight_decay", C.c_double), ("max_grad_norm", C.c_double)]
 
@@ -130,7 +131,8 @@ def _stream_handle(stream) -> Optional[int]:
 def fls_plan_create(n_params: int, unit_numel: Optional[Sequence[int]] = None, groups: int = 1, shard_dim: int = 1,
                     replicate_dim: int = 1, sync_period: int = 1, grad_dtype: int = FLS_GRAD_BF16, align_elems: int = 8,
                     fedavg_what: int = FLS_AVG_PARAMS, lr: float = 3e-4, beta1: float = 0.9, beta2: float = 0.95,
-                    eps: float = 1e-8, weight_decay: float = 0.1, max_grad_norm: float = 1.0) -> int:
+                    eps: float = 1e-8, weight_decay: float = 0.1, max_grad_norm: float = 1.0,
+                    reduce_wire: int = FLS_WIRE_F32) -> int:
     """Returns the opaque plan handle."""
     d = fls_plan_desc()
     d.n_params = n_params
@@ -138,7 +140,7 @@ def fls_plan_create(n_params: int, unit_numel: Optional[Sequence[int]] = None, g
         arr = (C.c_uint64 * len(unit_numel))(*unit_numel)
         d.n_units, d.unit_numel = len(unit_numel), arr
     d.groups, d.shard_dim, d.replicate_dim, d.sync_period = groups, shard_dim, replicate_dim, sync_period
-    d.grad_dtype, d.align_elems, d.fedavg_what = grad_dtype, align_elems, fedavg_what
+    d.grad_dtype, d.align_elems, d.fedavg_what, d.reduce_wire = grad_dtype, align_elems, fedavg_what, reduce_wire
     d.lr, d.beta1, d.beta2, d.eps, d.weight_decay, d.max_grad_norm = lr, beta1, beta2, eps, weight_decay, max_grad_norm
     out = C.c_void_p()
     _check(lib.fls_plan_create(C.byref(d), C.byref(out)))

@@ -170,7 +170,6 @@ int run_group(fls_plan* p, uint32_t g, double lr, uint64_t t_new, cudaStream_t s
   p->last_slot = slot;
   ra.idx = p->seg_index();
   ra.K = p->K;
-  ra.S = d.shard_dim;
   ra.k_float = float(p->K);
   ra.inv_k = 1.0f / float(p->K);
   ra.k_is_pow2 = (p->K & (p->K - 1)) == 0 ? 1u : 0u;
@@ -235,7 +234,9 @@ int fls_plan_create(const fls_plan_desc* desc, fls_plan** out) {
   if (d.grad_dtype != FLS_GRAD_BF16 && d.grad_dtype != FLS_GRAD_F32) return fail(FLS_EINVAL, "unknown grad_dtype %u", d.grad_dtype);
   if (!(d.fedavg_what & FLS_AVG_PARAMS) || (d.fedavg_what & ~uint32_t(FLS_AVG_PARAMS | FLS_AVG_OPT_STATE | FLS_AVG_FUSED)))
     return fail(FLS_EINVAL, "fedavg_what must be FLS_AVG_PARAMS, optionally | FLS_AVG_OPT_STATE | FLS_AVG_FUSED");
-  if (d.reserved != 0) return fail(FLS_EINVAL, "reserved must be 0");
+  if (d.reduce_wire != FLS_WIRE_F32 && d.reduce_wire != FLS_WIRE_BF16) return fail(FLS_EINVAL, "unknown reduce_wire %u", d.reduce_wire);
+  if (d.reduce_wire == FLS_WIRE_BF16 && d.grad_dtype != FLS_GRAD_BF16)
+    return fail(FLS_EINVAL, "FLS_WIRE_BF16 needs bf16 gradients");
   if (!(d.beta1 >= 0.0 && d.beta1 < 1.0) || !(d.beta2 >= 0.0 && d.beta2 < 1.0)) return fail(FLS_EINVAL, "betas must lie in [0, 1)");
   if (!(d.eps > 0.0) || !std::isfinite(d.eps)) return fail(FLS_EINVAL, "eps must be positive");
   if (!(d.lr >= 0.0) || !std::isfinite(d.lr)) return fail(FLS_EINVAL, "lr must be finite and >= 0");
@@ -280,6 +281,7 @@ int fls_plan_create(const fls_plan_desc* desc, fls_plan** out) {
   } else {
     p->reduce_sg = -1;
   }
+  if (d.reduce_wire == FLS_WIRE_BF16) p->reduce_sg = -2;   // generic kernel, bf16 rounding after every sum
   *out = p;
   return FLS_OK;
 }

@@ -211,6 +211,9 @@ __device__ __forceinline__ void unpack(const Raw<1, true>& x, float (&f)[1]) { f
 //             fold_mask says that batch i closes a group.
 //   SG = 1, 2, 4 : S == SG, a batch holds whole groups of SG buffers.
 //   SG = -1 : any other shape; bit k of end_mask says that buffer k closes a group.
+//   SG = -2 : as -1, with every partial sum and the final mean rounded to bf16 (the bf16-wire emulation).
+__device__ __forceinline__ float round_bf16(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
+
 template <int N, bool F32, int KT, int SG>
 __device__ __forceinline__ void reduce_elems(const ReduceArgs& a, uint64_t j, float (&mean)[N]) {
   constexpr int B = KT ? KT : 8;            // buffers per batch
@@ -263,10 +266,10 @@ __device__ __forceinline__ void reduce_elems(const ReduceArgs& a, uint64_t j, fl
           float x[N];
           unpack(raw[b], x);
 #pragma unroll
-          for (int e = 0; e < N; ++e) inner[e] += x[e];
+          for (int e = 0; e < N; ++e) inner[e] = (SG == -2) ? round_bf16(inner[e] + x[e]) : inner[e] + x[e];
           if ((a.end_mask >> k) & 1ull) {
 #pragma unroll
-            for (int e = 0; e < N; ++e) { outer[e] += inner[e]; inner[e] = 0.f; }
+            for (int e = 0; e < N; ++e) { outer[e] = (SG == -2) ? round_bf16(outer[e] + inner[e]) : outer[e] + inner[e]; inner[e] = 0.f; }
           }
         }
       }
@@ -280,16 +283,20 @@ __device__ __forceinline__ void reduce_elems(const ReduceArgs& a, uint64_t j, fl
 #pragma unroll
     for (int e = 0; e < N; ++e) mean[e] = __fdiv_rn(outer[e], a.k_float);
   }
+  if constexpr (SG == -2) {
+#pragma unroll
+    for (int e = 0; e < N; ++e) mean[e] = round_bf16(mean[e]);
+  }
 }
 
 // element-wise path of one thread's slice (unaligned runs and ragged tails); kept out of line so that
 // it does not cost the vector path registers
-template <bool F32>
+template <bool F32, bool WIRE>
 __device__ __noinline__ float reduce_slice_scalar(const ReduceArgs& a, uint64_t j, uint64_t addr, uint32_t n) {
   float sq = 0.f;
   for (uint32_t e = 0; e < n; ++e) {
     float g[1];
-    reduce_elems<1, F32, 0, -1>(a, j + e, g);
+    reduce_elems<1, F32, 0, WIRE ? -2 : -1>(a, j + e, g);
     a.gbar[addr + e] = g[0];
     sq = fmaf(g[0], g[0], sq);
   }
@@ -319,7 +326,7 @@ __global__ void __launch_bounds__(THREADS, MINB) fls_reduce_kernel(const __grid_
       st8_keep(a.gbar + s.a, o);
     } else if (s.n) {
       dep_wait();
-      sq = reduce_slice_scalar<F32>(a, s.j, s.a, s.n);
+      sq = reduce_slice_scalar<F32, SG == -2>(a, s.j, s.a, s.n);
     }
   }
   dep_wait();                            // partials, ticket and the norm slots belong to the predecessor until now
@@ -608,6 +615,7 @@ void launch_reduce_k(const ReduceArgs& a, int sg, unsigned grid, cudaStream_t st
   if constexpr (KT == 0 || KT >= 2) { if (sg == 1) { launch_reduce_shape<F32, KT, 1>(a, grid, st, ov); return; } }
   if constexpr (KT == 0 || KT >= 4) { if (sg == 2) { launch_reduce_shape<F32, KT, 2>(a, grid, st, ov); return; } }
   if constexpr (KT == 0 || KT == 8) { if (sg == 4) { launch_reduce_shape<F32, KT, 4>(a, grid, st, ov); return; } }
+  if constexpr (KT == 0 && !F32) { if (sg == -2) { launch_reduce_shape<F32, 0, -2>(a, grid, st, ov); return; } }
   launch_reduce_shape<F32, 0, -1>(a, grid, st, ov);
 }
 

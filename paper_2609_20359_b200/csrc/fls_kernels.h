@@ -21,7 +21,7 @@ struct ReduceArgs {
   const void* grad[FLS_MAX_GRAD_BUFFERS];  // device, K buffers of this group, index rho*S + sigma
   float* gbar;                             // device, reduced gradient (shard order)
   SegIndex idx;
-  uint32_t K, S;
+  uint32_t K;
   float k_float, inv_k;                    // K and 1/K as float: the mean is scaled by 1/K once
   uint32_t k_is_pow2;                      // 1/K exact: multiply; otherwise divide
   uint32_t fold_mask;                      // bit i set: the i-th batch of 8 buffers closes a sharding group
@@ -71,7 +71,8 @@ struct FusedArgs {
   float decay, beta1, omb1, beta2, omb2, step_size, inv_sqrt_bc2, eps;
 };
 
-// sg: level structure of the reduction (see reduce_elems): 0, 1, 2, 4 or -1 for the generic form.
+// sg: level structure of the reduction (see reduce_elems): 0, 1, 2, 4 or -1 for the generic form;
+// -2: the generic form with every partial sum and the mean rounded to bf16 (bf16 gradients only).
 // The reduce kernel has one launch shape; reduce_grid() is its grid (= number of norm partials it writes).
 unsigned reduce_grid(const ReduceArgs& a, int sg);
 // overlap: launch with programmatic stream serialization, so that the kernel's first CTAs may start during

@@ -20,7 +20,7 @@ class Session:
                  replicate_dim: int = 1, sync_period: int = 1, grad_dtype: str = "bf16", align_elems: int = 8,
                  opt_state: bool = False, lr: float = 3e-4, beta1: float = 0.9, beta2: float = 0.95, eps: float = 1e-8,
                  weight_decay: float = 0.1, max_grad_norm: float = 1.0, device: str = "cuda:0", guard_bytes: int = 0,
-                 alloc_grads: bool = True, fused: bool = False):
+                 alloc_grads: bool = True, fused: bool = False, wire_bf16: bool = False):
         if not torch.cuda.is_available():
             raise RuntimeError("libfls needs a CUDA device; there is no CPU path")
         self.device = torch.device(device)
@@ -34,7 +34,7 @@ class Session:
             n_params, unit_numel, groups, shard_dim, replicate_dim, sync_period,
             fls.FLS_GRAD_F32 if grad_dtype == "f32" else fls.FLS_GRAD_BF16, align_elems,
             fls.FLS_AVG_PARAMS | (fls.FLS_AVG_OPT_STATE if opt_state else 0) | (fls.FLS_AVG_FUSED if fused else 0),
-            lr, beta1, beta2, eps, weight_decay, max_grad_norm)
+            lr, beta1, beta2, eps, weight_decay, max_grad_norm, fls.FLS_WIRE_BF16 if wire_bf16 else fls.FLS_WIRE_F32)
         self.layout = fls.fls_plan_query(self.plan)
         N = self.layout["n_padded"]
         self.n_padded, self.n_params = N, n_params

@@ -79,7 +79,8 @@ class Case:
         z = np.zeros(self.P, np.float32)
         self.states = [orc.GroupState(th0.copy(), z.copy(), z.copy(), orc.f32_to_bf16_bits(th0)) for _ in range(G)]
         self.sess = Session(self.P, units, G, S, R_rep, H, grad_dtype, Q, opt_state, self.hp.lr, self.hp.beta1,
-                            self.hp.beta2, self.hp.eps, self.hp.weight_decay, self.hp.max_grad_norm, guard_bytes=guard, fused=fused)
+                            self.hp.beta2, self.hp.eps, self.hp.weight_decay, self.hp.max_grad_norm, guard_bytes=guard, fused=fused,
+                            wire_bf16=self.hp.wire_bf16)
         self.fused = fused
         lay = self.sess.layout
         assert lay["n_padded"] == self.L.n_padded and lay["shard_numel"] == self.L.shard_numel

@@ -122,6 +122,37 @@ def test_reduced_gradient_matches_oracle_exactly_for_bf16(fls):
     c.close()
 
 
+@pytest.mark.parametrize("units,G,S,R_rep,Q", [([40000, 30011], 2, 8, 1, 8), ([40000, 30011], 2, 4, 2, 8), ([70001], 1, 3, 2, 1), ([17], 2, 2, 2, 1)])
+def test_bf16_wire_emulation(fls, units, G, S, R_rep, Q):
+    """Partial sums and the mean rounded to bf16: the reduced gradient is bit-identical to the oracle's (every
+    operation is an fp32 add or divide followed by a bf16 rounding on both sides), the step follows to tolerance."""
+    hp = orc.Hyper(max_grad_norm=0.05, wire_bf16=True)
+    c = Case(units, G, S, R_rep, H=2, Q=Q, hp=hp, per_buffer_scale=True)
+    for t in range(1, 3):
+        grads = c.load_grads(t)
+        want = orc.pack_sharded(c.L, orc.reduce_mean(grads[G - 1], S, R_rep, wire_bf16=True))
+        c.step()
+        assert np.array_equal(c.sess.reduced_grad().cpu().numpy(), want)
+        c.compare()
+    c.close()
+
+
+def test_bf16_wire_orders_differ_on_the_gpu_too(fls):
+    """Same 8 buffers reduced flat (8 x 1) and two-level (4 x 2): with fp32 partial sums the two orders agree
+    on all but a handful of elements (where a tiny addend loses bits), with bf16 partial sums they differ widely."""
+    res = {}
+    for wire in (False, True):
+        for S, R_rep in ((8, 1), (4, 2)):
+            c = Case([65536], 1, S, R_rep, H=10, Q=8, hp=orc.Hyper(max_grad_norm=0.0, wire_bf16=wire))
+            c.load_grads(1)
+            c.sess.step()
+            torch.cuda.synchronize()
+            res[(wire, S)] = c.sess.reduced_grad().clone()
+            c.close()
+    assert (res[(False, 8)] != res[(False, 4)]).float().mean().item() < 1e-3
+    assert 0.02 < (res[(True, 8)] != res[(True, 4)]).float().mean().item() < 0.9
+
+
 def test_two_level_order_differs_from_flat_where_fp32_rounds(fls):
     """fp32 gradients spanning many binades: the shard-then-replicate order and the flat order round
     differently; each matches the oracle run in the same order (to fp32 rounding of the sum)."""

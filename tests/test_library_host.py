@@ -65,7 +65,8 @@ def test_single_unit_default_table(fls):
                                 dict(groups=65), dict(shard_dim=16, replicate_dim=8), dict(beta1=1.0), dict(beta2=-0.1),
                                 dict(eps=0.0), dict(lr=-1.0), dict(lr=float("nan")), dict(grad_dtype=7), dict(fedavg_what=2),
                                 dict(fedavg_what=0), dict(unit_numel=[10, 5]), dict(unit_numel=[16, 0]),
-                                dict(max_grad_norm=float("nan")), dict(weight_decay=-0.5)])
+                                dict(max_grad_norm=float("nan")), dict(weight_decay=-0.5),
+                                dict(reduce_wire=2), dict(reduce_wire=1, grad_dtype=1), dict(fedavg_what=8)])
 def test_plan_create_rejects_bad_arguments(fls, kw):
     args = dict(n_params=16, unit_numel=None, groups=2, shard_dim=2)
     args.update(kw)

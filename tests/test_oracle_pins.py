@@ -144,6 +144,43 @@ def test_reduce_mean_brute_force_p17(S, R_rep):
     assert got.dtype == np.float32
 
 
+@pytest.mark.parametrize("S,R_rep", [(4, 1), (2, 2), (4, 2), (3, 1), (1, 3)])
+def test_reduce_mean_bf16_wire_brute_force_p17(S, R_rep):
+    """bf16-wire mode: every partial sum and the mean rounded to bf16, exact rationals + an independent
+    nearest-even rounding (the one of the worked-case generator)."""
+    from tests.golden.make_worked_cases import _round_to_bits
+    r32 = lambda q: _round_to_bits(q, 23, -126)
+    rb = lambda q: _round_to_bits(r32(q), 7, -126)       # an fp32 add/divide, then the bf16 store
+    rng = np.random.default_rng(300 + S * 10 + R_rep)
+    K = S * R_rep
+    bits = [rng_bf16_bits(rng, 17, 1.0) for _ in range(K)]
+    got = orc.reduce_mean([orc.bf16_bits_to_f64(b) for b in bits], S, R_rep, wire_bf16=True)
+    for j in range(17):
+        outer = Fraction(0)
+        for rho in range(R_rep):
+            inner = Fraction(0)
+            for sigma in range(S):
+                inner = rb(inner + frac_of_bf16(bits[rho * S + sigma][j]))
+            outer = rb(outer + inner)
+        assert Fraction(float(got[j])) == rb(outer / K), j
+    # the values are bf16-representable, and close to (but in general not equal to) the fp32-accumulated mean
+    assert np.array_equal(orc.round_to_bf16(got), got.astype(np.float64))
+    plain = orc.reduce_mean([orc.bf16_bits_to_f64(b) for b in bits], S, R_rep)
+    assert np.allclose(got, plain, rtol=2 ** -6, atol=0.03)       # a bf16 ulp of the O(1) partial sums
+
+
+def test_bf16_wire_makes_the_two_orders_differ():
+    """The paper's remark: FSDP's single reduction and HSDP's two-tier reduction are the same mathematically
+    but not numerically in bf16.  In fp32 accumulation the two orders agree on these inputs; with bf16
+    partial sums they do not."""
+    rng = np.random.default_rng(77)
+    g = [orc.bf16_bits_to_f64(rng_bf16_bits(rng, 4000, 1e-3)) for _ in range(8)]
+    assert np.array_equal(orc.reduce_mean(g, 8, 1), orc.reduce_mean(g, 4, 2))
+    a, b = orc.reduce_mean(g, 8, 1, wire_bf16=True), orc.reduce_mean(g, 4, 2, wire_bf16=True)
+    assert 0.02 < np.mean(a != b) < 0.9
+    assert np.allclose(a, b, rtol=2 ** -5, atol=1e-5)
+
+
 def test_reduce_special_cases():
     rng = np.random.default_rng(7)
     g = [orc.bf16_bits_to_f64(rng_bf16_bits(rng, 1000)) for _ in range(8)]
