@@ -234,7 +234,7 @@ def run_ours(args, cfg):
     if args.ascending_adamw:
         fls.fls_plan_tune(sess.plan, fls.FLS_KERNEL_ADAMW, 0, 0)
     if args.no_overlap:
-        fls.fls_plan_tune(sess.plan, fls.FLS_KERNEL_ADAMW, -3, -1)
+        fls.fls_plan_set_overlap(sess.plan, False)
     fill_session(sess, cfg)
     stream = torch.cuda.current_stream()
 

@@ -198,10 +198,14 @@ int fls_comm_report(const fls_plan* plan, const double* bw_bytes_per_s, fls_comm
  * FedAvg kernels ctas_per_sm > 0 switches to a persistent grid of ctas_per_sm * (number of SMs) CTAs that
  * stride over the tiles; -2 restores the default; 0 and -1 keep the current value.  descending: 1 / 0 sets
  * the direction in which those two kernels walk the tiles, negative keeps it.  The reduce kernel has one
- * launch shape and ignores both.  Two more values of ctas_per_sm act on the whole plan: -3 launches every
- * kernel plainly, -4 (the default) lets each kernel of a call but the first start during the tail of the one
- * before it (programmatic dependent launch; the results are identical). */
+ * launch shape and ignores both. */
 int fls_plan_tune(fls_plan* plan, uint32_t kernel, int ctas_per_sm, int descending);
+
+/* enabled != 0 (the default): inside one call every kernel but the first is launched so that its first CTAs may
+ * start during the tail of the kernel before it (programmatic dependent launch); they fetch what that kernel does
+ * not write and wait for its completion before touching anything else, so the results are identical.  0: plain
+ * launches, each kernel starts when the previous one has finished. */
+int fls_plan_set_overlap(fls_plan* plan, int enabled);
 
 /* Per-kernel timing with CUDA events recorded on the caller's stream around every launch.
  * fls_set_profiling(plan, 1) turns it on; fls_get_kernel_ms waits for the recorded events, adds their

@@ -565,9 +565,13 @@ int fls_plan_tune(fls_plan* p, uint32_t kernel, int ctas_per_sm, int descending)
   if (!p || kernel >= FLS_KERNEL_COUNT) return fail(FLS_EINVAL, "fls_plan_tune: bad argument");
   if (ctas_per_sm > 0) p->ctas_per_sm[kernel] = std::min(ctas_per_sm, 1 << 16);
   if (ctas_per_sm == -2) p->ctas_per_sm[kernel] = 0;   // back to the default: one pass, the grid covers every tile
-  if (ctas_per_sm == -3) p->overlap = false;            // plain launches: no kernel overlaps its predecessor
-  if (ctas_per_sm == -4) p->overlap = true;
   if (descending >= 0) p->descending[kernel] = descending ? 1 : 0;
+  return FLS_OK;
+}
+
+int fls_plan_set_overlap(fls_plan* p, int enabled) {
+  if (!p) return fail(FLS_EINVAL, "fls_plan_set_overlap: null plan");
+  p->overlap = enabled != 0;
   return FLS_OK;
 }
 

@@ -92,15 +92,16 @@ def test_large_segment_table_uses_global_lookup(fls):
     c.close()
 
 
-@pytest.mark.parametrize("ctas,descending", [(1, 0), (3, 1), (0, 1), (64, 0)])
-def test_tuned_launch_shapes_give_identical_results(fls, ctas, descending):
-    """Persistent / descending launch shapes of the AdamW and FedAvg kernels change scheduling only: the
-    results are bit-identical to the default one-pass shape."""
+@pytest.mark.parametrize("ctas,descending,overlap", [(1, 0, True), (3, 1, False), (0, 1, False), (64, 0, True)])
+def test_tuned_launch_shapes_give_identical_results(fls, ctas, descending, overlap):
+    """Persistent / descending launch shapes of the AdamW and FedAvg kernels and plain instead of overlapped
+    launches change scheduling only: the results are bit-identical to the defaults."""
     def run(tune):
         c = Case([40000, 30011, 5000], 3, 4, 1, H=1, Q=8, opt_state=True, hp=orc.Hyper(max_grad_norm=0.05))
         if tune:
-            for kern in (fls.FLS_KERNEL_REDUCE, fls.FLS_KERNEL_ADAMW, fls.FLS_KERNEL_FEDAVG):
+            for kern in (fls.FLS_KERNEL_REDUCE, fls.FLS_KERNEL_ADAMW, fls.FLS_KERNEL_FEDAVG, fls.FLS_KERNEL_ADAMW_FEDAVG):
                 fls.fls_plan_tune(c.sess.plan, kern, ctas, descending)
+            fls.fls_plan_set_overlap(c.sess.plan, overlap)
         for _ in range(2):
             c.step([1, 2, 3])
         c.compare()
