@@ -233,6 +233,8 @@ def run_ours(args, cfg):
         fls.fls_plan_tune(sess.plan, fls.FLS_KERNEL_ADAMW, 0, 1)
     if args.ascending_adamw:
         fls.fls_plan_tune(sess.plan, fls.FLS_KERNEL_ADAMW, 0, 0)
+    if args.staged_reduce:
+        fls.fls_plan_set_staging(sess.plan, True)
     if args.no_overlap:
         fls.fls_plan_set_overlap(sess.plan, False)
     fill_session(sess, cfg)
@@ -339,7 +341,7 @@ def run_ours(args, cfg):
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": cfg["name"], "n_params": P, "groups": G, "shard_dim": cfg["shard_dim"],
                        "replicate_dim": cfg["replicate_dim"], "sync_period": cfg["sync_period"], "grad_dtype": cfg["grad_dtype"],
-                       "fedavg_opt_state": bool(args.opt_state), "fused_aggregation": bool(fused), "fedavg_calls_in_timed_region": fedavg_calls, "l2": "working set exceeds L2, no flush needed",
+                       "fedavg_opt_state": bool(args.opt_state), "fused_aggregation": bool(fused), "staged_reduce": bool(args.staged_reduce), "fedavg_calls_in_timed_region": fedavg_calls, "l2": "working set exceeds L2, no flush needed",
                        "parallelism": "replicas only" if world > 1 else "1 gpu"},
             "hbm_gbs": step_bytes / ms_step / 1e6, "hbm_frac_of_measured_peak": step_bytes / ms_step / 1e6 / peak,
             "hbm_frac_of_8tbs": step_bytes / ms_step / 1e6 / 8000.0,
@@ -460,6 +462,7 @@ def main():
     ap.add_argument("--ctas-fedavg", type=int, default=0)
     ap.add_argument("--descending-adamw", action="store_true")
     ap.add_argument("--ascending-adamw", action="store_true")
+    ap.add_argument("--staged-reduce", action="store_true", help="reduce kernel stages its tiles through shared memory (cp.async.bulk)")
     ap.add_argument("--no-overlap", action="store_true", help="plain launches instead of programmatic dependent launch")
     # slices of a workload, for profiler captures that must stay small (same kernels, fewer bytes)
     ap.add_argument("--n-params", type=int, default=0, help="override P (single flat unit)")

@@ -111,6 +111,28 @@ def test_tuned_launch_shapes_give_identical_results(fls, ctas, descending, overl
     assert all(torch.equal(x, y) for x, y in zip(run(False), run(True)))
 
 
+def test_staged_reduce_variant_is_bit_identical(fls):
+    """The shared-memory staged reduce kernel (bulk asynchronous copies) against the default kernel: same bits,
+    ragged last tiles included; it refuses plans it does not cover."""
+    def run(staged):
+        c = Case([40000, 30008, 8], 2, 8, 1, H=2, Q=8, hp=orc.Hyper(max_grad_norm=0.05))
+        if staged:
+            fls.fls_plan_set_staging(c.sess.plan, True)
+        for _ in range(2):
+            c.step([2, 1])
+            c.compare()
+        assert c.sess.status() == 0
+        out = [c.sess.reduced_grad().clone()] + [x.clone() for x in c.sess.master + c.sess.v + c.sess.param_bf16] + [c.sess.norms().clone()]
+        c.close()
+        return out
+    assert all(torch.equal(x, y) for x, y in zip(run(False), run(True)))
+    c = Case([40000], 1, 4, 2, H=2, Q=8)                     # two-level order: not covered
+    with pytest.raises(fls.FlsError) as e:
+        fls.fls_plan_set_staging(c.sess.plan, True)
+    assert e.value.code == fls.FLS_ESTATE
+    c.close()
+
+
 def test_reduced_gradient_matches_oracle_exactly_for_bf16(fls):
     """With bf16 inputs of similar magnitude the fp32 running sum is exact, so the mean gradient is
     bit-identical to the oracle's (this case is small enough that no element loses bits)."""
