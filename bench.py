@@ -473,7 +473,7 @@ def main():
     ap.add_argument("--grad-dtype", default="", choices=["", "bf16", "f32"], help="override the gradient dtype")
     ap.add_argument("--keep-units", action="store_true", help="with --n-params: keep the unit table's proportions")
     ap.add_argument("--sweep", action="store_true", help="run the bandwidth sweep instead of the benchmark")
-    ap.add_argument("--sweep-out", default="gpurun_out/sweep.jsonl")
+    ap.add_argument("--sweep-out", default="sweep_results.jsonl")
     ap.add_argument("--sweep-exps", default="20,22,24,26,28,30", help="log2 of the parameter counts to sweep")
     args = ap.parse_args()
     if args.sweep:
