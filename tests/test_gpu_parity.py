@@ -413,6 +413,41 @@ def test_bind_rejects_bad_buffers(fls):
     s.close()
 
 
+# ------------------------------------------------------------------ randomized combinations
+def _random_cases(n, seed=20260920):
+    rng = np.random.default_rng(seed)
+    out = []
+    for i in range(n):
+        n_units = int(rng.integers(1, 7))
+        units = [int(x) for x in rng.choice([1, 7, 8, 17, 255, 2048, 2049, 4096, 10007, 30000], n_units)]
+        S = int(rng.choice([1, 2, 3, 4, 8]))
+        R_rep = int(rng.choice([1, 1, 2, 3]))
+        wire = bool(rng.integers(0, 4) == 0)
+        dtype = "bf16" if wire or rng.integers(0, 3) else "f32"
+        out.append(dict(units=units, G=int(rng.choice([1, 2, 3, 4, 8])), S=S, R_rep=R_rep, Q=int(rng.choice([1, 4, 8, 16])),
+                        dtype=dtype, opt_state=bool(rng.integers(0, 2)), fused=bool(rng.integers(0, 2)), wire=wire,
+                        H=int(rng.choice([1, 2, 3])), clip=float(rng.choice([0.0, 0.02, 10.0])),
+                        ctas=int(rng.choice([0, 0, 1, 5])), desc=int(rng.integers(0, 2)), overlap=bool(rng.integers(0, 2)), idx=i))
+    return out
+
+
+@pytest.mark.parametrize("p", _random_cases(40), ids=lambda p: f"case{p['idx']}")
+def test_random_combinations(fls, p):
+    """Random unit tables, mesh shapes, alignment quanta, dtypes, FedAvg options and launch shapes, 3 steps each."""
+    hp = orc.Hyper(max_grad_norm=p["clip"], wire_bf16=p["wire"])
+    c = Case(p["units"], p["G"], p["S"], p["R_rep"], H=p["H"], Q=p["Q"], grad_dtype=p["dtype"], opt_state=p["opt_state"],
+             hp=hp, fused=p["fused"], per_buffer_scale=True, seed=1000 + p["idx"])
+    for kern in (fls.FLS_KERNEL_ADAMW, fls.FLS_KERNEL_FEDAVG, fls.FLS_KERNEL_ADAMW_FEDAVG):
+        fls.fls_plan_tune(c.sess.plan, kern, p["ctas"], p["desc"])
+    fls.fls_plan_set_overlap(c.sess.plan, p["overlap"])
+    counts = [sy.sample_count(p["idx"], g) for g in range(p["G"])]
+    for _ in range(3):
+        c.step(counts)
+        c.compare()
+    assert c.sess.status() == 0
+    c.close()
+
+
 # ------------------------------------------------------------------ full size, in the benchmark's launch configuration
 def _fill_full_size(s, cfg, L):
     """Fills a Session's device buffers from the generator by LOGICAL index (what the oracle samples)."""
