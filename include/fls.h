@@ -119,7 +119,8 @@ typedef struct {
   fls_cost5 wire_bytes;  /* bytes one rank sends per step when D of all-gather / reduce-scatter is the whole
                             unit (S*M_u), the convention of the NCCL performance notes the paper cites        */
   fls_cost5 seconds;     /* Eq. 1-5 with B_S, B_R, B_F; NaN when no bandwidths were given                     */
-  double hbm_bytes_sync_step; /* bytes one fls_sync_step must move in this library: G*N_pad*(K*e_g + 34)      */
+  double hbm_bytes_sync_step; /* bytes one fls_sync_step must move in this library: G*N_pad*(K*e_g + 34), or
+                                 G*N_pad*(2*K*e_g + 26) when K*e_g < 8 (gradients read twice, nothing stored)  */
   double hbm_bytes_fedavg;    /* bytes one fls_fedavg must move: G*N_pad*10, or *26 with optimizer state      */
 } fls_comm_costs;
 
@@ -178,7 +179,8 @@ int fls_sync_step_fedavg(fls_plan* plan, double lr, const uint64_t* sample_count
  * the last step, valid once that step has completed on its stream.  Either output may be NULL. */
 int fls_get_norms(const fls_plan* plan, const float** dev_norms, const float** dev_coefs);
 
-/* Device pointer to the reduced (mean) gradient of the LAST group processed: N_pad floats, shard order. */
+/* Device pointer to the reduced (mean) gradient of the LAST group processed: N_pad floats, shard order.
+ * FLS_ESTATE if the last step stored none (plans with K*e_g < 8 bytes recompute it, see fls_plan_set_recompute). */
 int fls_get_reduced_grad(const fls_plan* plan, const float** dev_gbar);
 
 /* Device pointer to the sticky status word (FLS_STATUS_* bits).  Non-finite values are not errors:
@@ -208,6 +210,13 @@ int fls_plan_tune(fls_plan* plan, uint32_t kernel, int ctas_per_sm, int descendi
  * it is kept so that this can be re-measured.  Results are identical.  Its wait on the copies is bounded: on
  * expiry FLS_STATUS_STAGING_TIMEOUT is set in the status word and the affected tile is left unwritten. */
 int fls_plan_set_staging(fls_plan* plan, int enabled);
+
+/* How fls_sync_step gets the mean gradient into AdamW.  With fewer than 8 gradient bytes per element (bf16 and
+ * K <= 3, fp32 and K = 1) reading the gradients twice (a norm pass, then AdamW forming the mean itself: 2*K*e_g +
+ * 26 bytes per element) is cheaper than storing the fp32 mean and reading it back (K*e_g + 34); such plans do
+ * that by default.  mode 0 forces store-and-reread, 1 forces recomputation (FLS_ESTATE if the plan does not
+ * qualify), -1 restores the default.  The results are identical either way. */
+int fls_plan_set_recompute(fls_plan* plan, int mode);
 
 /* enabled != 0 (the default): inside one call every kernel but the first is launched so that its first CTAs may
  * start during the tail of the kernel before it (programmatic dependent launch); they fetch what that kernel does

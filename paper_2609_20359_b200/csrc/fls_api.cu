@@ -64,6 +64,7 @@ struct fls_plan {
 
   bool overlap = true;     // programmatic dependent launch between the kernels of one call
   bool staged_reduce = false;
+  bool recompute = false;  // K * e_g < 8: the norm pass stores nothing and AdamW forms the mean gradient again
   bool profiling = false;
   std::vector<TimedLaunch> timed;
   std::vector<cudaEvent_t> event_pool;
@@ -75,6 +76,7 @@ struct fls_plan {
   const Segment* d_segs() const { return reinterpret_cast<const Segment*>(ws + kWsSegments); }
   float* d_gbar(uint32_t slot = 0) const { return reinterpret_cast<float*>(ws + lay.ws_scratch_offset + lay.scratch_stride * slot); }
   uint32_t last_slot = 0;   // where the last processed group's reduced gradient lives
+  bool gbar_valid = false;  // false after a step of a recompute plan: nothing was stored
   float* d_norms() const { return reinterpret_cast<float*>(ws + kWsNorms); }
   float* d_coefs() const { return reinterpret_cast<float*>(ws + kWsCoefs); }
   double* d_normsq() const { return reinterpret_cast<double*>(ws + kWsNormSq); }
@@ -183,6 +185,9 @@ int run_group(fls_plan* p, uint32_t g, double lr, uint64_t t_new, cudaStream_t s
   ra.normsq_out = p->d_normsq() + g;
   ra.status = p->d_status();
   ra.max_grad_norm = d.max_grad_norm;
+  const bool recompute = p->recompute && with_adamw;   // the fused aggregation needs the stored gradients
+  ra.store_gbar = recompute ? 0 : 1;
+  p->gbar_valid = !recompute;
   const bool f32 = d.grad_dtype == FLS_GRAD_F32;
   const bool overlap = p->overlap && !p->profiling;   // event records between kernels would serialise anyway
   cudaError_t e = timed_launch(p, FLS_KERNEL_REDUCE, st, [&] {
@@ -203,7 +208,15 @@ int run_group(fls_plan* p, uint32_t g, double lr, uint64_t t_new, cudaStream_t s
   aa.coef = p->d_coefs() + g;
   aa.decay = sc.decay; aa.beta1 = sc.beta1; aa.omb1 = sc.omb1; aa.beta2 = sc.beta2; aa.omb2 = sc.omb2;
   aa.step_size = sc.step_size; aa.inv_sqrt_bc2 = sc.inv_sqrt_bc2; aa.eps = sc.eps;
-  e = timed_launch(p, FLS_KERNEL_ADAMW, st, [&] { return launch_adamw(aa, p->grid_for(FLS_KERNEL_ADAMW), st, overlap); });
+  if (recompute) {
+    ReduceAdamArgs rp{};
+    rp.r = ra;
+    rp.a = aa;
+    e = timed_launch(p, FLS_KERNEL_ADAMW, st,
+                     [&] { return launch_reduce_adamw(rp, f32, p->reduce_sg, p->grid_for(FLS_KERNEL_ADAMW), st, overlap); });
+  } else {
+    e = timed_launch(p, FLS_KERNEL_ADAMW, st, [&] { return launch_adamw(aa, p->grid_for(FLS_KERNEL_ADAMW), st, overlap); });
+  }
   if (e != cudaSuccess) return cuda_fail(e, "adamw kernel launch");
   return FLS_OK;
 }
@@ -284,6 +297,8 @@ int fls_plan_create(const fls_plan_desc* desc, fls_plan** out) {
     p->reduce_sg = -1;
   }
   if (d.reduce_wire == FLS_WIRE_BF16) p->reduce_sg = -2;   // generic kernel, bf16 rounding after every sum
+  // fewer than 8 gradient bytes per element: a second read of the gradients costs less than the fp32 round trip
+  p->recompute = d.reduce_wire == FLS_WIRE_F32 && K * (d.grad_dtype == FLS_GRAD_F32 ? 4 : 2) < 8;
   *out = p;
   return FLS_OK;
 }
@@ -531,6 +546,7 @@ int fls_get_norms(const fls_plan* p, const float** dev_norms, const float** dev_
 int fls_get_reduced_grad(const fls_plan* p, const float** dev_gbar) {
   if (!p || !dev_gbar) return fail(FLS_EINVAL, "fls_get_reduced_grad: null argument");
   if (!p->bound) return fail(FLS_ESTATE, "fls_get_reduced_grad: plan has no buffers bound");
+  if (!p->gbar_valid) return fail(FLS_ESTATE, "fls_get_reduced_grad: the last step did not store the reduced gradient (recompute plan)");
   *dev_gbar = p->d_gbar(p->last_slot);
   return FLS_OK;
 }
@@ -578,6 +594,16 @@ int fls_plan_set_staging(fls_plan* p, int enabled) {
     if (!ok) return fail(FLS_ESTATE, "fls_plan_set_staging: needs bf16 gradients, flat order, K = 8 and 8-element aligned segments");
   }
   p->staged_reduce = enabled != 0;
+  return FLS_OK;
+}
+
+int fls_plan_set_recompute(fls_plan* p, int mode) {
+  if (!p) return fail(FLS_EINVAL, "fls_plan_set_recompute: null plan");
+  const fls_plan_desc& d = p->desc;
+  const bool small = uint64_t(p->K) * (d.grad_dtype == FLS_GRAD_F32 ? 4 : 2) < 8;
+  if (mode > 0 && (!small || d.reduce_wire != FLS_WIRE_F32))
+    return fail(FLS_ESTATE, "fls_plan_set_recompute: only for K*e_g < 8 bytes and fp32 partial sums");
+  p->recompute = mode > 0 || (mode < 0 && small && d.reduce_wire == FLS_WIRE_F32);
   return FLS_OK;
 }
 

@@ -297,7 +297,7 @@ __device__ __noinline__ float reduce_slice_scalar(const ReduceArgs& a, uint64_t 
   for (uint32_t e = 0; e < n; ++e) {
     float g[1];
     reduce_elems<1, F32, 0, WIRE ? -2 : -1>(a, j + e, g);
-    a.gbar[addr + e] = g[0];
+    if (a.store_gbar) a.gbar[addr + e] = g[0];
     sq = fmaf(g[0], g[0], sq);
   }
   return sq;
@@ -322,8 +322,10 @@ __global__ void __launch_bounds__(THREADS, MINB) fls_reduce_kernel(const __grid_
       F8 o;
 #pragma unroll
       for (int e = 0; e < 8; ++e) { o.v[e] = g[e]; sq = fmaf(g[e], g[e], sq); }
-      dep_wait();                        // the previous group's AdamW kernel may still be reading the scratch
-      st8_keep(a.gbar + s.a, o);
+      if (a.store_gbar) {
+        dep_wait();                      // the previous group's AdamW kernel may still be reading the scratch
+        st8_keep(a.gbar + s.a, o);
+      }
     } else if (s.n) {
       dep_wait();
       sq = reduce_slice_scalar<F32, SG == -2>(a, s.j, s.a, s.n);
@@ -507,6 +509,56 @@ __global__ void __launch_bounds__(kThreads, 3) fls_adamw_kernel(const __grid_con
     } else if (s.n) {
       if (!waited) { dep_wait(); dep_launch(); c = __ldcg(a.coef); waited = true; }
       adamw_slice_scalar(a, c, s.j, s.a, s.n);
+    }
+  }
+  if (!waited) { dep_wait(); dep_launch(); }
+}
+
+// AdamW with the mean gradient formed in place (recompute plan).  With few gradient bytes per element
+// (K * e_g < 8) reading the gradients a second time is cheaper than writing the fp32 mean and reading it
+// back; reduce_elems is the same code the norm pass ran, so the gradient and the result are the same bits.
+template <bool F32>
+__device__ __noinline__ void reduce_adamw_slice_scalar(const ReduceAdamArgs& p, float c, uint64_t j, uint64_t addr, uint32_t n) {
+  const AdamArgs& a = p.a;
+  for (uint32_t e = 0; e < n; ++e) {
+    float g[1];
+    reduce_elems<1, F32, 0, -1>(p.r, j + e, g);
+    float th = a.theta[addr + e], m = a.m[addr + e], v = a.v[addr + e];
+    adamw_one(a, c, g[0], th, m, v);
+    a.theta[addr + e] = th; a.m[addr + e] = m; a.v[addr + e] = v;
+    a.pbf16[j + e] = to_bf16_bits(th);
+  }
+}
+
+template <bool F32, int KT, int SG>
+__global__ void __launch_bounds__(kThreads, KT == 0 ? 2 : 3) fls_reduce_adamw_kernel(const __grid_constant__ ReduceAdamArgs p) {
+  const AdamArgs& a = p.a;
+  const uint32_t n_tiles = a.idx.n_tiles;
+  if (blockIdx.x >= n_tiles) { dep_wait(); dep_launch(); return; }
+  float c = 0.f;
+  bool waited = false;
+  Walker w;
+  w.init(a.idx, a.descending ? n_tiles - 1 - blockIdx.x : blockIdx.x);
+  for (uint32_t lin = blockIdx.x; lin < n_tiles; lin += gridDim.x) {
+    const uint32_t tile = a.descending ? n_tiles - 1 - lin : lin;
+    const Slice s = slice_of(w.seek(tile), tile, threadIdx.x);
+    if (s.vec) {
+      // nothing read here is written by the norm pass: all loads can precede the wait for it
+      F8 th = ld8_stream(a.theta + s.a);
+      F8 m = ld8_stream(a.m + s.a);
+      F8 v = ld8_stream(a.v + s.a);
+      float g[8];
+      reduce_elems<8, F32, KT, SG>(p.r, s.j, g);
+      if (!waited) { dep_wait(); dep_launch(); c = __ldcg(a.coef); waited = true; }
+#pragma unroll
+      for (int e = 0; e < 8; ++e) adamw_one(a, c, g[e], th.v[e], m.v[e], v.v[e]);
+      st8_stream(a.theta + s.a, th);
+      st8_stream(a.m + s.a, m);
+      st8_stream(a.v + s.a, v);
+      st_b128_stream(a.pbf16 + s.j, pack_bf16x8(th));
+    } else if (s.n) {
+      if (!waited) { dep_wait(); dep_launch(); c = __ldcg(a.coef); waited = true; }
+      reduce_adamw_slice_scalar<F32>(p, c, s.j, s.a, s.n);
     }
   }
   if (!waited) { dep_wait(); dep_launch(); }
@@ -750,6 +802,27 @@ cudaError_t launch_reduce(const ReduceArgs& a, bool f32, int sg, cudaStream_t st
     launch_reduce_t<true>(a, sg, grid, st, overlap);
   else
     launch_reduce_t<false>(a, sg, grid, st, overlap);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_reduce_adamw(const ReduceAdamArgs& a, bool f32, int sg, unsigned grid, cudaStream_t st, bool overlap) {
+  // the recompute plan exists for K * e_g < 8: bf16 with K <= 3, fp32 with K = 1
+  const uint32_t K = a.r.K;
+  if (f32) {
+    launch_k(fls_reduce_adamw_kernel<true, 1, 0>, a, grid, kThreads, st, overlap);
+  } else if (K == 1) {
+    launch_k(fls_reduce_adamw_kernel<false, 1, 0>, a, grid, kThreads, st, overlap);
+  } else if (K == 2 && sg == 0) {
+    launch_k(fls_reduce_adamw_kernel<false, 2, 0>, a, grid, kThreads, st, overlap);
+  } else if (K == 2 && sg == 1) {
+    launch_k(fls_reduce_adamw_kernel<false, 2, 1>, a, grid, kThreads, st, overlap);
+  } else if (sg == 0) {
+    launch_k(fls_reduce_adamw_kernel<false, 0, 0>, a, grid, kThreads, st, overlap);
+  } else if (sg == 1) {
+    launch_k(fls_reduce_adamw_kernel<false, 0, 1>, a, grid, kThreads, st, overlap);
+  } else {
+    launch_k(fls_reduce_adamw_kernel<false, 0, -1>, a, grid, kThreads, st, overlap);
+  }
   return cudaGetLastError();
 }
 

@@ -33,6 +33,7 @@ struct ReduceArgs {
   double* normsq_out;
   uint32_t* status;
   double max_grad_norm;
+  int store_gbar;                          // 0: norm only (the recompute plan: the mean gradient is formed again in AdamW)
 };
 
 struct AdamArgs {
@@ -43,6 +44,12 @@ struct AdamArgs {
   int descending;
   const float* coef;                       // device, written by the reduce kernel of the same group
   float decay, beta1, omb1, beta2, omb2, step_size, inv_sqrt_bc2, eps;
+};
+
+// AdamW that forms the mean gradient itself from the K gradient buffers (recompute plan, small K).
+struct ReduceAdamArgs {
+  ReduceArgs r;                            // gradient pointers, level structure, 1/K (its outputs are not used)
+  AdamArgs a;                              // state pointers, scalars (its gbar is not used)
 };
 
 struct FedavgArgs {
@@ -80,6 +87,7 @@ unsigned reduce_grid(const ReduceArgs& a, int sg);
 cudaError_t launch_reduce(const ReduceArgs& a, bool f32, int sg, cudaStream_t st, bool overlap);
 // Shared-memory staged variant of the reduce kernel (bf16, flat order, K = 8, fully vectorisable layout only).
 cudaError_t launch_reduce_staged(const ReduceArgs& a, cudaStream_t st, bool overlap);
+cudaError_t launch_reduce_adamw(const ReduceAdamArgs& a, bool f32, int sg, unsigned grid, cudaStream_t st, bool overlap);
 cudaError_t launch_adamw(const AdamArgs& a, unsigned grid, cudaStream_t st, bool overlap);
 cudaError_t launch_fedavg(const FedavgArgs& a, unsigned grid, cudaStream_t st, bool overlap);
 cudaError_t launch_adamw_fedavg(const FusedArgs& a, unsigned grid, cudaStream_t st, bool overlap);

@@ -57,7 +57,10 @@ void comm_report(const Layout& lay, const fls_plan_desc& d, const double* bw, fl
     out->seconds = fls_cost5{nan, nan, nan, nan, nan};
   }
   const double K = S * R;
-  out->hbm_bytes_sync_step = F * double(lay.n_padded) * (K * e + 34.0);
+  // store-and-reread moves K*e_g + 34 bytes per element; with K*e_g < 8 the library reads the gradients twice
+  // instead and moves 2*K*e_g + 26
+  const double per_elem = (K * e < 8.0 && d.reduce_wire == FLS_WIRE_F32) ? 2.0 * K * e + 26.0 : K * e + 34.0;
+  out->hbm_bytes_sync_step = F * double(lay.n_padded) * per_elem;
   out->hbm_bytes_fedavg = F * double(lay.n_padded) * ((d.fedavg_what & FLS_AVG_OPT_STATE) ? 26.0 : 10.0);
 }
 

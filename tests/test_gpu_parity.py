@@ -111,6 +111,34 @@ def test_tuned_launch_shapes_give_identical_results(fls, ctas, descending, overl
     assert all(torch.equal(x, y) for x, y in zip(run(False), run(True)))
 
 
+@pytest.mark.parametrize("units,G,S,R_rep,Q,dtype", [([40000, 30011], 2, 1, 1, 8, "bf16"), ([40000, 30011], 2, 2, 1, 8, "bf16"),
+                                                     ([40000, 30011], 2, 1, 2, 8, "bf16"), ([70001], 2, 3, 1, 1, "bf16"),
+                                                     ([70001], 2, 1, 3, 8, "bf16"), ([40000, 30011], 2, 1, 1, 8, "f32")])
+def test_recompute_plan_is_bit_identical_to_store_and_reread(fls, units, G, S, R_rep, Q, dtype):
+    """K*e_g < 8 bytes: by default the mean gradient is recomputed inside AdamW instead of stored; forcing the
+    stored path gives the same bits, both match the oracle, and the stored gradient is only offered when it exists."""
+    outs = []
+    for mode in (-1, 0):
+        c = Case(units, G, S, R_rep, H=2, Q=Q, grad_dtype=dtype, hp=orc.Hyper(max_grad_norm=0.05), per_buffer_scale=True)
+        fls.fls_plan_set_recompute(c.sess.plan, mode)
+        for _ in range(3):
+            c.step()
+            c.compare()
+        if mode == -1:
+            with pytest.raises(fls.FlsError) as e:
+                c.sess.reduced_grad()
+            assert e.value.code == fls.FLS_ESTATE
+        else:
+            assert c.sess.reduced_grad().numel() == c.L.n_padded
+        outs.append([x.clone() for x in c.sess.master + c.sess.m + c.sess.v + c.sess.param_bf16] + [c.sess.norms().clone()])
+        c.close()
+    assert all(torch.equal(x, y) for x, y in zip(*outs))
+    c = Case([4096], 1, 8, 1, H=2, Q=8)
+    with pytest.raises(fls.FlsError):
+        fls.fls_plan_set_recompute(c.sess.plan, 1)          # 16 gradient bytes per element: does not qualify
+    c.close()
+
+
 def test_staged_reduce_variant_is_bit_identical(fls):
     """The shared-memory staged reduce kernel (bulk asynchronous copies) against the default kernel: same bits,
     ragged last tiles included; it refuses plans it does not cover."""
