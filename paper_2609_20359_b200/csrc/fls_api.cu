@@ -142,8 +142,6 @@ cudaError_t timed_launch(fls_plan* p, int kernel, cudaStream_t st, F&& launch) {
   return e;
 }
 
-// chain: the previous operation on `st` is a kernel of this same call, so this group's first kernel may
-// overlap its tail
 struct AdamScalars { float decay, beta1, omb1, beta2, omb2, step_size, inv_sqrt_bc2, eps; };
 
 // Scalars of the AdamW step, in double on the host, handed to the kernels as fp32.
@@ -162,8 +160,10 @@ AdamScalars adam_scalars(const fls_plan_desc& d, double lr, uint64_t t_new) {
   return s;
 }
 
-// slot: which reduced-gradient buffer of the workspace receives the mean gradient; with_adamw = false stops
-// after the reduction (the fused aggregation applies AdamW to all groups afterwards)
+// One group's reduce (+ AdamW) launches.  chain: the previous operation on `st` is a kernel of this same call,
+// so this group's first kernel may overlap its tail.  slot: which reduced-gradient buffer of the workspace
+// receives the mean gradient; with_adamw = false stops after the reduction (the fused aggregation applies AdamW
+// to all groups afterwards).
 int run_group(fls_plan* p, uint32_t g, double lr, uint64_t t_new, cudaStream_t st, bool chain, uint32_t slot = 0,
               bool with_adamw = true) {
   const fls_plan_desc& d = p->desc;
