@@ -7,11 +7,15 @@ fls_* name loads libfls.so and raises if it is missing (build it with
 """
 import importlib
 
-__all__ = ["build"]
+_SUBMODULES = ("build", "session", "_binding")
+__all__ = list(_SUBMODULES)
 
 
 def __getattr__(name):
-    # loaded on first use so that `python -m paper_2609_20359_b200.build` can run before the library exists
+    # Submodules first (so that `from paper_2609_20359_b200 import build` works before the library exists);
+    # every other name is looked up in the binding, which loads libfls.so on first use.
+    if name in _SUBMODULES:
+        return importlib.import_module("." + name, __name__)
     if name.startswith("__"):
         raise AttributeError(name)
     binding = importlib.import_module("._binding", __name__)
