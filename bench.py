@@ -322,6 +322,9 @@ def run_ours(args, cfg):
         # written), m and v 8 B each; the figure is the mean over the launches of one call
         per_launch = {"reduce": N * (sess.K * eg + 4), "adamw": N * 30, "fedavg": N * G * (26 / 3 if args.opt_state else 10),
                       "adamw_fedavg": N * G * 30}
+        if sess.K * eg < 8:
+            # small K: nothing is stored by the norm pass and AdamW reads the gradients again
+            per_launch.update(reduce=N * sess.K * eg, adamw=N * (sess.K * eg + 26))
         kernels = {}
         for i, name in enumerate(("reduce", "adamw", "fedavg", "adamw_fedavg")):
             if kn[i]:

@@ -214,68 +214,9 @@ __device__ __forceinline__ void unpack(const Raw<1, true>& x, float (&f)[1]) { f
 //   SG = -2 : as -1, with every partial sum and the final mean rounded to bf16 (the bf16-wire emulation).
 __device__ __forceinline__ float round_bf16(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
 
-template <int N, bool F32, int KT, int SG>
-__device__ __forceinline__ void reduce_elems(const ReduceArgs& a, uint64_t j, float (&mean)[N]) {
-  constexpr int B = KT ? KT : 8;            // buffers per batch
-  const uint32_t K = KT ? uint32_t(KT) : a.K;
-  float inner[N], outer[N];
-#pragma unroll
-  for (int e = 0; e < N; ++e) inner[e] = outer[e] = 0.f;
-#pragma unroll 1
-  for (uint32_t k0 = 0; k0 < K; k0 += B) {
-    Raw<N, F32> raw[B];
-#pragma unroll
-    for (int b = 0; b < B; ++b)
-      if (KT || k0 + b < K) load_raw(raw[b], a.grad[KT ? b : k0 + b], j);
-    if constexpr (SG == 0) {
-#pragma unroll
-      for (int b = 0; b < B; ++b) {
-        if (KT || k0 + b < K) {
-          float x[N];
-          unpack(raw[b], x);
-#pragma unroll
-          for (int e = 0; e < N; ++e) inner[e] += x[e];
-        }
-      }
-      if (KT || ((a.fold_mask >> (k0 >> 3)) & 1u)) {
-#pragma unroll
-        for (int e = 0; e < N; ++e) { outer[e] += inner[e]; inner[e] = 0.f; }
-      }
-    } else if constexpr (SG > 0) {
-#pragma unroll
-      for (int g0 = 0; g0 < B; g0 += SG) {
-        if (KT || k0 + g0 < K) {
-          float s[N];
-          unpack(raw[g0], s);
-#pragma unroll
-          for (int i = 1; i < SG; ++i) {
-            float x[N];
-            unpack(raw[g0 + i], x);
-#pragma unroll
-            for (int e = 0; e < N; ++e) s[e] += x[e];
-          }
-#pragma unroll
-          for (int e = 0; e < N; ++e) outer[e] += s[e];
-        }
-      }
-    } else {
-#pragma unroll
-      for (int b = 0; b < B; ++b) {
-        const uint32_t k = k0 + b;
-        if (k < K) {
-          float x[N];
-          unpack(raw[b], x);
-#pragma unroll
-          for (int e = 0; e < N; ++e) inner[e] = (SG == -2) ? round_bf16(inner[e] + x[e]) : inner[e] + x[e];
-          if ((a.end_mask >> k) & 1ull) {
-#pragma unroll
-            for (int e = 0; e < N; ++e) { outer[e] = (SG == -2) ? round_bf16(outer[e] + inner[e]) : outer[e] + inner[e]; inner[e] = 0.f; }
-          }
-        }
-      }
-    }
-  }
-  // one scaling by 1/K after the last level: a multiply when 1/K is exact, else an IEEE division
+// one scaling by 1/K after the last level: a multiply when 1/K is exact, else an IEEE division
+template <int N>
+__device__ __forceinline__ void scale_mean(const ReduceArgs& a, const float (&outer)[N], float (&mean)[N]) {
   if (a.k_is_pow2) {
 #pragma unroll
     for (int e = 0; e < N; ++e) mean[e] = outer[e] * a.inv_k;
@@ -283,9 +224,119 @@ __device__ __forceinline__ void reduce_elems(const ReduceArgs& a, uint64_t j, fl
 #pragma unroll
     for (int e = 0; e < N; ++e) mean[e] = __fdiv_rn(outer[e], a.k_float);
   }
-  if constexpr (SG == -2) {
+}
+
+// Static K (KT = K in {1, 2, 4, 8}, SG in {0, 1, 2, 4}): the mean of KT values already loaded.
+template <int N, bool F32, int KT, int SG>
+__device__ __forceinline__ void combine_loaded(const ReduceArgs& a, const Raw<N, F32> (&raw)[KT], float (&mean)[N]) {
+  static_assert(KT > 0 && SG >= 0, "static shapes only");
+  float outer[N];
 #pragma unroll
-    for (int e = 0; e < N; ++e) mean[e] = round_bf16(mean[e]);
+  for (int e = 0; e < N; ++e) outer[e] = 0.f;
+  if constexpr (SG == 0) {
+    float inner[N];
+#pragma unroll
+    for (int e = 0; e < N; ++e) inner[e] = 0.f;
+#pragma unroll
+    for (int b = 0; b < KT; ++b) {
+      float x[N];
+      unpack(raw[b], x);
+#pragma unroll
+      for (int e = 0; e < N; ++e) inner[e] += x[e];
+    }
+#pragma unroll
+    for (int e = 0; e < N; ++e) outer[e] += inner[e];
+  } else {
+#pragma unroll
+    for (int g0 = 0; g0 < KT; g0 += SG) {
+      float s[N];
+      unpack(raw[g0], s);
+#pragma unroll
+      for (int i = 1; i < SG; ++i) {
+        float x[N];
+        unpack(raw[g0 + i], x);
+#pragma unroll
+        for (int e = 0; e < N; ++e) s[e] += x[e];
+      }
+#pragma unroll
+      for (int e = 0; e < N; ++e) outer[e] += s[e];
+    }
+  }
+  scale_mean<N>(a, outer, mean);
+}
+
+template <int N, bool F32, int KT, int SG>
+__device__ __forceinline__ void reduce_elems(const ReduceArgs& a, uint64_t j, float (&mean)[N]) {
+  if constexpr (KT > 0 && SG >= 0) {
+    Raw<N, F32> raw[KT];
+#pragma unroll
+    for (int b = 0; b < KT; ++b) load_raw(raw[b], a.grad[b], j);
+    combine_loaded<N, F32, KT, SG>(a, raw, mean);
+  } else {
+    // run-time K: batches of 8 buffers
+    const uint32_t K = a.K;
+    float inner[N], outer[N];
+#pragma unroll
+    for (int e = 0; e < N; ++e) inner[e] = outer[e] = 0.f;
+#pragma unroll 1
+    for (uint32_t k0 = 0; k0 < K; k0 += 8) {
+      Raw<N, F32> raw[8];
+#pragma unroll
+      for (int b = 0; b < 8; ++b)
+        if (k0 + b < K) load_raw(raw[b], a.grad[k0 + b], j);
+      if constexpr (SG == 0) {
+#pragma unroll
+        for (int b = 0; b < 8; ++b) {
+          if (k0 + b < K) {
+            float x[N];
+            unpack(raw[b], x);
+#pragma unroll
+            for (int e = 0; e < N; ++e) inner[e] += x[e];
+          }
+        }
+        if ((a.fold_mask >> (k0 >> 3)) & 1u) {
+#pragma unroll
+          for (int e = 0; e < N; ++e) { outer[e] += inner[e]; inner[e] = 0.f; }
+        }
+      } else if constexpr (SG > 0) {
+#pragma unroll
+        for (int g0 = 0; g0 < 8; g0 += SG) {
+          if (k0 + g0 < K) {
+            float s[N];
+            unpack(raw[g0], s);
+#pragma unroll
+            for (int i = 1; i < SG; ++i) {
+              float x[N];
+              unpack(raw[g0 + i], x);
+#pragma unroll
+              for (int e = 0; e < N; ++e) s[e] += x[e];
+            }
+#pragma unroll
+            for (int e = 0; e < N; ++e) outer[e] += s[e];
+          }
+        }
+      } else {
+#pragma unroll
+        for (int b = 0; b < 8; ++b) {
+          const uint32_t k = k0 + b;
+          if (k < K) {
+            float x[N];
+            unpack(raw[b], x);
+#pragma unroll
+            for (int e = 0; e < N; ++e) inner[e] = (SG == -2) ? round_bf16(inner[e] + x[e]) : inner[e] + x[e];
+            if ((a.end_mask >> k) & 1ull) {
+#pragma unroll
+              for (int e = 0; e < N; ++e) { outer[e] = (SG == -2) ? round_bf16(outer[e] + inner[e]) : outer[e] + inner[e]; inner[e] = 0.f; }
+            }
+          }
+        }
+      }
+    }
+    scale_mean<N>(a, outer, mean);
+    if constexpr (SG == -2) {
+#pragma unroll
+      for (int e = 0; e < N; ++e) mean[e] = round_bf16(mean[e]);
+    }
   }
 }
 
@@ -303,32 +354,84 @@ __device__ __noinline__ float reduce_slice_scalar(const ReduceArgs& a, uint64_t 
   return sq;
 }
 
-// One pass, no loop: a CTA of THREADS threads owns THREADS/256 consecutive tiles, one per group of 256
-// threads, and the grid covers the whole buffer.  MINB resident CTAs per SM fix the register budget:
-// 1024 x 2 (32 registers) for the flat order, 512 x 3 (42 registers) for the two-level orders, which
-// carry a second set of accumulators, 256 x 2 for a run-time K.
-template <bool F32, int KT, int SG, int THREADS, int MINB>
+// One pass, no loop: a CTA of THREADS threads owns U * THREADS/256 consecutive tiles (each group of 256
+// threads takes every (THREADS/256)-th of them, U in all) and the grid covers the whole buffer.  MINB resident
+// CTAs per SM fix the register budget: 1024 x 2 (32 registers) for the flat order with K = 4 or 8, 512 x 3 (42
+// registers) for the two-level orders, which carry a second set of accumulators, 256 x 2 for a run-time K.
+// With K = 1 or 2 a thread would have only one or two 16-byte loads in flight, so those shapes take U > 1 tiles
+// per thread (512 x 2 CTAs) and issue the loads of all of them before the first add.
+template <bool F32, int KT, int SG>
+__device__ __forceinline__ float reduce_one_tile(const ReduceArgs& a, uint32_t tile, uint32_t lane) {
+  float sq = 0.f;
+  const Slice s = slice_of(a.idx.segs + find_segment(a.idx, tile), tile, lane);
+  if (s.vec) {
+    float g[8];
+    reduce_elems<8, F32, KT, SG>(a, s.j, g);
+    F8 o;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) { o.v[e] = g[e]; sq = fmaf(g[e], g[e], sq); }
+    if (a.store_gbar) {
+      dep_wait();                        // the previous group's AdamW kernel may still be reading the scratch
+      st8_keep(a.gbar + s.a, o);
+    }
+  } else if (s.n) {
+    dep_wait();
+    sq = reduce_slice_scalar<F32, SG == -2>(a, s.j, s.a, s.n);
+  }
+  return sq;
+}
+
+template <bool F32, int KT, int SG, int THREADS, int MINB, int U>
 __global__ void __launch_bounds__(THREADS, MINB) fls_reduce_kernel(const __grid_constant__ ReduceArgs a) {
   __shared__ double sh[THREADS / 32];
   __shared__ bool is_last;
+  constexpr uint32_t T = THREADS / kThreads;
+  const uint32_t lane = threadIdx.x % kThreads;
+  const uint32_t first = blockIdx.x * (T * U) + threadIdx.x / kThreads;   // this thread's tiles: first + u*T
   float sq = 0.f;
-  const uint32_t tile = blockIdx.x * (THREADS / kThreads) + threadIdx.x / kThreads;
-  if (tile < a.idx.n_tiles) {
-    // the segment table and the gradients are not written by any kernel of the step: read them at once
-    const Slice s = slice_of(a.idx.segs + find_segment(a.idx, tile), tile, threadIdx.x % kThreads);
-    if (s.vec) {
-      float g[8];
-      reduce_elems<8, F32, KT, SG>(a, s.j, g);
-      F8 o;
-#pragma unroll
-      for (int e = 0; e < 8; ++e) { o.v[e] = g[e]; sq = fmaf(g[e], g[e], sq); }
-      if (a.store_gbar) {
-        dep_wait();                      // the previous group's AdamW kernel may still be reading the scratch
-        st8_keep(a.gbar + s.a, o);
+  if constexpr (U == 1) {
+    if (first < a.idx.n_tiles) sq = reduce_one_tile<F32, KT, SG>(a, first, lane);
+  } else {
+    static_assert(KT > 0 && SG >= 0, "several tiles per thread only for a static K");
+    // fast path: all U tiles lie in one aligned segment and are full, so their addresses are a stride apart
+    const uint32_t last = first + (U - 1) * T;
+    bool fast = false;
+    uint64_t j0 = 0, a0 = 0;
+    if (last < a.idx.n_tiles) {
+      const Segment* sg = a.idx.segs + find_segment(a.idx, first);
+      const uint64_t begin = __ldg(&sg->tile_begin);
+      if (uint64_t(last) < __ldg(&sg->tile_end) && __ldg(&sg->aligned) &&
+          (uint64_t(last) - begin + 1) * kTile <= __ldg(&sg->len)) {
+        const uint64_t e0 = (uint64_t(first) - begin) * kTile + lane * kVec;
+        j0 = __ldg(&sg->j0) + e0;
+        a0 = __ldg(&sg->a0) + e0;
+        fast = true;
       }
-    } else if (s.n) {
-      dep_wait();
-      sq = reduce_slice_scalar<F32, SG == -2>(a, s.j, s.a, s.n);
+    }
+    if (fast) {
+      constexpr uint64_t stride = uint64_t(T) * kTile;
+      Raw<8, F32> raw[U][KT];
+#pragma unroll
+      for (int u = 0; u < U; ++u)
+#pragma unroll
+        for (int b = 0; b < KT; ++b) load_raw(raw[u][b], a.grad[b], j0 + u * stride);
+      if (a.store_gbar) dep_wait();
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        float g[8];
+        combine_loaded<8, F32, KT, SG>(a, raw[u], g);
+        F8 o;
+        float s8 = 0.f;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) { o.v[e] = g[e]; s8 = fmaf(g[e], g[e], s8); }
+        sq += s8;
+        if (a.store_gbar) st8_keep(a.gbar + a0 + u * stride, o);
+      }
+    } else {
+      for (int u = 0; u < U; ++u) {
+        const uint32_t tile = first + u * T;
+        if (tile < a.idx.n_tiles) sq += reduce_one_tile<F32, KT, SG>(a, tile, lane);
+      }
     }
   }
   dep_wait();                            // partials, ticket and the norm slots belong to the predecessor until now
@@ -727,6 +830,10 @@ __global__ void __launch_bounds__(kThreads, 3) fls_adamw_fedavg_kernel(const __g
 constexpr int kFlatThreads = FLS_FLAT_THREADS, kFlatMinB = FLS_FLAT_MINB;       // SG == 0 with a static K
 constexpr int kLevelThreads = FLS_LEVEL_THREADS, kLevelMinB = FLS_LEVEL_MINB;   // two-level orders with a static K
 constexpr int kAnyThreads = 256, kAnyMinB = 2;         // run-time K: batches of 8 loads need the registers
+constexpr int kFewThreads = 512, kFewMinB = 2;         // K = 1 or 2: several tiles per thread (see tiles_per_thread)
+
+// tiles per thread so that 8 (bf16) or 4 (fp32, 32-byte) loads are in flight per thread; 1 for K >= 4
+template <bool F32, int KT> constexpr int tiles_per_thread() { return (KT == 1 || KT == 2) ? (F32 ? 4 : 8) / KT : 1; }
 
 // Launch, with programmatic stream serialization if `overlap` (see dep_wait / dep_launch above).
 template <typename Args>
@@ -744,19 +851,24 @@ void launch_k(void (*kernel)(Args), const Args& a, unsigned grid, unsigned threa
   cudaLaunchKernelEx(&cfg, kernel, a);
 }
 
-inline int reduce_threads(const ReduceArgs& a, int sg) {
+// tiles one CTA of the reduce kernel covers, for the shape that launch_reduce_shape picks
+inline unsigned reduce_tiles_per_cta(const ReduceArgs& a, int sg, bool f32) {
   const bool static_k = sg >= 0 && (a.K == 1 || a.K == 2 || a.K == 4 || a.K == 8);
-  return !static_k ? kAnyThreads : (sg == 0 ? kFlatThreads : kLevelThreads);
+  if (!static_k) return kAnyThreads / kThreads;
+  if (a.K <= 2) return (kFewThreads / kThreads) * ((f32 ? 4u : 8u) / a.K);
+  return (sg == 0 ? kFlatThreads : kLevelThreads) / kThreads;
 }
 
 template <bool F32, int KT, int SG>
 void launch_reduce_shape(const ReduceArgs& a, unsigned grid, cudaStream_t st, bool ov) {
   if constexpr (KT == 0)
-    launch_k(fls_reduce_kernel<F32, KT, SG, kAnyThreads, kAnyMinB>, a, grid, kAnyThreads, st, ov);
+    launch_k(fls_reduce_kernel<F32, KT, SG, kAnyThreads, kAnyMinB, 1>, a, grid, kAnyThreads, st, ov);
+  else if constexpr (KT <= 2)
+    launch_k(fls_reduce_kernel<F32, KT, SG, kFewThreads, kFewMinB, tiles_per_thread<F32, KT>()>, a, grid, kFewThreads, st, ov);
   else if constexpr (SG == 0)
-    launch_k(fls_reduce_kernel<F32, KT, SG, kFlatThreads, kFlatMinB>, a, grid, kFlatThreads, st, ov);
+    launch_k(fls_reduce_kernel<F32, KT, SG, kFlatThreads, kFlatMinB, 1>, a, grid, kFlatThreads, st, ov);
   else
-    launch_k(fls_reduce_kernel<F32, KT, SG, kLevelThreads, kLevelMinB>, a, grid, kLevelThreads, st, ov);
+    launch_k(fls_reduce_kernel<F32, KT, SG, kLevelThreads, kLevelMinB, 1>, a, grid, kLevelThreads, st, ov);
 }
 
 template <bool F32, int KT>
@@ -786,8 +898,8 @@ void launch_reduce_t(const ReduceArgs& a, int sg, unsigned grid, cudaStream_t st
 
 }  // namespace
 
-unsigned reduce_grid(const ReduceArgs& a, int sg) {
-  const unsigned tiles_per_cta = reduce_threads(a, sg) / kThreads;
+unsigned reduce_grid(const ReduceArgs& a, int sg, bool f32) {
+  const unsigned tiles_per_cta = reduce_tiles_per_cta(a, sg, f32);
   return (a.idx.n_tiles + tiles_per_cta - 1) / tiles_per_cta;
 }
 
@@ -797,7 +909,7 @@ cudaError_t launch_reduce_staged(const ReduceArgs& a, cudaStream_t st, bool over
 }
 
 cudaError_t launch_reduce(const ReduceArgs& a, bool f32, int sg, cudaStream_t st, bool overlap) {
-  const unsigned grid = reduce_grid(a, sg);
+  const unsigned grid = reduce_grid(a, sg, f32);
   if (f32)
     launch_reduce_t<true>(a, sg, grid, st, overlap);
   else

@@ -81,7 +81,7 @@ struct FusedArgs {
 // sg: level structure of the reduction (see reduce_elems): 0, 1, 2, 4 or -1 for the generic form;
 // -2: the generic form with every partial sum and the mean rounded to bf16 (bf16 gradients only).
 // The reduce kernel has one launch shape; reduce_grid() is its grid (= number of norm partials it writes).
-unsigned reduce_grid(const ReduceArgs& a, int sg);
+unsigned reduce_grid(const ReduceArgs& a, int sg, bool f32);
 // overlap: launch with programmatic stream serialization, so that the kernel's first CTAs may start during
 // the tail of the kernel launched just before it on the same stream (which must be one of these three).
 cudaError_t launch_reduce(const ReduceArgs& a, bool f32, int sg, cudaStream_t st, bool overlap);
