@@ -4,6 +4,7 @@ gate on m and v, whose magnitudes make the absolute gate weak); the bf16 copy wi
 the fp32 tolerance where a bf16 ulp is smaller than it) and bit-exactly the rounding of the GPU's own
 fp32 master."""
 import math
+import os
 
 import numpy as np
 import pytest
@@ -571,5 +572,71 @@ def test_full_size_workloads_sampled(fls, cfg_index):
         assert_state_close(s.master[g][at].cpu().numpy(), states[g].theta, f"fedavg master[{g}]")
         assert_bf16_close(bf16_bits(s.param_bf16[g][jt]), states[g].param_bf16, f"fedavg bf16[{g}]")
     assert torch.equal(s.master[0], s.master[G - 1]) and torch.equal(s.param_bf16[0], s.param_bf16[G - 1])
+    assert s.status() == 0
+    s.close()
+
+
+def _fill_grads_full_size(s, cfg, L, step):
+    starts = np.concatenate([[0], np.cumsum(L.unit_numel)])
+    for g in range(cfg["groups"]):
+        for u, n in enumerate(L.unit_numel):
+            for k in range(s.K):
+                scale = sy.uniform_scale(cfg["seed"], g, k) if cfg["per_buffer_scale"] else 1.0
+                sy.normal_fill_(s.grads[g][k][L.unit_offset[u]:L.unit_offset[u] + n], sy.stream_key(cfg["seed"], sy.KIND_GRAD, step, g, k),
+                                cfg["grad_sigma"], scale, start=int(starts[u]))
+    torch.cuda.synchronize()
+
+
+@pytest.mark.skipif(not os.environ.get("FLS_LONG_TESTS"), reason="full schedules take minutes; set FLS_LONG_TESTS=1")
+@pytest.mark.parametrize("cfg_index", [1, 2, 3])
+def test_full_schedule_sampled(fls, cfg_index):
+    """The whole schedule of a workload at full size (32 / 8 / 16 steps, fresh gradients every step, FedAvg every
+    H steps through the fused call): the oracle follows 100,000 sampled parameters with norms computed over the
+    full gradients of every group and step; state compared after every aggregation and at the end."""
+    from paper_2609_20359_b200.session import Session
+    cfg = sy.CONFIGS[cfg_index]
+    P, G, S, R_rep, H = cfg["n_params"], cfg["groups"], cfg["shard_dim"], cfg["replicate_dim"], cfg["sync_period"]
+    K = S * R_rep
+    hp = orc.Hyper()
+    L = orc.plan(cfg["unit_numel"], S, 8)
+    s = Session(P, cfg["unit_numel"], G, S, R_rep, H, "bf16", 8, False, fused=True)
+    _fill_full_size(s, cfg, L)
+    counts = [sy.sample_count(cfg["seed"], g) for g in range(G)] if cfg["weights"] == "counts" else None
+    idx = np.unique(np.random.default_rng(5).integers(0, P, 100_000))
+    tidx = torch.from_numpy(idx)
+    j_np, a_np = orc.addresses_of(L, idx)
+    jt, at = torch.from_numpy(j_np).cuda(), torch.from_numpy(a_np).cuda()
+    th0 = sy.normal_at(tidx, sy.stream_key(cfg["seed"], sy.KIND_MASTER), cfg["master_sigma"]).numpy()
+    z = np.zeros(idx.size, np.float32)
+    states = [orc.GroupState(th0.copy(), z.copy(), z.copy(), orc.f32_to_bf16_bits(th0)) for _ in range(G)]
+    worst = 0.0
+    for t in range(1, cfg["steps"] + 1):
+        _fill_grads_full_size(s, cfg, L, t)
+        norms = [_oracle_norm_full(s.grads[g], S, R_rep) for g in range(G)]
+        for g in range(G):
+            samp = [orc.bf16_bits_to_f64(bf16_bits(sy.normal_at(tidx, sy.stream_key(cfg["seed"], sy.KIND_GRAD, t, g, k), cfg["grad_sigma"],
+                                                                 sy.uniform_scale(cfg["seed"], g, k) if cfg["per_buffer_scale"] else 1.0,
+                                                                 torch.bfloat16))) for k in range(K)]
+            gb = orc.reduce_mean(samp, S, R_rep)
+            st = states[g]
+            st.theta, st.m, st.v, st.param_bf16 = orc.adamw(st.theta, st.m, st.v, gb, orc.clip_coef(norms[g], hp.max_grad_norm), t,
+                                                           hp.lr, hp.beta1, hp.beta2, hp.eps, hp.weight_decay)
+        if t % H == 0:
+            orc.fedavg(states, counts)
+            s.step_fedavg(counts)
+        else:
+            assert not s.step()
+        torch.cuda.synchronize()
+        got_n = s.norms().cpu().numpy().astype(np.float64)
+        assert np.allclose(got_n, norms, rtol=1e-6, atol=0), (t, got_n, norms)
+        if t % H == 0 or t == cfg["steps"]:
+            for g in range(G):
+                th = s.master[g][at].cpu().numpy()
+                worst = max(worst, float(np.max(np.abs(th.astype(np.float64) - states[g].theta))))
+                assert_state_close(th, states[g].theta, f"step {t} master[{g}]")
+                assert_state_close(s.m[g][at].cpu().numpy(), states[g].m, f"step {t} m[{g}]", 1e-5, "rms")
+                assert_state_close(s.v[g][at].cpu().numpy(), states[g].v, f"step {t} v[{g}]", 1e-5, "rms")
+                assert_bf16_close(bf16_bits(s.param_bf16[g][jt]), states[g].param_bf16, f"step {t} bf16[{g}]")
+    print(f"full schedule {cfg['name']}: {cfg['steps']} steps, worst |dtheta| on the sample = {worst:.3e}")
     assert s.status() == 0
     s.close()
