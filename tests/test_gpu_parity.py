@@ -393,6 +393,26 @@ def test_nonfinite_gradients_propagate_and_set_status(fls):
     c.close()
 
 
+def test_non_default_stream(fls):
+    """Everything enqueued on a side stream (overlapped launches, fused aggregation, host-gradient step): same
+    results as the oracle; the library never touches another stream's work."""
+    side = torch.cuda.Stream()
+    c = Case([50000, 1234, 4096], 3, 4, 2, H=2, Q=8, opt_state=True, hp=orc.Hyper(max_grad_norm=0.05), fused=True)
+    torch.cuda.synchronize()
+    with torch.cuda.stream(side):
+        for _ in range(4):
+            c.step([3, 5, 1])
+            c.compare()
+        host = [[c.sess.grads[g][k].cpu().pin_memory() for k in range(c.K)] for g in range(c.G)]
+        before = [x.clone() for x in c.sess.master]
+        norms = torch.zeros(c.G, dtype=torch.float32)
+        c.sess.step_host(host, host_norms=norms)            # step 5 on the same gradients, fed from the host
+        side.synchronize()
+        assert torch.equal(norms, c.sess.norms().cpu())
+        assert all(not torch.equal(a, b) for a, b in zip(before, c.sess.master))
+    c.close()
+
+
 def test_step_from_host_buffers_matches_device_step(fls):
     a = Case([50000, 777], 2, 2, 2, H=2, Q=8, hp=orc.Hyper(max_grad_norm=0.02))
     b = Case([50000, 777], 2, 2, 2, H=2, Q=8, hp=orc.Hyper(max_grad_norm=0.02))
