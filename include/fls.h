@@ -166,6 +166,20 @@ int fls_sync_step_host(fls_plan* plan, const void* const* host_grads, double lr,
  * Errors: FLS_EINVAL if all counts are zero, FLS_ESTATE, FLS_ECUDA. */
 int fls_fedavg(fls_plan* plan, const uint64_t* sample_counts, void* cuda_stream);
 
+/* Aggregation with an outer optimizer (the FedOpt family of the paper's related work: AdamW inside the groups,
+ * SGD with optional Nesterov momentum across them; "FedAvg as a base aggregation strategy, enabling easy
+ * integration of more complex ones").  With xbar = sum_g w_g x_g as in fls_fedavg:
+ *   delta = x_global - xbar;  buf = momentum*buf + delta;  d = nesterov ? delta + momentum*buf : buf;
+ *   x_global -= outer_lr * d;  every group's master = x_global, every bf16 copy = bf16(x_global).
+ * outer_lr = 1, momentum = 0 is plain FedAvg (up to fp32 rounding of x - (x - xbar)).  global_params and
+ * outer_momentum: device, N_pad floats each, shard order, FLS_BUFFER_ALIGN-aligned, caller-owned, in/out (start
+ * them as a copy of the initial parameters and as zeros).  m and v are averaged as in fls_fedavg when the plan has
+ * FLS_AVG_OPT_STATE.  fp32 arithmetic, fma accumulation of xbar in ascending g.
+ * Errors: FLS_EPTR / FLS_EALIGN for the two buffers, FLS_EINVAL (non-finite outer_lr or momentum, all counts zero),
+ * FLS_ESTATE, FLS_ECUDA. */
+int fls_fedavg_outer(fls_plan* plan, const uint64_t* sample_counts, double outer_lr, double momentum, int nesterov,
+                     float* global_params, float* outer_momentum, void* cuda_stream);
+
 /* One local step of all groups immediately followed by FedAvg, i.e. exactly fls_sync_step then fls_fedavg
  * (same results bit for bit), for the steps on which aggregation is due ("after the local update every A
  * training steps").  With FLS_AVG_FUSED in the plan and G <= FLS_MAX_FUSED_GROUPS the aggregation is fused

@@ -293,6 +293,30 @@ def fedavg(states: Sequence[GroupState], sample_counts: Optional[Sequence[int]] 
             s.m = m.copy(); s.v = v.copy()
 
 
+def fedavg_outer(states: Sequence[GroupState], x_global: np.ndarray, buf: np.ndarray, sample_counts=None,
+                 outer_lr: float = 1.0, momentum: float = 0.0, nesterov: bool = False):
+    """Aggregation with an outer optimizer (the FedOpt family the paper's related work describes: AdamW inside
+    the groups, SGD with (Nesterov) momentum outside; plain FedAvg is the case outer_lr = 1, momentum = 0).
+    The weighted average of the groups is turned into a pseudo-gradient against the global copy:
+        xbar = sum_g w_g x_g ;  delta = x_global - xbar ;  buf = momentum*buf + delta
+        d = delta + momentum*buf  (Nesterov)  or  buf ;  x_global = x_global - outer_lr*d
+    and every group restarts from x_global.  Double arithmetic, fp32 stores.  Returns (x_global, buf)."""
+    G = len(states)
+    w = fedavg_weights(sample_counts, G)
+    xbar = np.zeros(np.asarray(x_global).shape, np.float64)
+    for g, st in enumerate(states):
+        xbar = xbar + w[g] * np.asarray(st.theta, dtype=np.float32).astype(np.float64)
+    xg = np.asarray(x_global, dtype=np.float32).astype(np.float64)
+    delta = xg - xbar
+    b = momentum * np.asarray(buf, dtype=np.float32).astype(np.float64) + delta
+    d = delta + momentum * b if nesterov else b
+    xg = (xg - outer_lr * d).astype(np.float32)
+    bits = f32_to_bf16_bits(xg)
+    for st in states:
+        st.theta = xg.copy(); st.param_bf16 = bits.copy()
+    return xg, b.astype(np.float32)
+
+
 # --------------------------------------------------------------------------- driver loop
 def run(states: List[GroupState], grads_for_step, S: int, R_rep: int, H: int, n_steps: int, hp: Hyper,
         sample_counts=None, opt_state: bool = False, t0: int = 0):

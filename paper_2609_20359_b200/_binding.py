@@ -24,7 +24,7 @@ FLS_NOALLOC_MAX_ELEMS = 1 << 29
 
 EXPORTS = [
     "fls_plan_create", "fls_plan_query", "fls_plan_bind", "fls_sync_step", "fls_sync_step_host", "fls_fedavg",
-    "fls_sync_step_fedavg",
+    "fls_sync_step_fedavg", "fls_fedavg_outer",
     "fls_get_norms", "fls_get_reduced_grad", "fls_get_status", "fls_get_step", "fls_set_step", "fls_comm_report",
     "fls_plan_tune", "fls_plan_set_staging", "fls_plan_set_recompute", "fls_plan_set_overlap", "fls_set_profiling", "fls_get_kernel_ms", "fls_get_launch_count", "fls_plan_destroy",
     "fls_last_error", "fls_reduce_norm_noalloc",
@@ -84,6 +84,7 @@ def _load() -> C.CDLL:
     lib.fls_sync_step_host.argtypes = [P, C.POINTER(C.c_void_p), C.c_double, P, C.POINTER(C.c_float), C.POINTER(C.c_int)]
     lib.fls_fedavg.argtypes = [P, C.POINTER(C.c_uint64), P]
     lib.fls_sync_step_fedavg.argtypes = [P, C.c_double, C.POINTER(C.c_uint64), P]
+    lib.fls_fedavg_outer.argtypes = [P, C.POINTER(C.c_uint64), C.c_double, C.c_double, C.c_int, P, P, P]
     lib.fls_get_norms.argtypes = [P, C.POINTER(P), C.POINTER(P)]
     lib.fls_get_reduced_grad.argtypes = [P, C.POINTER(P)]
     lib.fls_get_status.argtypes = [P, C.POINTER(P)]
@@ -191,6 +192,15 @@ def fls_sync_step_host(plan: int, host_grads: Sequence, lr: float = math.nan, st
 def fls_fedavg(plan: int, sample_counts: Optional[Sequence[int]] = None, stream=None) -> None:
     arr = (C.c_uint64 * len(sample_counts))(*sample_counts) if sample_counts is not None else None
     _check(lib.fls_fedavg(plan, arr, _stream_handle(stream)))
+
+
+def fls_fedavg_outer(plan: int, sample_counts: Optional[Sequence[int]], outer_lr: float, momentum: float, nesterov: bool,
+                     global_params, outer_momentum, stream=None) -> None:
+    """FedAvg followed by an SGD(+momentum/Nesterov) step on the global copy; global_params and outer_momentum
+    are float32 device tensors of N_pad elements in shard order, updated in place."""
+    arr = (C.c_uint64 * len(sample_counts))(*sample_counts) if sample_counts is not None else None
+    _check(lib.fls_fedavg_outer(plan, arr, outer_lr, momentum, int(nesterov), _ptr(global_params), _ptr(outer_momentum),
+                                _stream_handle(stream)))
 
 
 def fls_sync_step_fedavg(plan: int, lr: float = math.nan, sample_counts: Optional[Sequence[int]] = None, stream=None) -> None:

@@ -462,13 +462,14 @@ int fls_sync_step_host(fls_plan* p, const void* const* host_grads, double lr, vo
   return FLS_OK;
 }
 
-int fls_fedavg(fls_plan* p, const uint64_t* sample_counts, void* cuda_stream) {
-  if (!p) return fail(FLS_EINVAL, "fls_fedavg: null plan");
-  if (!p->bound) return fail(FLS_ESTATE, "fls_fedavg: plan has no buffers bound");
+namespace {
+struct OuterOpt { float* x_global; float* buf; double lr, momentum; int nesterov; };
+
+int fedavg_impl(fls_plan* p, const uint64_t* sample_counts, void* cuda_stream, const OuterOpt* outer, const char* who) {
   const uint32_t G = p->desc.groups;
   long double total = 0;
   for (uint32_t g = 0; g < G; ++g) total += sample_counts ? (long double)sample_counts[g] : 1.0L;
-  if (!(total > 0)) return fail(FLS_EINVAL, "fls_fedavg: all sample counts are zero");
+  if (!(total > 0)) return fail(FLS_EINVAL, "%s: all sample counts are zero", who);
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   FedavgArgs fa{};
   for (uint32_t g = 0; g < G; ++g) {
@@ -485,11 +486,37 @@ int fls_fedavg(fls_plan* p, const uint64_t* sample_counts, void* cuda_stream) {
       fa.pbf16[g] = p->pbf16[g];
     }
     fa.write_bf16 = arr == 0 ? 1 : 0;
+    const bool use_outer = outer && arr == 0;       // the outer optimizer acts on the parameters only
+    fa.x_global = use_outer ? outer->x_global : nullptr;
+    fa.outer_buf = use_outer ? outer->buf : nullptr;
+    fa.outer_lr = use_outer ? float(outer->lr) : 0.f;
+    fa.momentum = use_outer ? float(outer->momentum) : 0.f;
+    fa.nesterov = use_outer ? outer->nesterov : 0;
     const bool overlap = p->overlap && !p->profiling && arr > 0;
     cudaError_t e = timed_launch(p, FLS_KERNEL_FEDAVG, st, [&] { return launch_fedavg(fa, p->grid_for(FLS_KERNEL_FEDAVG), st, overlap); });
     if (e != cudaSuccess) return cuda_fail(e, "fedavg kernel launch");
   }
   return FLS_OK;
+}
+}  // namespace
+
+int fls_fedavg(fls_plan* p, const uint64_t* sample_counts, void* cuda_stream) {
+  if (!p) return fail(FLS_EINVAL, "fls_fedavg: null plan");
+  if (!p->bound) return fail(FLS_ESTATE, "fls_fedavg: plan has no buffers bound");
+  return fedavg_impl(p, sample_counts, cuda_stream, nullptr, "fls_fedavg");
+}
+
+int fls_fedavg_outer(fls_plan* p, const uint64_t* sample_counts, double outer_lr, double momentum, int nesterov,
+                     float* global_params, float* outer_momentum, void* cuda_stream) {
+  if (!p) return fail(FLS_EINVAL, "fls_fedavg_outer: null plan");
+  if (!p->bound) return fail(FLS_ESTATE, "fls_fedavg_outer: plan has no buffers bound");
+  if (!global_params || !outer_momentum) return fail(FLS_EPTR, "fls_fedavg_outer: null buffer");
+  if (reinterpret_cast<uintptr_t>(global_params) % FLS_BUFFER_ALIGN || reinterpret_cast<uintptr_t>(outer_momentum) % FLS_BUFFER_ALIGN)
+    return fail(FLS_EALIGN, "fls_fedavg_outer: buffers must be %d-byte aligned", FLS_BUFFER_ALIGN);
+  if (global_params == outer_momentum) return fail(FLS_EPTR, "fls_fedavg_outer: the two buffers are the same");
+  if (!std::isfinite(outer_lr) || !std::isfinite(momentum)) return fail(FLS_EINVAL, "fls_fedavg_outer: outer_lr and momentum must be finite");
+  const OuterOpt o{global_params, outer_momentum, outer_lr, momentum, nesterov ? 1 : 0};
+  return fedavg_impl(p, sample_counts, cuda_stream, &o, "fls_fedavg_outer");
 }
 
 int fls_sync_step_fedavg(fls_plan* p, double lr, const uint64_t* sample_counts, void* cuda_stream) {

@@ -671,10 +671,25 @@ __global__ void __launch_bounds__(kThreads, KT == 0 ? 2 : 3) fls_reduce_adamw_ke
 // K3: FedAvg.  x_bar = sum_g w_g x_g, ascending g from zero, written to all G copies.
 // GT = G for G in {1, 2, 4, 8} (unrolled, pointers straight from the kernel parameters), else 0.
 // ------------------------------------------------------------------------------------------------
+// Outer optimizer on one element: xbar becomes the new global value.  delta = x_global - xbar,
+// buf = momentum*buf + delta, d = delta + momentum*buf (Nesterov) or buf, x_global -= outer_lr*d.
+__device__ __forceinline__ float outer_step(const FedavgArgs& a, float xbar, float xg, float& buf) {
+  const float delta = xg - xbar;
+  buf = fmaf(a.momentum, buf, delta);
+  const float d = a.nesterov ? fmaf(a.momentum, buf, delta) : buf;
+  return fmaf(-a.outer_lr, d, xg);
+}
+
 __device__ __noinline__ void fedavg_slice_scalar(const FedavgArgs& a, uint64_t j, uint64_t addr, uint32_t n) {
   for (uint32_t e = 0; e < n; ++e) {
     float acc = 0.f;
     for (uint32_t g = 0; g < a.G; ++g) acc = fmaf(a.w[g], a.x[g][addr + e], acc);
+    if (a.x_global) {
+      float b = a.outer_buf[addr + e];
+      acc = outer_step(a, acc, a.x_global[addr + e], b);
+      a.x_global[addr + e] = acc;
+      a.outer_buf[addr + e] = b;
+    }
     for (uint32_t g = 0; g < a.G; ++g) a.x[g][addr + e] = acc;
     if (a.write_bf16) {
       const uint16_t b = to_bf16_bits(acc);
@@ -714,6 +729,14 @@ __global__ void __launch_bounds__(kThreads, MINB) fls_fedavg_kernel(const __grid
             for (int e = 0; e < 8; ++e) acc.v[e] = fmaf(wg, raw[b].v[e], acc.v[e]);   // acc starts at 0: first term w_0 x_0
           }
         }
+      }
+      if (a.x_global) {
+        const F8 xg = ld8_stream(a.x_global + s.a);
+        F8 b = ld8_stream(a.outer_buf + s.a);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc.v[e] = outer_step(a, acc.v[e], xg.v[e], b.v[e]);
+        st8_stream(a.x_global + s.a, acc);
+        st8_stream(a.outer_buf + s.a, b);
       }
       if constexpr (GT != 0) {
 #pragma unroll

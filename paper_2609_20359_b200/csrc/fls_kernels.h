@@ -60,6 +60,11 @@ struct FedavgArgs {
   uint32_t G;
   int write_bf16;
   int descending;
+  // outer optimizer (both null: plain FedAvg)
+  float* x_global;                         // device, in/out
+  float* outer_buf;                        // device, in/out: momentum buffer
+  float outer_lr, momentum;
+  int nesterov;
 };
 
 // AdamW of all G groups + FedAvg of the results in one pass (G <= FLS_MAX_FUSED_GROUPS).

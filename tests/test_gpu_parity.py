@@ -296,6 +296,39 @@ def test_fused_step_fedavg_matches_oracle_and_unfused(fls, units, G, S, R_rep, Q
     assert all(torch.equal(x, y) for x, y in zip(*outs))
 
 
+@pytest.mark.parametrize("G,nesterov,opt_state,units,Q", [(4, True, False, [30000, 517], 8), (3, False, True, [70001], 1), (9, True, False, [999], 8)])
+def test_fedavg_outer_optimizer(fls, G, nesterov, opt_state, units, Q):
+    """Aggregation through an outer SGD step with momentum on a global copy, three rounds, against the oracle."""
+    c = Case(units, G, 2, 1, H=1, Q=Q, opt_state=opt_state, hp=orc.Hyper(max_grad_norm=0.01))
+    counts = [sy.sample_count(31, g) for g in range(G)]
+    xg = c.states[0].theta.copy()
+    buf = np.zeros_like(xg)
+    d_xg = c.sess.master[0].clone()
+    d_buf = torch.zeros_like(d_xg)
+    for r in range(3):
+        c.step(counts, fedavg=False)
+        xg, buf = orc.fedavg_outer(c.states, xg, buf, counts, outer_lr=0.7, momentum=0.9, nesterov=nesterov)
+        if opt_state:       # m and v are averaged as in plain FedAvg
+            w = orc.fedavg_weights(counts, G)
+            mbar = orc.fedavg_array([st.m for st in c.states], w); vbar = orc.fedavg_array([st.v for st in c.states], w)
+            for st in c.states:
+                st.m = mbar.copy(); st.v = vbar.copy()
+        fls.fls_fedavg_outer(c.sess.plan, counts, 0.7, 0.9, nesterov, d_xg, d_buf)
+        c.compare(check_norms=False)
+        assert_state_close(d_xg.cpu().numpy(), orc.pack_sharded(c.L, xg), "x_global")
+        # the buffer accumulates x_global - xbar, a difference of nearly equal fp32 numbers: its error is a few
+        # ulps of the parameters' magnitude (0.02 -> 2e-9), whatever the size of the difference itself
+        assert np.allclose(d_buf.cpu().numpy(), orc.pack_sharded(c.L, buf), rtol=1e-5, atol=3e-8)
+        assert torch.equal(c.sess.master[G - 1], d_xg)
+    with pytest.raises(fls.FlsError) as e:
+        fls.fls_fedavg_outer(c.sess.plan, counts, float("nan"), 0.9, True, d_xg, d_buf)
+    assert e.value.code == fls.FLS_EINVAL
+    with pytest.raises(fls.FlsError) as e:
+        fls.fls_fedavg_outer(c.sess.plan, counts, 0.7, 0.9, True, d_xg, d_xg)
+    assert e.value.code == fls.FLS_EPTR
+    c.close()
+
+
 def test_fedavg_g1_is_bit_exact_identity_and_idempotent(fls):
     c = Case([5000], 1, 2, 1, H=1, Q=8, opt_state=True)
     c.step(fedavg=False)

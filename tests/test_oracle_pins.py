@@ -357,6 +357,37 @@ def test_fedavg_identity_cases():
     assert np.allclose(s1[0].theta, s2[0].theta, rtol=2e-7, atol=0)
 
 
+def test_fedavg_outer_special_case_and_torch_sgd():
+    """Outer optimizer: lr 1 / momentum 0 is plain FedAvg; in general it is torch.optim.SGD (momentum, Nesterov)
+    on the pseudo-gradient x_global - xbar, followed over several rounds."""
+    rng = np.random.default_rng(23)
+    n, G = 3000, 4
+    counts = [int(c) for c in rng.integers(1, 1001, G)]
+    xg0 = rng.normal(0, 0.02, n).astype(np.float32)
+    def groups(r):
+        return [orc.GroupState((xg0 + rng.normal(0, 1e-3, n)).astype(np.float32), None, None, None) for _ in range(G)]
+    # special case
+    sts = groups(0)
+    plain = [orc.GroupState(s.theta.copy(), None, None, None) for s in sts]
+    orc.fedavg(plain, counts)
+    xg, buf = orc.fedavg_outer(sts, xg0, np.zeros(n, np.float32), counts, outer_lr=1.0, momentum=0.0)
+    assert np.allclose(xg, plain[0].theta, rtol=0, atol=4e-9) and all(np.array_equal(s.theta, xg) for s in sts)
+    # against the library optimizer, three rounds
+    for nesterov in (False, True):
+        p = torch.nn.Parameter(torch.from_numpy(xg0.astype(np.float64)))
+        opt = torch.optim.SGD([p], lr=0.7, momentum=0.9, nesterov=nesterov)
+        xg, buf = xg0.copy(), np.zeros(n, np.float32)
+        for r in range(3):
+            sts = [orc.GroupState((xg + rng.normal(0, 1e-3, n)).astype(np.float32), None, None, None) for _ in range(G)]
+            w = np.asarray(counts, np.float64) / sum(counts)
+            xbar = sum(w[g] * sts[g].theta.astype(np.float64) for g in range(G))
+            p.grad = p.detach() - torch.from_numpy(xbar)
+            opt.step()
+            xg, buf = orc.fedavg_outer(sts, xg, buf, counts, outer_lr=0.7, momentum=0.9, nesterov=nesterov)
+            assert np.allclose(xg, p.detach().numpy(), rtol=0, atol=2e-8 * (r + 1))
+            assert np.array_equal(sts[2].param_bf16, orc.f32_to_bf16_bits(xg))
+
+
 # ----------------------------------------------------------------------------- whole loop
 def _make_states(rng, G, n):
     th = rng.normal(0, 0.02, n).astype(np.float32)
