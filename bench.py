@@ -301,9 +301,13 @@ def run_ours(args, cfg):
         sampler.start()
     ms_total, launches = timed(args.steps, False, sampler if rank == 0 else None)
     fedavg_calls = n_fedavg[0]
-    clocks = sampler.stop() if rank == 0 else None
+    in_region = len(sampler.sm)
     # second pass over the same number of steps with events around every kernel: per-kernel durations
-    ms_prof, _ = timed(args.steps, True)
+    # (the clocks keep being sampled: an NVML reading can take as long as a short timed region)
+    ms_prof, _ = timed(args.steps, True, sampler if rank == 0 else None)
+    clocks = sampler.stop() if rank == 0 else None
+    if clocks is not None:
+        clocks["samples_in_timed_region"] = in_region
     kms, kn = fls.fls_get_kernel_ms(sess.plan)
     fls.fls_set_profiling(sess.plan, False)
 
