@@ -54,6 +54,21 @@ def test_planner_matches_oracle(fls, units, S, Q):
     fls.fls_plan_destroy(p)
 
 
+def test_planner_matches_oracle_on_random_unit_tables(fls):
+    rng = np.random.default_rng(99)
+    for _ in range(300):
+        units = [int(x) for x in rng.integers(1, 10 ** int(rng.integers(1, 8)), int(rng.integers(1, 40)))]
+        S, Q = int(rng.integers(1, 17)), int(rng.choice([1, 2, 3, 8, 16, 64]))
+        p = fls.fls_plan_create(sum(units), units, groups=int(rng.integers(1, 5)), shard_dim=S, align_elems=Q)
+        lay = fls.fls_plan_query(p)
+        L = orc.plan(units, S, Q)
+        assert (lay["n_padded"], lay["shard_numel"]) == (L.n_padded, L.shard_numel)
+        assert lay["unit_offset"] == L.unit_offset and lay["unit_shard_numel"] == L.unit_shard_numel
+        assert lay["unit_shard_offset"] == L.unit_shard_offset
+        assert lay["vector_path"] == all(m % 8 == 0 for m in L.unit_shard_numel) or len(units) == 1 or S == 1
+        fls.fls_plan_destroy(p)
+
+
 def test_single_unit_default_table(fls):
     p = fls.fls_plan_create(1000, None, groups=1, shard_dim=4, align_elems=8)
     lay = fls.fls_plan_query(p)
