@@ -347,7 +347,10 @@ def run_ours(args, cfg):
         # written), m and v 8 B each; the figure is the mean over the launches of one call
         per_launch = {"reduce": N * (sess.K * eg + 4), "adamw": N * 30, "fedavg": N * G * (26 / 3 if args.opt_state else 10),
                       "adamw_fedavg": N * G * 30}
-        if sess.K * eg < 8:
+        if not cfg["max_grad_norm"] > 0:
+            # no clipping: one kernel per group does the whole step (timed under "adamw")
+            per_launch.update(adamw=N * (sess.K * eg + 26))
+        elif sess.K * eg < 8:
             # small K: nothing is stored by the norm pass and AdamW reads the gradients again
             per_launch.update(reduce=N * sess.K * eg, adamw=N * (sess.K * eg + 26))
         kernels = {}
@@ -500,6 +503,7 @@ def main():
     ap.add_argument("--replicate-dim", type=int, default=0, help="override R_rep")
     ap.add_argument("--grad-dtype", default="", choices=["", "bf16", "f32"], help="override the gradient dtype")
     ap.add_argument("--keep-units", action="store_true", help="with --n-params: keep the unit table's proportions")
+    ap.add_argument("--clip", type=float, default=None, help="override max_grad_norm (0 disables clipping: single-pass step)")
     ap.add_argument("--sweep", action="store_true", help="run the bandwidth sweep instead of the benchmark")
     ap.add_argument("--sweep-out", default="sweep_results.jsonl")
     ap.add_argument("--sweep-exps", default="20,22,24,26,28,30", help="log2 of the parameter counts to sweep")
@@ -519,6 +523,8 @@ def main():
         cfg.update(shard_dim=args.shard_dim, name=cfg["name"] + f"[S={args.shard_dim}]")
     if args.replicate_dim:
         cfg.update(replicate_dim=args.replicate_dim, name=cfg["name"] + f"[R={args.replicate_dim}]")
+    if args.clip is not None:
+        cfg.update(max_grad_norm=args.clip, name=cfg["name"] + f"[clip={args.clip}]")
     if args.grad_dtype:
         cfg.update(grad_dtype=args.grad_dtype, name=cfg["name"] + f"[{args.grad_dtype}]")
     if args.impl == "reference":

@@ -120,7 +120,8 @@ typedef struct {
                             unit (S*M_u), the convention of the NCCL performance notes the paper cites        */
   fls_cost5 seconds;     /* Eq. 1-5 with B_S, B_R, B_F; NaN when no bandwidths were given                     */
   double hbm_bytes_sync_step; /* bytes one fls_sync_step must move in this library: G*N_pad*(K*e_g + 34), or
-                                 G*N_pad*(2*K*e_g + 26) when K*e_g < 8 (gradients read twice, nothing stored)  */
+                                 G*N_pad*(2*K*e_g + 26) when K*e_g < 8 (gradients read twice, nothing stored),
+                                 or G*N_pad*(K*e_g + 26) without clipping (single pass)                        */
   double hbm_bytes_fedavg;    /* bytes one fls_fedavg must move: G*N_pad*10, or *26 with optimizer state      */
 } fls_comm_costs;
 
@@ -194,7 +195,8 @@ int fls_sync_step_fedavg(fls_plan* plan, double lr, const uint64_t* sample_count
 int fls_get_norms(const fls_plan* plan, const float** dev_norms, const float** dev_coefs);
 
 /* Device pointer to the reduced (mean) gradient of the LAST group processed: N_pad floats, shard order.
- * FLS_ESTATE if the last step stored none (plans with K*e_g < 8 bytes recompute it, see fls_plan_set_recompute). */
+ * FLS_ESTATE if the last step stored none (plans with K*e_g < 8 bytes recompute it, see fls_plan_set_recompute;
+ * plans without clipping run a single pass, see fls_plan_set_single_pass). */
 int fls_get_reduced_grad(const fls_plan* plan, const float** dev_gbar);
 
 /* Device pointer to the sticky status word (FLS_STATUS_* bits).  Non-finite values are not errors:
@@ -231,6 +233,13 @@ int fls_plan_set_staging(fls_plan* plan, int enabled);
  * that by default.  mode 0 forces store-and-reread, 1 forces recomputation (FLS_ESTATE if the plan does not
  * qualify), -1 restores the default.  The results are identical either way. */
 int fls_plan_set_recompute(fls_plan* plan, int mode);
+
+/* Plans without clipping (max_grad_norm <= 0) need no second pass: the clip coefficient is 1 before the norm is
+ * known, so by default one kernel per group reduces the gradients, applies AdamW and accumulates the norm (which
+ * is still reported): K*e_g + 26 bytes per element.  mode 0 forces the two-pass route, 1 forces the single pass
+ * (FLS_ESTATE if the plan clips or uses FLS_WIRE_BF16), -1 restores the default.  master, m, v and the bf16 copy
+ * are identical either way; after a single-pass step fls_get_reduced_grad has nothing to offer (FLS_ESTATE). */
+int fls_plan_set_single_pass(fls_plan* plan, int mode);
 
 /* enabled != 0 (the default): inside one call every kernel but the first is launched so that its first CTAs may
  * start during the tail of the kernel before it (programmatic dependent launch); they fetch what that kernel does

@@ -26,7 +26,7 @@ EXPORTS = [
     "fls_plan_create", "fls_plan_query", "fls_plan_bind", "fls_sync_step", "fls_sync_step_host", "fls_fedavg",
     "fls_sync_step_fedavg", "fls_fedavg_outer",
     "fls_get_norms", "fls_get_reduced_grad", "fls_get_status", "fls_get_step", "fls_set_step", "fls_comm_report",
-    "fls_plan_tune", "fls_plan_set_staging", "fls_plan_set_recompute", "fls_plan_set_overlap", "fls_set_profiling", "fls_get_kernel_ms", "fls_get_launch_count", "fls_plan_destroy",
+    "fls_plan_tune", "fls_plan_set_staging", "fls_plan_set_recompute", "fls_plan_set_single_pass", "fls_plan_set_overlap", "fls_set_profiling", "fls_get_kernel_ms", "fls_get_launch_count", "fls_plan_destroy",
     "fls_last_error", "fls_reduce_norm_noalloc",
 ]
 
@@ -94,6 +94,7 @@ def _load() -> C.CDLL:
     lib.fls_plan_tune.argtypes = [P, C.c_uint32, C.c_int, C.c_int]
     lib.fls_plan_set_staging.argtypes = [P, C.c_int]
     lib.fls_plan_set_recompute.argtypes = [P, C.c_int]
+    lib.fls_plan_set_single_pass.argtypes = [P, C.c_int]
     lib.fls_plan_set_overlap.argtypes = [P, C.c_int]
     lib.fls_set_profiling.argtypes = [P, C.c_int]
     lib.fls_get_kernel_ms.argtypes = [P, C.POINTER(C.c_double), C.POINTER(C.c_uint64)]
@@ -256,6 +257,10 @@ def fls_plan_set_staging(plan: int, enabled: bool) -> None:
 
 def fls_plan_set_recompute(plan: int, mode: int) -> None:
     _check(lib.fls_plan_set_recompute(plan, mode))
+
+
+def fls_plan_set_single_pass(plan: int, mode: int) -> None:
+    _check(lib.fls_plan_set_single_pass(plan, mode))
 
 
 def fls_plan_set_overlap(plan: int, enabled: bool) -> None:

@@ -65,6 +65,7 @@ struct fls_plan {
   bool overlap = true;     // programmatic dependent launch between the kernels of one call
   bool staged_reduce = false;
   bool recompute = false;  // K * e_g < 8: the norm pass stores nothing and AdamW forms the mean gradient again
+  bool single_pass = false;  // no clipping: reduce + norm + AdamW in one kernel
   bool profiling = false;
   std::vector<TimedLaunch> timed;
   std::vector<cudaEvent_t> event_pool;
@@ -185,11 +186,28 @@ int run_group(fls_plan* p, uint32_t g, double lr, uint64_t t_new, cudaStream_t s
   ra.normsq_out = p->d_normsq() + g;
   ra.status = p->d_status();
   ra.max_grad_norm = d.max_grad_norm;
-  const bool recompute = p->recompute && with_adamw;   // the fused aggregation needs the stored gradients
-  ra.store_gbar = recompute ? 0 : 1;
-  p->gbar_valid = !recompute;
+  const bool single = p->single_pass && with_adamw;
+  const bool recompute = p->recompute && with_adamw && !single;   // the fused aggregation needs the stored gradients
+  ra.store_gbar = (recompute || single) ? 0 : 1;
+  p->gbar_valid = ra.store_gbar != 0;
   const bool f32 = d.grad_dtype == FLS_GRAD_F32;
   const bool overlap = p->overlap && !p->profiling;   // event records between kernels would serialise anyway
+  if (single) {
+    // no clipping: the coefficient is 1 before the norm is known, so one kernel does the whole step of the group
+    const AdamScalars sc1 = adam_scalars(d, lr, t_new);
+    ReduceAdamArgs rp{};
+    rp.r = ra;
+    rp.a.theta = p->master[g];
+    rp.a.m = p->m[g];
+    rp.a.v = p->v[g];
+    rp.a.pbf16 = p->pbf16[g];
+    rp.a.idx = ra.idx;
+    rp.a.decay = sc1.decay; rp.a.beta1 = sc1.beta1; rp.a.omb1 = sc1.omb1; rp.a.beta2 = sc1.beta2; rp.a.omb2 = sc1.omb2;
+    rp.a.step_size = sc1.step_size; rp.a.inv_sqrt_bc2 = sc1.inv_sqrt_bc2; rp.a.eps = sc1.eps;
+    cudaError_t e1 = timed_launch(p, FLS_KERNEL_ADAMW, st, [&] { return launch_step_noclip(rp, f32, p->reduce_sg, st, overlap && chain); });
+    if (e1 != cudaSuccess) return cuda_fail(e1, "single-pass step kernel launch");
+    return FLS_OK;
+  }
   cudaError_t e = timed_launch(p, FLS_KERNEL_REDUCE, st, [&] {
     return p->staged_reduce ? launch_reduce_staged(ra, st, overlap && chain) : launch_reduce(ra, f32, p->reduce_sg, st, overlap && chain);
   });
@@ -299,6 +317,8 @@ int fls_plan_create(const fls_plan_desc* desc, fls_plan** out) {
   if (d.reduce_wire == FLS_WIRE_BF16) p->reduce_sg = -2;   // generic kernel, bf16 rounding after every sum
   // fewer than 8 gradient bytes per element: a second read of the gradients costs less than the fp32 round trip
   p->recompute = d.reduce_wire == FLS_WIRE_F32 && K * (d.grad_dtype == FLS_GRAD_F32 ? 4 : 2) < 8;
+  // without clipping the coefficient is 1 whatever the norm: the step needs no second pass at all
+  p->single_pass = d.reduce_wire == FLS_WIRE_F32 && !(d.max_grad_norm > 0.0);
   *out = p;
   return FLS_OK;
 }
@@ -573,7 +593,7 @@ int fls_get_norms(const fls_plan* p, const float** dev_norms, const float** dev_
 int fls_get_reduced_grad(const fls_plan* p, const float** dev_gbar) {
   if (!p || !dev_gbar) return fail(FLS_EINVAL, "fls_get_reduced_grad: null argument");
   if (!p->bound) return fail(FLS_ESTATE, "fls_get_reduced_grad: plan has no buffers bound");
-  if (!p->gbar_valid) return fail(FLS_ESTATE, "fls_get_reduced_grad: the last step did not store the reduced gradient (recompute plan)");
+  if (!p->gbar_valid) return fail(FLS_ESTATE, "fls_get_reduced_grad: the last step did not store the reduced gradient (recompute or single-pass plan)");
   *dev_gbar = p->d_gbar(p->last_slot);
   return FLS_OK;
 }
@@ -631,6 +651,14 @@ int fls_plan_set_recompute(fls_plan* p, int mode) {
   if (mode > 0 && (!small || d.reduce_wire != FLS_WIRE_F32))
     return fail(FLS_ESTATE, "fls_plan_set_recompute: only for K*e_g < 8 bytes and fp32 partial sums");
   p->recompute = mode > 0 || (mode < 0 && small && d.reduce_wire == FLS_WIRE_F32);
+  return FLS_OK;
+}
+
+int fls_plan_set_single_pass(fls_plan* p, int mode) {
+  if (!p) return fail(FLS_EINVAL, "fls_plan_set_single_pass: null plan");
+  const bool can = p->desc.reduce_wire == FLS_WIRE_F32 && !(p->desc.max_grad_norm > 0.0);
+  if (mode > 0 && !can) return fail(FLS_ESTATE, "fls_plan_set_single_pass: only for plans without clipping and with fp32 partial sums");
+  p->single_pass = mode > 0 || (mode < 0 && can);
   return FLS_OK;
 }
 

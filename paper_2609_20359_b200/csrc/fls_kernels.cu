@@ -354,6 +354,41 @@ __device__ __noinline__ float reduce_slice_scalar(const ReduceArgs& a, uint64_t 
   return sq;
 }
 
+// End of every kernel that computes the norm: CTA partial -> workspace; the CTA that takes the last ticket adds
+// all partials in index order (so the norm does not depend on the order in which CTAs finish), then writes the
+// group's norm and clip coefficient and re-arms the ticket.  Must be reached by all threads of the CTA.
+template <int THREADS>
+__device__ __forceinline__ void finish_norm(const ReduceArgs& a, float sq) {
+  __shared__ double sh[THREADS / 32];
+  __shared__ bool is_last;
+  double total = block_sum<THREADS>(double(sq), sh);
+  if (threadIdx.x == 0) {
+    a.partials[blockIdx.x] = total;
+    __threadfence();
+    const uint32_t ticket = atomicAdd(a.ticket, 1u);
+    is_last = (ticket == gridDim.x - 1);
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  double s = 0.0;
+  for (uint32_t i = threadIdx.x; i < gridDim.x; i += THREADS) s += __ldcg(a.partials + i);
+  total = block_sum<THREADS>(s, sh);
+  if (threadIdx.x == 0) {
+    const double nrm = sqrt(total);
+    double c = 1.0;
+    if (a.max_grad_norm > 0.0) {
+      c = a.max_grad_norm / (nrm + 1e-6);
+      if (c >= 1.0) c = 1.0;            // NaN compares false and stays NaN: non-finite norms propagate
+    }
+    *a.normsq_out = total;
+    *a.norm_out = float(nrm);
+    *a.coef_out = float(c);
+    if (!isfinite(nrm)) atomicOr(a.status, uint32_t(FLS_STATUS_NONFINITE_NORM));
+    *a.ticket = 0u;                      // ready for the next launch (stream order)
+  }
+}
+
 // One pass, no loop: a CTA of THREADS threads owns U * THREADS/256 consecutive tiles (each group of 256
 // threads takes every (THREADS/256)-th of them, U in all) and the grid covers the whole buffer.  MINB resident
 // CTAs per SM fix the register budget: 1024 x 2 (32 registers) for the flat order with K = 4 or 8, 512 x 3 (42
@@ -383,8 +418,6 @@ __device__ __forceinline__ float reduce_one_tile(const ReduceArgs& a, uint32_t t
 
 template <bool F32, int KT, int SG, int THREADS, int MINB, int U>
 __global__ void __launch_bounds__(THREADS, MINB) fls_reduce_kernel(const __grid_constant__ ReduceArgs a) {
-  __shared__ double sh[THREADS / 32];
-  __shared__ bool is_last;
   constexpr uint32_t T = THREADS / kThreads;
   const uint32_t lane = threadIdx.x % kThreads;
   const uint32_t first = blockIdx.x * (T * U) + threadIdx.x / kThreads;   // this thread's tiles: first + u*T
@@ -436,34 +469,7 @@ __global__ void __launch_bounds__(THREADS, MINB) fls_reduce_kernel(const __grid_
   }
   dep_wait();                            // partials, ticket and the norm slots belong to the predecessor until now
   dep_launch();
-  // CTA partial -> workspace; the CTA that takes the last ticket adds all partials in index order, so
-  // the norm does not depend on the order in which CTAs finish.
-  double total = block_sum<THREADS>(double(sq), sh);
-  if (threadIdx.x == 0) {
-    a.partials[blockIdx.x] = total;
-    __threadfence();
-    const uint32_t ticket = atomicAdd(a.ticket, 1u);
-    is_last = (ticket == gridDim.x - 1);
-  }
-  __syncthreads();
-  if (!is_last) return;
-  __threadfence();
-  double s = 0.0;
-  for (uint32_t i = threadIdx.x; i < gridDim.x; i += THREADS) s += __ldcg(a.partials + i);
-  total = block_sum<THREADS>(s, sh);
-  if (threadIdx.x == 0) {
-    const double nrm = sqrt(total);
-    double c = 1.0;
-    if (a.max_grad_norm > 0.0) {
-      c = a.max_grad_norm / (nrm + 1e-6);
-      if (c >= 1.0) c = 1.0;            // NaN compares false and stays NaN: non-finite norms propagate
-    }
-    *a.normsq_out = total;
-    *a.norm_out = float(nrm);
-    *a.coef_out = float(c);
-    if (!isfinite(nrm)) atomicOr(a.status, uint32_t(FLS_STATUS_NONFINITE_NORM));
-    *a.ticket = 0u;                      // ready for the next launch (stream order)
-  }
+  finish_norm<THREADS>(a, sq);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -481,8 +487,6 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) { return uint32_t(__
 __global__ void __launch_bounds__(kThreads, 5) fls_reduce_staged_kernel(const __grid_constant__ ReduceArgs a) {
   __shared__ __align__(128) uint16_t stage[8][kTile];   // 32 KiB: one tile of each buffer
   __shared__ __align__(8) uint64_t bar;
-  __shared__ double sh[kThreads / 32];
-  __shared__ bool is_last;
   float sq = 0.f;
   const uint32_t tile = blockIdx.x;
   const Segment* sg = a.idx.segs + find_segment(a.idx, tile);
@@ -538,31 +542,7 @@ __global__ void __launch_bounds__(kThreads, 5) fls_reduce_staged_kernel(const __
   }
   dep_wait();
   dep_launch();
-  double total = block_sum<kThreads>(double(sq), sh);
-  if (threadIdx.x == 0) {
-    a.partials[blockIdx.x] = total;
-    __threadfence();
-    is_last = atomicAdd(a.ticket, 1u) == gridDim.x - 1;
-  }
-  __syncthreads();
-  if (!is_last) return;
-  __threadfence();
-  double s = 0.0;
-  for (uint32_t i = threadIdx.x; i < gridDim.x; i += kThreads) s += __ldcg(a.partials + i);
-  total = block_sum<kThreads>(s, sh);
-  if (threadIdx.x == 0) {
-    const double nrm = sqrt(total);
-    double c = 1.0;
-    if (a.max_grad_norm > 0.0) {
-      c = a.max_grad_norm / (nrm + 1e-6);
-      if (c >= 1.0) c = 1.0;
-    }
-    *a.normsq_out = total;
-    *a.norm_out = float(nrm);
-    *a.coef_out = float(c);
-    if (!isfinite(nrm)) atomicOr(a.status, uint32_t(FLS_STATUS_NONFINITE_NORM));
-    *a.ticket = 0u;
-  }
+  finish_norm<kThreads>(a, sq);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -665,6 +645,51 @@ __global__ void __launch_bounds__(kThreads, KT == 0 ? 2 : 3) fls_reduce_adamw_ke
     }
   }
   if (!waited) { dep_wait(); dep_launch(); }
+}
+
+// Whole step in one pass, for plans without clipping: the clip coefficient is 1 whatever the norm turns out
+// to be, so AdamW does not have to wait for it.  One 256-thread CTA per tile forms the mean gradient, applies
+// AdamW and contributes to the norm (still reported): K*e_g + 26 bytes per element instead of K*e_g + 34.
+// theta, m and v come out bit-identical to the two-pass route (there the gradient is multiplied by exactly 1).
+// (4 CTAs per SM measured best: 2 and 3 leave loads in flight on the table, 5 and 6 spill)
+template <bool F32, int KT, int SG>
+__global__ void __launch_bounds__(kThreads, 4) fls_step_noclip_kernel(const __grid_constant__ ReduceAdamArgs p) {
+  const AdamArgs& a = p.a;
+  float sq = 0.f;
+  const uint32_t tile = blockIdx.x;        // the grid covers every tile exactly once
+  const Slice s = slice_of(a.idx.segs + find_segment(a.idx, tile), tile, threadIdx.x);
+  if (s.vec) {
+    // nothing read here is written by the kernel before this one in the call (another group's step)
+    F8 th = ld8_stream(a.theta + s.a);
+    F8 m = ld8_stream(a.m + s.a);
+    F8 v = ld8_stream(a.v + s.a);
+    float g[8];
+    reduce_elems<8, F32, KT, SG>(p.r, s.j, g);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      sq = fmaf(g[e], g[e], sq);
+      adamw_one(a, 1.0f, g[e], th.v[e], m.v[e], v.v[e]);
+    }
+    dep_wait();
+    st8_stream(a.theta + s.a, th);
+    st8_stream(a.m + s.a, m);
+    st8_stream(a.v + s.a, v);
+    st_b128_stream(a.pbf16 + s.j, pack_bf16x8(th));
+  } else if (s.n) {
+    dep_wait();
+    for (uint32_t e = 0; e < s.n; ++e) {
+      float g[1];
+      reduce_elems<1, F32, 0, -1>(p.r, s.j + e, g);
+      sq = fmaf(g[0], g[0], sq);
+      float th = a.theta[s.a + e], m = a.m[s.a + e], v = a.v[s.a + e];
+      adamw_one(a, 1.0f, g[0], th, m, v);
+      a.theta[s.a + e] = th; a.m[s.a + e] = m; a.v[s.a + e] = v;
+      a.pbf16[s.j + e] = to_bf16_bits(th);
+    }
+  }
+  dep_wait();
+  dep_launch();
+  finish_norm<kThreads>(p.r, sq);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -937,6 +962,40 @@ cudaError_t launch_reduce(const ReduceArgs& a, bool f32, int sg, cudaStream_t st
     launch_reduce_t<true>(a, sg, grid, st, overlap);
   else
     launch_reduce_t<false>(a, sg, grid, st, overlap);
+  return cudaGetLastError();
+}
+
+namespace {
+template <bool F32, int KT>
+void launch_noclip_k(const ReduceAdamArgs& a, int sg, unsigned grid, cudaStream_t st, bool ov) {
+  if (sg == 0) { launch_k(fls_step_noclip_kernel<F32, KT, 0>, a, grid, kThreads, st, ov); return; }
+  if constexpr (KT == 0 || KT >= 2) { if (sg == 1) { launch_k(fls_step_noclip_kernel<F32, KT, 1>, a, grid, kThreads, st, ov); return; } }
+  if constexpr (KT == 0 || KT >= 4) { if (sg == 2) { launch_k(fls_step_noclip_kernel<F32, KT, 2>, a, grid, kThreads, st, ov); return; } }
+  if constexpr (KT == 0 || KT == 8) { if (sg == 4) { launch_k(fls_step_noclip_kernel<F32, KT, 4>, a, grid, kThreads, st, ov); return; } }
+  launch_k(fls_step_noclip_kernel<F32, 0, -1>, a, grid, kThreads, st, ov);
+}
+template <bool F32>
+void launch_noclip_t(const ReduceAdamArgs& a, int sg, unsigned grid, cudaStream_t st, bool ov) {
+  if (sg >= 0) {
+    switch (a.r.K) {
+      case 1: launch_noclip_k<F32, 1>(a, sg, grid, st, ov); return;
+      case 2: launch_noclip_k<F32, 2>(a, sg, grid, st, ov); return;
+      case 4: launch_noclip_k<F32, 4>(a, sg, grid, st, ov); return;
+      case 8: launch_noclip_k<F32, 8>(a, sg, grid, st, ov); return;
+      default: break;
+    }
+  }
+  launch_noclip_k<F32, 0>(a, sg, grid, st, ov);
+}
+}  // namespace
+
+// Single pass for plans without clipping; the grid is one CTA per tile (= the number of norm partials).
+cudaError_t launch_step_noclip(const ReduceAdamArgs& a, bool f32, int sg, cudaStream_t st, bool overlap) {
+  const unsigned grid = a.a.idx.n_tiles;
+  if (f32)
+    launch_noclip_t<true>(a, sg, grid, st, overlap);
+  else
+    launch_noclip_t<false>(a, sg, grid, st, overlap);
   return cudaGetLastError();
 }
 

@@ -92,6 +92,7 @@ unsigned reduce_grid(const ReduceArgs& a, int sg, bool f32);
 cudaError_t launch_reduce(const ReduceArgs& a, bool f32, int sg, cudaStream_t st, bool overlap);
 // Shared-memory staged variant of the reduce kernel (bf16, flat order, K = 8, fully vectorisable layout only).
 cudaError_t launch_reduce_staged(const ReduceArgs& a, cudaStream_t st, bool overlap);
+cudaError_t launch_step_noclip(const ReduceAdamArgs& a, bool f32, int sg, cudaStream_t st, bool overlap);
 cudaError_t launch_reduce_adamw(const ReduceAdamArgs& a, bool f32, int sg, unsigned grid, cudaStream_t st, bool overlap);
 cudaError_t launch_adamw(const AdamArgs& a, unsigned grid, cudaStream_t st, bool overlap);
 cudaError_t launch_fedavg(const FedavgArgs& a, unsigned grid, cudaStream_t st, bool overlap);

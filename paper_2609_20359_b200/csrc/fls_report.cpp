@@ -59,7 +59,11 @@ void comm_report(const Layout& lay, const fls_plan_desc& d, const double* bw, fl
   const double K = S * R;
   // store-and-reread moves K*e_g + 34 bytes per element; with K*e_g < 8 the library reads the gradients twice
   // instead and moves 2*K*e_g + 26
-  const double per_elem = (K * e < 8.0 && d.reduce_wire == FLS_WIRE_F32) ? 2.0 * K * e + 26.0 : K * e + 34.0;
+  // ... and without clipping one pass does everything: K*e_g + 26
+  const bool f32_sums = d.reduce_wire == FLS_WIRE_F32;
+  const double per_elem = (f32_sums && !(d.max_grad_norm > 0.0)) ? K * e + 26.0
+                          : (f32_sums && K * e < 8.0)            ? 2.0 * K * e + 26.0
+                                                                 : K * e + 34.0;
   out->hbm_bytes_sync_step = F * double(lay.n_padded) * per_elem;
   out->hbm_bytes_fedavg = F * double(lay.n_padded) * ((d.fedavg_what & FLS_AVG_OPT_STATE) ? 26.0 : 10.0);
 }

@@ -140,6 +140,31 @@ def test_recompute_plan_is_bit_identical_to_store_and_reread(fls, units, G, S, R
     c.close()
 
 
+@pytest.mark.parametrize("units,G,S,R_rep,Q,dtype", [([40000, 30011], 2, 8, 1, 8, "bf16"), ([40000, 30011], 2, 4, 2, 8, "bf16"),
+                                                     ([70001], 2, 3, 2, 1, "bf16"), ([40000, 30011], 2, 2, 1, 8, "f32"),
+                                                     ([40000, 30011], 1, 1, 1, 8, "bf16"), ([17], 2, 4, 1, 1, "bf16")])
+def test_single_pass_without_clipping(fls, units, G, S, R_rep, Q, dtype):
+    """max_grad_norm = 0: one kernel per group does reduce + norm + AdamW.  Against the oracle, and bit for bit against
+    the forced two-pass route (norms to rounding: the partial sums are grouped differently)."""
+    outs, norms = [], []
+    for mode in (-1, 0):
+        c = Case(units, G, S, R_rep, H=2, Q=Q, grad_dtype=dtype, hp=orc.Hyper(max_grad_norm=0.0), per_buffer_scale=True, fused=(G > 1))
+        fls.fls_plan_set_single_pass(c.sess.plan, mode)
+        for _ in range(4):
+            c.step([2, 1][:G])
+            c.compare()
+        assert c.sess.coefs().cpu().tolist() == [1.0] * G
+        outs.append([x.clone() for x in c.sess.master + c.sess.m + c.sess.v + c.sess.param_bf16])
+        norms.append(c.sess.norms().cpu())
+        c.close()
+    assert all(torch.equal(x, y) for x, y in zip(*outs))
+    assert torch.allclose(norms[0], norms[1], rtol=1e-6, atol=0)
+    c = Case([4096], 1, 8, 1, H=2, Q=8)                     # this plan clips
+    with pytest.raises(fls.FlsError):
+        fls.fls_plan_set_single_pass(c.sess.plan, 1)
+    c.close()
+
+
 def test_staged_reduce_variant_is_bit_identical(fls):
     """The shared-memory staged reduce kernel (bulk asynchronous copies) against the default kernel: same bits,
     ragged last tiles included; it refuses plans it does not cover."""
@@ -196,6 +221,7 @@ def test_bf16_wire_orders_differ_on_the_gpu_too(fls):
     for wire in (False, True):
         for S, R_rep in ((8, 1), (4, 2)):
             c = Case([65536], 1, S, R_rep, H=10, Q=8, hp=orc.Hyper(max_grad_norm=0.0, wire_bf16=wire))
+            fls.fls_plan_set_single_pass(c.sess.plan, 0)      # two passes, so that the mean gradient is stored
             c.load_grads(1)
             c.sess.step()
             torch.cuda.synchronize()
@@ -215,6 +241,7 @@ def test_two_level_order_differs_from_flat_where_fp32_rounds(fls):
     res = {}
     for (S, R_rep) in ((8, 1), (4, 2)):
         c = Case(units, 1, S, R_rep, H=10, Q=8, grad_dtype="f32", hp=orc.Hyper(max_grad_norm=0.0))
+        fls.fls_plan_set_single_pass(c.sess.plan, 0)          # two passes, so that the mean gradient is stored
         grads = c.load_grads(1, big)
         c.sess.step()
         torch.cuda.synchronize()

@@ -128,6 +128,10 @@ def test_comm_report_matches_oracle_and_paper_table(fls):
         assert math.isclose(rep["wire_bytes"]["fsdp"], sum(3 * (S - 1) * m for m in Mb), rel_tol=1e-12, abs_tol=1e-9)
         K = S * R
         assert rep["hbm_bytes_sync_step"] == F * L.n_padded * ((2 * K * e + 26) if K * e < 8 else (K * e + 34))
+        p0 = fls.fls_plan_create(sum(units), units, groups=F, shard_dim=S, replicate_dim=R, sync_period=A, max_grad_norm=0.0,
+                                 grad_dtype=fls.FLS_GRAD_F32 if f32 else fls.FLS_GRAD_BF16, align_elems=1)
+        assert fls.fls_comm_report(p0)["hbm_bytes_sync_step"] == F * L.n_padded * (K * e + 26)      # no clipping: one pass
+        fls.fls_plan_destroy(p0)
         assert rep["hbm_bytes_fedavg"] == F * L.n_padded * 10
         fls.fls_plan_destroy(p)
 
