@@ -614,7 +614,7 @@ __device__ __noinline__ void reduce_adamw_slice_scalar(const ReduceAdamArgs& p, 
 }
 
 template <bool F32, int KT, int SG>
-__global__ void __launch_bounds__(kThreads, KT == 0 ? 2 : 3) fls_reduce_adamw_kernel(const __grid_constant__ ReduceAdamArgs p) {
+__global__ void __launch_bounds__(kThreads, KT == 0 ? 2 : 4) fls_reduce_adamw_kernel(const __grid_constant__ ReduceAdamArgs p) {
   const AdamArgs& a = p.a;
   const uint32_t n_tiles = a.idx.n_tiles;
   if (blockIdx.x >= n_tiles) { dep_wait(); dep_launch(); return; }
