@@ -4,9 +4,12 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl ours|reference]
 
 A step is one fls_sync_step over all G groups, followed by fls_fedavg when the step counter is a
-multiple of H.  Metric: synced params/s = G*P*K / time (logical parameters, whole job).  Prints one
-JSON line on rank 0.  With N > 1 every rank runs an independent replica of the workload (the path has
-no inter-GPU exchange); the time is the maximum over ranks.
+multiple of H (one fused call on those steps).  Metric: synced params/s = G*P*K / time (logical
+parameters, whole job).  Prints one JSON line on rank 0.  The default workload is the largest one that
+fits a single GPU, the Llama-3.2-1B-sized FL+HSDP configuration; the 8B-block and GPT-2-small-sized
+workloads are timed afterwards and reported under "other_workloads" of the same line.
+With N > 1 every rank runs an independent replica of the workload (the path has no inter-GPU exchange);
+the time is the maximum over ranks.  Started without a launcher, `--gpus N` starts the N ranks itself.
 `--impl reference` times the CPU oracle on a bounded sample of the same workload instead.
 """
 from __future__ import annotations
@@ -29,10 +32,17 @@ import synthetic as sy
 
 METRIC = "synced_params_per_s"
 UNIT = "params/s"
-DEFAULT_CONFIG = "gpt2_small_fl_fsdp"
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture summarised in
-# profiles/dram_traffic_gpt2_small.md; None for workloads that have no capture.
-NCU_TRAFFIC_BYTES = {("gpt2_small_fl_fsdp", "adamw"): 3673.2e6, ("gpt2_small_fl_fsdp", "reduce"): 2444.6e6}
+DEFAULT_CONFIG = "llama32_1b_fl_hsdp"
+OTHER_WORKLOADS = ("llama31_8b_block_fl_fsdp", "gpt2_small_fl_fsdp")
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per group-element and launch, measured with ncu on
+# slices of the workloads (one kernel per capture, a few GB on the device); the traffic of these streams grows
+# in proportion to the element count, so a launch over N elements moves N times the figure.  Keyed by kernel
+# and, for the kernels that read the gradients, by the gradient bytes per element K*e_g.
+NCU_TRAFFIC_BYTES_PER_ELEM = {("reduce", 16): 19.45, ("adamw", None): 29.52, ("adamw_fedavg", None): 29.17}
+# The CPU oracle is timed on the first ORACLE_SAMPLE parameters of every buffer: once on one thread, once with
+# the sample cut into chunks that a pool of all host cores works through.
+ORACLE_SAMPLE_ONE_CORE = 1 << 24
+ORACLE_SAMPLE_ALL_CORES = 1 << 26
 
 
 def measured_peak_gbs():
@@ -120,12 +130,24 @@ def max_over_ranks(value: float, world: int, device=None) -> float:
 
 
 # --------------------------------------------------------------------------------------- CPU oracle leg
-def oracle_sample(cfg: dict, sample_params: int):
+def host_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def oracle_sample(cfg: dict, sample_params: int, threads: int = 1):
     """One oracle step of all G groups and one FedAvg on the first `sample_params` parameters of every
-    buffer, as the oracle stands, on one host thread.  The sample's inputs come from the shared generator
-    (filled on the GPU when there is one, since the fill is not what is being timed, then copied to the
-    host).  Returns (params/s with FedAvg counted once per H steps, seconds of oracle work, threads)."""
+    buffer, with the oracle's functions as they stand.  threads = 1: the plain whole-array calls on one host
+    thread.  threads > 1: the sample is cut into 2^20-parameter chunks that a pool of `threads` workers goes
+    through (numpy releases the interpreter lock inside its loops): per chunk the mean gradient and its squared
+    norm, then the clip coefficient from the sum, then per chunk AdamW; FedAvg per chunk likewise.  The sample's
+    inputs come from the shared generator (filled on the GPU when there is one, since the fill is not what is
+    being timed, then copied to the host).  Returns (params/s with FedAvg counted once per H steps, seconds of
+    oracle work, threads)."""
     from oracle import fls_oracle as orc
+    from concurrent.futures import ThreadPoolExecutor
     try:
         from threadpoolctl import threadpool_limits
     except Exception:                                   # pragma: no cover
@@ -149,41 +171,92 @@ def oracle_sample(cfg: dict, sample_params: int):
             row.append(t.numpy() if f32 else t.view(torch.int16).numpy().view(np.uint16))
         raw.append(row)
     counts = [sy.sample_count(cfg["seed"], g) for g in range(G)] if cfg["weights"] == "counts" else None
+    as_f64 = (lambda x: x.astype(np.float64)) if f32 else orc.bf16_bits_to_f64
     with threadpool_limits(limits=1):
-        t0 = time.perf_counter()
-        for g in range(G):
-            grads = [x.astype(np.float64) if f32 else orc.bf16_bits_to_f64(x) for x in raw[g]]
-            orc.sync_step_group(states[g], grads, S, R, 1, hp)
-            del grads
-        t_step = time.perf_counter() - t0
-        t0 = time.perf_counter()
-        orc.fedavg(states, counts)
-        t_avg = time.perf_counter() - t0
+        if threads <= 1:
+            t0 = time.perf_counter()
+            for g in range(G):
+                grads = [as_f64(x) for x in raw[g]]
+                orc.sync_step_group(states[g], grads, S, R, 1, hp)
+                del grads
+            t_step = time.perf_counter() - t0
+            t0 = time.perf_counter()
+            orc.fedavg(states, counts)
+            t_avg = time.perf_counter() - t0
+        else:
+            chunk = 1 << 20
+            los = list(range(0, P, chunk))
+            bits = [np.zeros(P, np.uint16) for _ in range(G)]
+            with ThreadPoolExecutor(threads) as ex:
+                t0 = time.perf_counter()
+                for g in range(G):
+                    st = states[g]
+                    def reduce_chunk(lo, g=g):
+                        gb = orc.reduce_mean([as_f64(x[lo:lo + chunk]) for x in raw[g]], S, R)
+                        return gb, orc.grad_norm(gb) ** 2
+                    parts = list(ex.map(reduce_chunk, los))
+                    c = orc.clip_coef(float(np.sqrt(sum(sq for _, sq in parts))), hp.max_grad_norm)
+                    def adamw_chunk(i, st=st, g=g):
+                        lo = los[i]
+                        sl = slice(lo, lo + chunk)
+                        st.theta[sl], st.m[sl], st.v[sl], bits[g][sl] = orc.adamw(
+                            st.theta[sl], st.m[sl], st.v[sl], parts[i][0], c, 1, hp.lr, hp.beta1, hp.beta2, hp.eps, hp.weight_decay)
+                    list(ex.map(adamw_chunk, range(len(los))))
+                    del parts
+                t_step = time.perf_counter() - t0
+                t0 = time.perf_counter()
+                w = orc.fedavg_weights(counts, G)
+                avg = np.empty(P, np.float32)
+                def fedavg_chunk(lo):
+                    sl = slice(lo, lo + chunk)
+                    avg[sl] = orc.fedavg_array([st.theta[sl] for st in states], w)
+                    bits[0][sl] = orc.f32_to_bf16_bits(avg[sl])
+                list(ex.map(fedavg_chunk, los))
+                for st in states:
+                    st.theta[:] = avg
+                t_avg = time.perf_counter() - t0
     sec = t_step + t_avg / cfg["sync_period"]
-    return G * P / sec, t_step + t_avg, 1
+    return G * P / sec, t_step + t_avg, max(1, threads)
+
+
+def sample_text(cfg: dict, n: int) -> str:
+    return f"one oracle step of all {cfg['groups']} groups + FedAvg/H on the first {min(n, cfg['n_params'])} params of every buffer"
+
+
+def cpu_baseline(cfg: dict) -> dict:
+    """The oracle on this machine's host cores: all of them (the headline figure of this object), and one."""
+    cores = host_cores()
+    v1, s1, _ = oracle_sample(cfg, ORACLE_SAMPLE_ONE_CORE, 1)
+    va, sa, used = oracle_sample(cfg, ORACLE_SAMPLE_ALL_CORES, cores)
+    return {"value": va, "unit": UNIT, "cores": used, "kind": "oracle", "seconds": sa, "sample": sample_text(cfg, ORACLE_SAMPLE_ALL_CORES),
+            "host_cores": cores,
+            "one_core": {"value": v1, "unit": UNIT, "cores": 1, "seconds": s1, "sample": sample_text(cfg, ORACLE_SAMPLE_ONE_CORE)}}
 
 
 def run_reference(args, cfg):
     """The reference arm of this build is the CPU oracle (the paper ships no code): every "step" is one
-    oracle step + FedAvg/H on a bounded sample of the workload.  Rank 0 only."""
+    oracle step + FedAvg/H on a bounded sample of the workload, on all host cores.  Rank 0 only."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    sample = 1 << 24
+    cores = host_cores()
     vals, secs = [], []
     if args.warmup:
-        oracle_sample(cfg, 1 << 18)
+        oracle_sample(cfg, 1 << 18, cores)
     n = max(1, min(args.steps, 3))
     for _ in range(n):
-        v, s, cores = oracle_sample(cfg, sample)
+        v, s, used = oracle_sample(cfg, ORACLE_SAMPLE_ALL_CORES, cores)
         vals.append(v); secs.append(s)
     value = float(np.mean(vals))
-    what = f"one oracle step of all {cfg['groups']} groups + FedAvg/H on the first {min(sample, cfg['n_params'])} params of every buffer"
+    v1, s1, _ = oracle_sample(cfg, ORACLE_SAMPLE_ONE_CORE, 1)
+    what = sample_text(cfg, ORACLE_SAMPLE_ALL_CORES)
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": n,
             "warmup": 1 if args.warmup else 0, "ms_per_step": 1e3 * float(np.mean(secs)), "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": cfg["name"], "sample": what},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": what},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": used, "kind": "oracle", "sample": what, "host_cores": cores,
+                             "one_core": {"value": v1, "unit": UNIT, "cores": 1, "seconds": s1,
+                                          "sample": sample_text(cfg, ORACLE_SAMPLE_ONE_CORE)}},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
 
@@ -200,25 +273,11 @@ def fill_session(sess, cfg):
     torch.cuda.synchronize()
 
 
-def run_ours(args, cfg):
+def measure_workload(args, cfg, fls, Session, rank, world, local, with_e2e, sampler):
+    """Times one workload on this rank's GPU: K steps with events around the whole region, K more with events
+    around every launch (per-kernel durations), optionally the end-to-end form with host gradients.  Returns the
+    fields of the JSON line that describe this workload (rank 0) or None (other ranks)."""
     import torch.distributed as dist
-    from paper_2609_20359_b200 import build
-
-    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device (there is no CPU path); use --impl reference for the oracle")
-    torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    if rank == 0:
-        build.build()
-    if world > 1:
-        dist.barrier()
-    # only now: importing the binding loads libfls.so, which rank 0 may just have built
-    from paper_2609_20359_b200 import _binding as fls
-    from paper_2609_20359_b200.session import Session
-
     G, P = cfg["groups"], cfg["n_params"]
     counts = [sy.sample_count(cfg["seed"], g) for g in range(G)] if cfg["weights"] == "counts" else None
     fused = not args.unfused and G <= fls.FLS_MAX_FUSED_GROUPS
@@ -233,8 +292,6 @@ def run_ours(args, cfg):
         fls.fls_plan_tune(sess.plan, fls.FLS_KERNEL_ADAMW, 0, 1)
     if args.ascending_adamw:
         fls.fls_plan_tune(sess.plan, fls.FLS_KERNEL_ADAMW, 0, 0)
-    if args.staged_reduce:
-        fls.fls_plan_set_staging(sess.plan, True)
     if args.no_overlap:
         fls.fls_plan_set_overlap(sess.plan, False)
     fill_session(sess, cfg)
@@ -259,11 +316,11 @@ def run_ours(args, cfg):
 
     # Inputs larger than L2 need no flush.  A workload whose buffers fit in twice the L2 is timed step by step
     # with a write of a 512 MB buffer (untimed) before every step, so that no step starts with its inputs cached.
-    eg0 = 4 if cfg["grad_dtype"] == "f32" else 2
-    footprint = G * sess.n_padded * (sess.K * eg0 + 14) + 4 * sess.n_padded
+    eg = 4 if cfg["grad_dtype"] == "f32" else 2
+    footprint = G * sess.n_padded * (sess.K * eg + 14) + 4 * sess.n_padded
     flush_buf = torch.empty(512 << 20, dtype=torch.uint8, device="cuda") if footprint < 2 * 126e6 else None
 
-    def timed(n_steps, profiling, sampler=None):
+    def timed(n_steps, profiling, smp=None):
         fls.fls_set_profiling(sess.plan, profiling)
         barrier()
         l0 = fls.fls_get_launch_count(sess.plan)
@@ -274,8 +331,8 @@ def run_ours(args, cfg):
             for _ in range(n_steps):
                 one_step()
             e1.record(stream)
-            if sampler is not None:
-                sampler.wait_for(e1)
+            if smp is not None:
+                smp.wait_for(e1)
             barrier()
             ms = e0.elapsed_time(e1)
         else:
@@ -286,8 +343,8 @@ def run_ours(args, cfg):
                 e0.record(stream)
                 one_step()
                 e1.record(stream)
-                if sampler is not None:
-                    sampler.wait_for(e1)
+                if smp is not None:
+                    smp.wait_for(e1)
                 torch.cuda.synchronize()
                 ms += e0.elapsed_time(e1)
             barrier()
@@ -296,28 +353,22 @@ def run_ours(args, cfg):
 
     for _ in range(args.warmup):
         one_step()
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
-    ms_total, launches = timed(args.steps, False, sampler if rank == 0 else None)
+    ms_total, launches = timed(args.steps, False, sampler)
     fedavg_calls = n_fedavg[0]
-    in_region = len(sampler.sm)
+    in_region = len(sampler.sm) if sampler is not None else 0
     # second pass over the same number of steps with events around every kernel: per-kernel durations
     # (the clocks keep being sampled: an NVML reading can take as long as a short timed region)
-    ms_prof, _ = timed(args.steps, True, sampler if rank == 0 else None)
-    clocks = sampler.stop() if rank == 0 else None
-    if clocks is not None:
-        clocks["samples_in_timed_region"] = in_region
+    ms_prof, _ = timed(args.steps, True, sampler)
     kms, kn = fls.fls_get_kernel_ms(sess.plan)
     fls.fls_set_profiling(sess.plan, False)
 
     # end to end: gradients start in pinned host memory, norms come back to the host, every step
     e2e = None
-    eg_bytes = 4 if cfg["grad_dtype"] == "f32" else 2
-    if not args.no_e2e and G * sess.K * sess.n_padded * eg_bytes > args.e2e_max_gb * 2 ** 30:
-        e2e = {"value": None, "unit": UNIT, "skipped": f"pinned staging above --e2e-max-gb {args.e2e_max_gb}"}
-    elif not args.no_e2e:
-        host = [[torch.empty(sess.n_padded, dtype=sess.grad_torch_dtype).pin_memory() for _ in range(sess.K)] for _ in range(G)]
+    h2d = G * sess.K * sess.n_padded * eg
+    if with_e2e and h2d > args.e2e_max_gb * 2 ** 30:
+        e2e = {"value": None, "unit": UNIT, "skipped": f"pinned host buffers above --e2e-max-gb {args.e2e_max_gb}"}
+    elif with_e2e:
+        host = [[torch.empty(sess.n_padded, dtype=sess.grad_torch_dtype, pin_memory=True) for _ in range(sess.K)] for _ in range(G)]
         for g in range(G):
             for k in range(sess.K):
                 host[g][k].copy_(sess.grads[g][k])
@@ -334,63 +385,148 @@ def run_ours(args, cfg):
             e2e_step()
         torch.cuda.synchronize()
         dt = max_over_ranks(time.perf_counter() - t0, world, "cuda")
-        eg = 4 if cfg["grad_dtype"] == "f32" else 2
-        e2e = {"value": world * G * P * n_e2e / dt, "unit": UNIT, "h2d_bytes_per_step": G * sess.K * sess.n_padded * eg,
+        e2e = {"value": world * G * P * n_e2e / dt, "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": 4 * G, "steps": n_e2e, "ms_per_step": 1e3 * dt / n_e2e}
         del host
 
+    out = None
     if rank == 0:
         peak, peak_kind = measured_peak_gbs()
         N = sess.n_padded
-        eg = 4 if cfg["grad_dtype"] == "f32" else 2
+        kbytes = sess.K * eg
         # FedAvg runs one launch per averaged array: parameters move 10 B per group-element (4 read, 4 + 2
         # written), m and v 8 B each; the figure is the mean over the launches of one call
-        per_launch = {"reduce": N * (sess.K * eg + 4), "adamw": N * 30, "fedavg": N * G * (26 / 3 if args.opt_state else 10),
+        per_launch = {"reduce": N * (kbytes + 4), "adamw": N * 30, "fedavg": N * G * (26 / 3 if args.opt_state else 10),
                       "adamw_fedavg": N * G * 30}
+        traffic_key = {"reduce": ("reduce", kbytes), "adamw": ("adamw", None), "fedavg": ("fedavg", None), "adamw_fedavg": ("adamw_fedavg", None)}
+        units = {"reduce": N, "adamw": N, "fedavg": N * G, "adamw_fedavg": N * G}
         if not cfg["max_grad_norm"] > 0:
             # no clipping: one kernel per group does the whole step (timed under "adamw")
-            per_launch.update(adamw=N * (sess.K * eg + 26))
-        elif sess.K * eg < 8:
+            per_launch.update(adamw=N * (kbytes + 26))
+            traffic_key.update(adamw=("step_noclip", kbytes))
+        elif kbytes < 8:
             # small K: nothing is stored by the norm pass and AdamW reads the gradients again
-            per_launch.update(reduce=N * sess.K * eg, adamw=N * (sess.K * eg + 26))
+            per_launch.update(reduce=N * kbytes, adamw=N * (kbytes + 26))
+            traffic_key.update(reduce=("norm_only", kbytes), adamw=("reduce_adamw", kbytes))
         kernels = {}
         for i, name in enumerate(("reduce", "adamw", "fedavg", "adamw_fedavg")):
             if kn[i]:
                 avg_ms = kms[i] / kn[i]
+                per_elem = NCU_TRAFFIC_BYTES_PER_ELEM.get(traffic_key[name])
                 kernels[name] = {"launches": kn[i], "avg_ms": avg_ms, "bytes_per_launch": per_launch[name],
                                  "gbs": per_launch[name] / avg_ms / 1e6, "frac": per_launch[name] / avg_ms / 1e6 / peak,
-                                 "share": kms[i] / sum(kms)}
+                                 "frac_of_8tbs": per_launch[name] / avg_ms / 1e6 / 8000.0,
+                                 "share": kms[i] / sum(kms), "traffic": per_elem * units[name] if per_elem else None}
         dom = max(kernels, key=lambda n: kernels[n]["share"])
         rep = fls.fls_comm_report(sess.plan)
         # bytes the timed steps had to move: every sync step, plus the FedAvg calls that fell inside the region
         # (the fused aggregation moves no bytes of its own: an aggregation step costs what a plain step costs)
         step_bytes = rep["hbm_bytes_sync_step"] + (0 if fused else rep["hbm_bytes_fedavg"] * fedavg_calls / args.steps)
         ms_step = ms_total / args.steps
-        line = {
-            "metric": METRIC, "value": world * G * P * args.steps / (ms_total / 1e3), "unit": UNIT, "n_gpus": world,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        out = {
+            "value": world * G * P * args.steps / (ms_total / 1e3), "ms_per_step": ms_step,
             "config": {"workload": cfg["name"], "n_params": P, "groups": G, "shard_dim": cfg["shard_dim"],
                        "replicate_dim": cfg["replicate_dim"], "sync_period": cfg["sync_period"], "grad_dtype": cfg["grad_dtype"],
-                       "fedavg_opt_state": bool(args.opt_state), "fused_aggregation": bool(fused), "staged_reduce": bool(args.staged_reduce), "fedavg_calls_in_timed_region": fedavg_calls, "l2": "working set exceeds L2, no flush needed" if flush_buf is None else "L2 flushed (512 MB write, untimed) before every timed step",
+                       "fedavg_opt_state": bool(args.opt_state), "fused_aggregation": bool(fused),
+                       "fedavg_calls_in_timed_region": fedavg_calls,
+                       "l2": "working set exceeds L2, no flush needed" if flush_buf is None else "L2 flushed (512 MB write, untimed) before every timed step",
                        "parallelism": "replicas only" if world > 1 else "1 gpu"},
             "hbm_gbs": step_bytes / ms_step / 1e6, "hbm_frac_of_measured_peak": step_bytes / ms_step / 1e6 / peak,
             "hbm_frac_of_8tbs": step_bytes / ms_step / 1e6 / 8000.0,
             "roofline": {"bound": "hbm", "kernel": dom, "achieved": kernels[dom]["gbs"], "peak": peak, "peak_kind": peak_kind,
-                         "unit": "GB/s", "frac": kernels[dom]["frac"], "traffic": NCU_TRAFFIC_BYTES.get((cfg["name"], dom))},
+                         "unit": "GB/s", "frac": kernels[dom]["frac"], "traffic": kernels[dom]["traffic"]},
             "kernels": kernels, "ms_per_step_profiled": ms_prof / args.steps,
-            "gpu_launches": launches, "clocks": clocks, "e2e": e2e,
+            "gpu_launches": launches, "samples_in_timed_region": in_region, "e2e": e2e,
         }
     sess.close()
+    del sess, flush_buf
+    torch.cuda.empty_cache()
+    return out
+
+
+def run_ours(args, cfg):
+    import torch.distributed as dist
+    from paper_2609_20359_b200 import build
+
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path); use --impl reference for the oracle")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     if rank == 0:
+        build.build()
+    if world > 1:
+        dist.barrier()
+    # only now: importing the binding loads libfls.so, which rank 0 may just have built
+    from paper_2609_20359_b200 import _binding as fls
+    from paper_2609_20359_b200.session import Session
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    if sampler is not None:
+        sampler.start()
+    main = measure_workload(args, cfg, fls, Session, rank, world, local, not args.no_e2e, sampler)
+    others = {}
+    if args.others:
+        # the other two workloads of the target list, device-resident timing only; every rank runs them so that the
+        # barriers match, rank 0 reports them
+        for name in OTHER_WORKLOADS:
+            if name == cfg["name"]:
+                continue
+            r = measure_workload(args, sy.config_by_name(name), fls, Session, rank, world, local, False, sampler)
+            if r is not None:
+                others[name] = {k: r[k] for k in ("value", "ms_per_step", "hbm_gbs", "hbm_frac_of_measured_peak", "hbm_frac_of_8tbs",
+                                                  "roofline", "kernels", "gpu_launches", "config")}
+    if rank == 0:
+        clocks = sampler.stop()
+        clocks["samples_in_timed_region"] = main.pop("samples_in_timed_region")
+        line = {"metric": METRIC, "value": main["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+                "ms_per_step": main["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "f32", "data": "synthetic"}
+        line.update({k: v for k, v in main.items() if k not in ("value", "ms_per_step")})
+        line["clocks"] = clocks
+        if others:
+            line["other_workloads"] = others
         if world == 1 and not args.no_cpu_baseline:
-            torch.cuda.empty_cache()
-            n_s = min(1 << 25, P)
-            v, s, cores = oracle_sample(cfg, n_s)
-            line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "seconds": s,
-                                    "sample": f"one oracle step of all {G} groups + FedAvg/H on the first {n_s} params of every buffer"}
+            line["cpu_baseline"] = cpu_baseline(cfg)
         print(json.dumps(line), flush=True)
     if world > 1:
+        dist.destroy_process_group()
+
+
+# --------------------------------------------------------------------------------------- launching N ranks
+def free_port() -> int:
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def spawn_ranks(n: int, argv) -> int:
+    """`--gpus N` without a launcher: run this same command as N ranks, one process per GPU, under
+    torch.distributed.run on this node.  Returns the launcher's exit code."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(free_port()), os.path.abspath(__file__)] + list(argv)
+    return subprocess.run(cmd).returncode
+
+
+def run_stub(args):
+    """Launch plumbing without a GPU (used by the CPU tests): every rank "times" a step whose duration depends on
+    its rank, the ranks agree on the slowest over gloo, rank 0 prints the line."""
+    import torch.distributed as dist
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group("gloo")
+    ms = max_over_ranks(10.0 * (rank + 1) * args.steps, world)
+    units = 1000
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "value": world * units * args.steps / (ms / 1e3), "unit": UNIT, "n_gpus": world,
+                          "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+                          "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                          "config": {"workload": "stub", "parallelism": "replicas only" if world > 1 else "1 gpu"}}), flush=True)
+    if world > 1:
+        dist.barrier()
         dist.destroy_process_group()
 
 
@@ -488,12 +624,13 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-max-gb", type=float, default=48.0, help="skip the end-to-end pass if its pinned host staging would exceed this")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-others", dest="others", action="store_false", help="time only the chosen workload (default: the default workload is followed by the other two target workloads)")
+    ap.add_argument("--stub-workload", action="store_true", help=argparse.SUPPRESS)   # launch plumbing on CPU, for the tests
     ap.add_argument("--ctas-reduce", type=int, default=0)
     ap.add_argument("--ctas-adamw", type=int, default=0)
     ap.add_argument("--ctas-fedavg", type=int, default=0)
     ap.add_argument("--descending-adamw", action="store_true")
     ap.add_argument("--ascending-adamw", action="store_true")
-    ap.add_argument("--staged-reduce", action="store_true", help="reduce kernel stages its tiles through shared memory (cp.async.bulk)")
     ap.add_argument("--no-overlap", action="store_true", help="plain launches instead of programmatic dependent launch")
     # slices of a workload, for profiler captures that must stay small (same kernels, fewer bytes)
     ap.add_argument("--n-params", type=int, default=0, help="override P (single flat unit)")
@@ -508,12 +645,25 @@ def main():
     ap.add_argument("--sweep-out", default="sweep_results.jsonl")
     ap.add_argument("--sweep-exps", default="20,22,24,26,28,30", help="log2 of the parameter counts to sweep")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started without a launcher: become N ranks
+        raise SystemExit(spawn_ranks(args.gpus, sys.argv[1:]))
+    if args.stub_workload:
+        run_stub(args)
+        return
     if args.sweep:
         os.makedirs(os.path.dirname(args.sweep_out) or ".", exist_ok=True)
         run_sweep(args)
         return
     cfg = sy.config_by_name(args.config)
-    if args.n_params:
+    sliced = any([args.n_params, args.groups, args.sync_period, args.shard_dim, args.replicate_dim, args.clip is not None, args.grad_dtype])
+    if sliced or args.config != DEFAULT_CONFIG:
+        args.others = False
+    if args.n_params and args.keep_units:
+        # same unit table, every unit scaled by n_params / P and rounded to a multiple of 64 elements
+        units = [max(64, int(round(u * args.n_params / cfg["n_params"] / 64)) * 64) for u in cfg["unit_numel"]]
+        cfg.update(n_params=sum(units), unit_numel=units, name=cfg["name"] + f"[P={sum(units)}, {len(units)} units]")
+    elif args.n_params:
         cfg.update(n_params=args.n_params, unit_numel=[args.n_params], name=cfg["name"] + f"[P={args.n_params}]")
     if args.groups:
         cfg.update(groups=args.groups, name=cfg["name"] + f"[G={args.groups}]")

@@ -45,7 +45,7 @@ enum { FLS_GRAD_BF16 = 0, FLS_GRAD_F32 = 1 };
 enum { FLS_WIRE_F32 = 0, FLS_WIRE_BF16 = 1 };          /* reduce_wire */
 enum { FLS_AVG_PARAMS = 1, FLS_AVG_OPT_STATE = 2, FLS_AVG_FUSED = 4 }; /* fedavg_what bit mask */
 enum { FLS_KERNEL_REDUCE = 0, FLS_KERNEL_ADAMW = 1, FLS_KERNEL_FEDAVG = 2, FLS_KERNEL_ADAMW_FEDAVG = 3, FLS_KERNEL_COUNT = 4 };
-enum { FLS_STATUS_NONFINITE_NORM = 1, FLS_STATUS_STAGING_TIMEOUT = 2 }; /* sticky bits of the device status word */
+enum { FLS_STATUS_NONFINITE_NORM = 1 }; /* sticky bits of the device status word */
 
 #define FLS_MAX_GROUPS 64        /* G <= 64 */
 #define FLS_MAX_GRAD_BUFFERS 64  /* K = shard_dim * replicate_dim <= 64 */
@@ -218,14 +218,6 @@ int fls_comm_report(const fls_plan* plan, const double* bw_bytes_per_s, fls_comm
  * the direction in which those two kernels walk the tiles, negative keeps it.  The reduce kernel has one
  * launch shape and ignores both. */
 int fls_plan_tune(fls_plan* plan, uint32_t kernel, int ctas_per_sm, int descending);
-
-/* enabled != 0: the reduce kernel stages each tile of the K gradient buffers through shared memory with bulk
- * asynchronous copies (cp.async.bulk + mbarrier) instead of loading it into registers.  Applies only to bf16
- * gradients in the flat order with K = 8 on a layout whose every segment is 8-element aligned (otherwise the
- * call returns FLS_ESTATE and nothing changes).  Off by default: it measured no faster than the plain kernel;
- * it is kept so that this can be re-measured.  Results are identical.  Its wait on the copies is bounded: on
- * expiry FLS_STATUS_STAGING_TIMEOUT is set in the status word and the affected tile is left unwritten. */
-int fls_plan_set_staging(fls_plan* plan, int enabled);
 
 /* How fls_sync_step gets the mean gradient into AdamW.  With fewer than 8 gradient bytes per element (bf16 and
  * K <= 3, fp32 and K = 1) reading the gradients twice (a norm pass, then AdamW forming the mean itself: 2*K*e_g +

@@ -15,7 +15,7 @@ FLS_GRAD_BF16, FLS_GRAD_F32 = 0, 1
 FLS_WIRE_F32, FLS_WIRE_BF16 = 0, 1
 FLS_AVG_PARAMS, FLS_AVG_OPT_STATE, FLS_AVG_FUSED = 1, 2, 4
 FLS_KERNEL_REDUCE, FLS_KERNEL_ADAMW, FLS_KERNEL_FEDAVG, FLS_KERNEL_ADAMW_FEDAVG, FLS_KERNEL_COUNT = 0, 1, 2, 3, 4
-FLS_STATUS_NONFINITE_NORM, FLS_STATUS_STAGING_TIMEOUT = 1, 2
+FLS_STATUS_NONFINITE_NORM = 1
 FLS_MAX_GROUPS = 64
 FLS_MAX_GRAD_BUFFERS = 64
 FLS_MAX_FUSED_GROUPS = 16
@@ -26,7 +26,7 @@ EXPORTS = [
     "fls_plan_create", "fls_plan_query", "fls_plan_bind", "fls_sync_step", "fls_sync_step_host", "fls_fedavg",
     "fls_sync_step_fedavg", "fls_fedavg_outer",
     "fls_get_norms", "fls_get_reduced_grad", "fls_get_status", "fls_get_step", "fls_set_step", "fls_comm_report",
-    "fls_plan_tune", "fls_plan_set_staging", "fls_plan_set_recompute", "fls_plan_set_single_pass", "fls_plan_set_overlap", "fls_set_profiling", "fls_get_kernel_ms", "fls_get_launch_count", "fls_plan_destroy",
+    "fls_plan_tune", "fls_plan_set_recompute", "fls_plan_set_single_pass", "fls_plan_set_overlap", "fls_set_profiling", "fls_get_kernel_ms", "fls_get_launch_count", "fls_plan_destroy",
     "fls_last_error", "fls_reduce_norm_noalloc",
 ]
 
@@ -92,7 +92,6 @@ def _load() -> C.CDLL:
     lib.fls_set_step.argtypes = [P, C.c_uint64]
     lib.fls_comm_report.argtypes = [P, C.POINTER(C.c_double), C.POINTER(fls_comm_costs)]
     lib.fls_plan_tune.argtypes = [P, C.c_uint32, C.c_int, C.c_int]
-    lib.fls_plan_set_staging.argtypes = [P, C.c_int]
     lib.fls_plan_set_recompute.argtypes = [P, C.c_int]
     lib.fls_plan_set_single_pass.argtypes = [P, C.c_int]
     lib.fls_plan_set_overlap.argtypes = [P, C.c_int]
@@ -249,10 +248,6 @@ def fls_comm_report(plan: int, bw_bytes_per_s: Optional[Sequence[float]] = None)
 
 def fls_plan_tune(plan: int, kernel: int, ctas_per_sm: int = 0, descending: int = -1) -> None:
     _check(lib.fls_plan_tune(plan, kernel, ctas_per_sm, descending))
-
-
-def fls_plan_set_staging(plan: int, enabled: bool) -> None:
-    _check(lib.fls_plan_set_staging(plan, int(enabled)))
 
 
 def fls_plan_set_recompute(plan: int, mode: int) -> None:

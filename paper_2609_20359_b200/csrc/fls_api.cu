@@ -63,7 +63,6 @@ struct fls_plan {
   int descending[FLS_KERNEL_COUNT] = {0, 1, 0, 1};   // AdamW starts where the reduce kernel stopped: those lines are still in L2
 
   bool overlap = true;     // programmatic dependent launch between the kernels of one call
-  bool staged_reduce = false;
   bool recompute = false;  // K * e_g < 8: the norm pass stores nothing and AdamW forms the mean gradient again
   bool single_pass = false;  // no clipping: reduce + norm + AdamW in one kernel
   bool profiling = false;
@@ -208,9 +207,7 @@ int run_group(fls_plan* p, uint32_t g, double lr, uint64_t t_new, cudaStream_t s
     if (e1 != cudaSuccess) return cuda_fail(e1, "single-pass step kernel launch");
     return FLS_OK;
   }
-  cudaError_t e = timed_launch(p, FLS_KERNEL_REDUCE, st, [&] {
-    return p->staged_reduce ? launch_reduce_staged(ra, st, overlap && chain) : launch_reduce(ra, f32, p->reduce_sg, st, overlap && chain);
-  });
+  cudaError_t e = timed_launch(p, FLS_KERNEL_REDUCE, st, [&] { return launch_reduce(ra, f32, p->reduce_sg, st, overlap && chain); });
   if (e != cudaSuccess) return cuda_fail(e, "reduce kernel launch");
   if (!with_adamw) return FLS_OK;
 
@@ -631,16 +628,6 @@ int fls_plan_tune(fls_plan* p, uint32_t kernel, int ctas_per_sm, int descending)
   if (ctas_per_sm > 0) p->ctas_per_sm[kernel] = std::min(ctas_per_sm, 1 << 16);
   if (ctas_per_sm == -2) p->ctas_per_sm[kernel] = 0;   // back to the default: one pass, the grid covers every tile
   if (descending >= 0) p->descending[kernel] = descending ? 1 : 0;
-  return FLS_OK;
-}
-
-int fls_plan_set_staging(fls_plan* p, int enabled) {
-  if (!p) return fail(FLS_EINVAL, "fls_plan_set_staging: null plan");
-  if (enabled) {
-    const bool ok = p->desc.grad_dtype == FLS_GRAD_BF16 && p->reduce_sg == 0 && p->K == 8 && p->lay.vector_path;
-    if (!ok) return fail(FLS_ESTATE, "fls_plan_set_staging: needs bf16 gradients, flat order, K = 8 and 8-element aligned segments");
-  }
-  p->staged_reduce = enabled != 0;
   return FLS_OK;
 }
 

@@ -473,79 +473,6 @@ __global__ void __launch_bounds__(THREADS, MINB) fls_reduce_kernel(const __grid_
 }
 
 // ------------------------------------------------------------------------------------------------
-// K1, staged variant (optional, off by default): the K = 8 bf16 tiles of a CTA travel to shared memory
-// as eight bulk asynchronous copies (cp.async.bulk, no tensor map, no multicast) that complete on one
-// mbarrier; the threads then read their 8 x 16 bytes from shared memory.  It exists so that the choice
-// "plain loads, no staging" stays a measured one: on the same workloads it is no faster than the
-// kernel above (the numbers are in the design notes), so nothing selects it unless asked to.
-// Preconditions (checked by the launcher's caller): bf16 gradients, flat order (SG = 0), K = 8, every
-// segment 8-element aligned with a length that is a multiple of 8 (16-byte bulk copies).
-// The wait on the mbarrier is bounded; on expiry the CTA sets a status bit, skips its tile and exits.
-// ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return uint32_t(__cvta_generic_to_shared(p)); }
-
-__global__ void __launch_bounds__(kThreads, 5) fls_reduce_staged_kernel(const __grid_constant__ ReduceArgs a) {
-  __shared__ __align__(128) uint16_t stage[8][kTile];   // 32 KiB: one tile of each buffer
-  __shared__ __align__(8) uint64_t bar;
-  float sq = 0.f;
-  const uint32_t tile = blockIdx.x;
-  const Segment* sg = a.idx.segs + find_segment(a.idx, tile);
-  const uint64_t t0 = (uint64_t(tile) - __ldg(&sg->tile_begin)) * kTile;     // first element of the tile in its segment
-  const uint64_t len = __ldg(&sg->len);
-  const uint32_t n_valid = uint32_t(len - t0 < kTile ? len - t0 : kTile);    // a multiple of 8 by precondition
-  const uint64_t j0 = __ldg(&sg->j0) + t0, a0 = __ldg(&sg->a0) + t0;
-  if (threadIdx.x == 0) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(&bar)));
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    const uint32_t bytes = n_valid * 2;
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(smem_u32(&bar)), "r"(8 * bytes) : "memory");
-#pragma unroll
-    for (int k = 0; k < 8; ++k)
-      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                   :: "r"(smem_u32(&stage[k][0])), "l"(static_cast<const uint16_t*>(a.grad[k]) + j0), "r"(bytes), "r"(smem_u32(&bar))
-                   : "memory");
-  }
-  // bounded wait for the eight copies (phase 0 of the barrier)
-  bool arrived = false;
-  for (uint32_t spin = 0; spin < (1u << 22) && !arrived; ++spin) {
-    uint32_t ok;
-    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n selp.u32 %0, 1, 0, p;\n}\n"
-                 : "=r"(ok) : "r"(smem_u32(&bar)) : "memory");
-    arrived = ok != 0;
-  }
-  if (!arrived) {
-    if (threadIdx.x == 0) atomicOr(a.status, uint32_t(FLS_STATUS_STAGING_TIMEOUT));
-  } else {
-    const uint32_t e0 = threadIdx.x * kVec;
-    if (e0 < n_valid) {
-      float acc[8];
-#pragma unroll
-      for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-#pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        Raw<8, false> raw;
-        raw.r = *reinterpret_cast<const uint4*>(&stage[k][e0]);
-        float x[8];
-        unpack(raw, x);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) acc[e] += x[e];
-      }
-      F8 o;
-#pragma unroll
-      for (int e = 0; e < 8; ++e) { o.v[e] = acc[e] * a.inv_k; sq = fmaf(o.v[e], o.v[e], sq); }
-      dep_wait();
-      st8_keep(a.gbar + a0 + e0, o);
-    }
-  }
-  dep_wait();
-  dep_launch();
-  finish_norm<kThreads>(a, sq);
-}
-
-// ------------------------------------------------------------------------------------------------
 // K2: clip + AdamW + bf16 copy.
 // ------------------------------------------------------------------------------------------------
 __device__ __forceinline__ void adamw_one(const AdamArgs& a, float c, float gbar, float& th, float& m, float& v) {
@@ -949,11 +876,6 @@ void launch_reduce_t(const ReduceArgs& a, int sg, unsigned grid, cudaStream_t st
 unsigned reduce_grid(const ReduceArgs& a, int sg, bool f32) {
   const unsigned tiles_per_cta = reduce_tiles_per_cta(a, sg, f32);
   return (a.idx.n_tiles + tiles_per_cta - 1) / tiles_per_cta;
-}
-
-cudaError_t launch_reduce_staged(const ReduceArgs& a, cudaStream_t st, bool overlap) {
-  launch_k(fls_reduce_staged_kernel, a, a.idx.n_tiles, kThreads, st, overlap);
-  return cudaGetLastError();
 }
 
 cudaError_t launch_reduce(const ReduceArgs& a, bool f32, int sg, cudaStream_t st, bool overlap) {

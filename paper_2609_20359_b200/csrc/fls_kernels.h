@@ -90,8 +90,6 @@ unsigned reduce_grid(const ReduceArgs& a, int sg, bool f32);
 // overlap: launch with programmatic stream serialization, so that the kernel's first CTAs may start during
 // the tail of the kernel launched just before it on the same stream (which must be one of these three).
 cudaError_t launch_reduce(const ReduceArgs& a, bool f32, int sg, cudaStream_t st, bool overlap);
-// Shared-memory staged variant of the reduce kernel (bf16, flat order, K = 8, fully vectorisable layout only).
-cudaError_t launch_reduce_staged(const ReduceArgs& a, cudaStream_t st, bool overlap);
 cudaError_t launch_step_noclip(const ReduceAdamArgs& a, bool f32, int sg, cudaStream_t st, bool overlap);
 cudaError_t launch_reduce_adamw(const ReduceAdamArgs& a, bool f32, int sg, unsigned grid, cudaStream_t st, bool overlap);
 cudaError_t launch_adamw(const AdamArgs& a, unsigned grid, cudaStream_t st, bool overlap);

@@ -25,7 +25,9 @@ def test_reference_arm_line():
     assert BASE_KEYS <= set(d) and d["impl"] == "reference"
     assert d["metric"] == "synced_params_per_s" and d["unit"] == "params/s" and d["higher_is_better"] is True
     assert d["vs_baseline"] is None and d["data"] == "synthetic" and d["config"]["workload"] == "tiny_fl_fsdp"
-    assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] == 1 and d["cpu_baseline"]["value"] == d["value"]
+    cb = d["cpu_baseline"]
+    assert cb["kind"] == "oracle" and cb["cores"] == cb["host_cores"] >= 1 and cb["value"] == d["value"]
+    assert cb["one_core"]["cores"] == 1 and cb["one_core"]["value"] > 0
     assert d["e2e"] == {"value": d["value"], "unit": d["unit"], "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
     assert d["value"] > 0
 
@@ -43,6 +45,8 @@ def test_own_arm_line():
     assert e["value"] > 0 and e["h2d_bytes_per_step"] == 2 * 4 * 1_000_032 * 2 and e["d2h_bytes_per_step"] == 8
     assert e["value"] < d["value"]                       # copies inside the timed region can only slow it down
     c = d["cpu_baseline"]
-    assert c["kind"] == "oracle" and c["cores"] == 1 and c["value"] > 0 and c["sample"]
+    assert c["kind"] == "oracle" and c["cores"] >= 1 and c["value"] > 0 and c["sample"]
+    assert c["one_core"]["cores"] == 1 and c["one_core"]["value"] > 0
+    assert "other_workloads" not in d                    # only the default workload brings the other two along
     # value = G * P * steps / time
     assert abs(d["value"] - 2 * 1_000_003 * 8 / (d["ms_per_step"] * 8 / 1e3)) / d["value"] < 1e-6

@@ -165,28 +165,6 @@ def test_single_pass_without_clipping(fls, units, G, S, R_rep, Q, dtype):
     c.close()
 
 
-def test_staged_reduce_variant_is_bit_identical(fls):
-    """The shared-memory staged reduce kernel (bulk asynchronous copies) against the default kernel: same bits,
-    ragged last tiles included; it refuses plans it does not cover."""
-    def run(staged):
-        c = Case([40000, 30008, 8], 2, 8, 1, H=2, Q=8, hp=orc.Hyper(max_grad_norm=0.05))
-        if staged:
-            fls.fls_plan_set_staging(c.sess.plan, True)
-        for _ in range(2):
-            c.step([2, 1])
-            c.compare()
-        assert c.sess.status() == 0
-        out = [c.sess.reduced_grad().clone()] + [x.clone() for x in c.sess.master + c.sess.v + c.sess.param_bf16] + [c.sess.norms().clone()]
-        c.close()
-        return out
-    assert all(torch.equal(x, y) for x, y in zip(run(False), run(True)))
-    c = Case([40000], 1, 4, 2, H=2, Q=8)                     # two-level order: not covered
-    with pytest.raises(fls.FlsError) as e:
-        fls.fls_plan_set_staging(c.sess.plan, True)
-    assert e.value.code == fls.FLS_ESTATE
-    c.close()
-
-
 def test_reduced_gradient_matches_oracle_exactly_for_bf16(fls):
     """With bf16 inputs of similar magnitude the fp32 running sum is exact, so the mean gradient is
     bit-identical to the oracle's (this case is small enough that no element loses bits)."""
@@ -590,19 +568,28 @@ def _oracle_norm_full(grads, S, R_rep, chunk=1 << 22, threads=16):
     return math.sqrt(math.fsum(parts))
 
 
+def _sample_grads(cfg, tidx, step, g, K):
+    """The K gradient buffers of (step, group) at the sampled logical positions, as exact float64 values."""
+    return [orc.bf16_bits_to_f64(bf16_bits(sy.normal_at(tidx, sy.stream_key(cfg["seed"], sy.KIND_GRAD, step, g, k), cfg["grad_sigma"],
+                                                        sy.uniform_scale(cfg["seed"], g, k) if cfg["per_buffer_scale"] else 1.0,
+                                                        torch.bfloat16))) for k in range(K)]
+
+
 @pytest.mark.parametrize("cfg_index", [1, 2, 3])
 def test_full_size_workloads_sampled(fls, cfg_index):
     """The GPT-2-small, Llama-3.2-1B (18 units, two-level order) and Llama-3.1-8B-block (9 tensors) workloads at
-    full size, launched as the benchmark launches them.  The oracle computes every group's norm over the full
-    gradient, then the step and FedAvg at sampled logical positions: the first and last 4096 parameters, 16
-    around every unit and shard boundary, and 200,000 random ones."""
+    full size on the route the benchmark times: a plan with the fused aggregation, a plain step through
+    fls_sync_step, then -- with fresh gradients, so that non-zero m and v enter AdamW -- an aggregation step through
+    fls_sync_step_fedavg (the sync period is set to 2 for this).  The oracle computes every group's norm over the
+    full gradient of both steps, then the steps and FedAvg at sampled logical positions: the first and last 4096
+    parameters, 16 around every unit and shard boundary, and 200,000 random ones."""
     from paper_2609_20359_b200.session import Session
     cfg = sy.CONFIGS[cfg_index]
     P, G, S, R_rep = cfg["n_params"], cfg["groups"], cfg["shard_dim"], cfg["replicate_dim"]
     K = S * R_rep
     hp = orc.Hyper()
     L = orc.plan(cfg["unit_numel"], S, 8)
-    s = Session(P, cfg["unit_numel"], G, S, R_rep, cfg["sync_period"], "bf16", 8, False)
+    s = Session(P, cfg["unit_numel"], G, S, R_rep, 2, "bf16", 8, False, fused=True)
     assert s.n_padded == L.n_padded
     _fill_full_size(s, cfg, L)
     counts = [sy.sample_count(cfg["seed"], g) for g in range(G)] if cfg["weights"] == "counts" else None
@@ -617,41 +604,52 @@ def test_full_size_workloads_sampled(fls, cfg_index):
     jt, at = torch.from_numpy(j_np).cuda(), torch.from_numpy(a_np).cuda()
     th0 = sy.normal_at(tidx, sy.stream_key(cfg["seed"], sy.KIND_MASTER), cfg["master_sigma"]).numpy()
     assert np.array_equal(s.master[0][at].cpu().numpy(), th0)            # the fill put every sample where the oracle's planner says
-    norms, gbar_s, samp_last = [], [], None
-    for g in range(G):
-        norms.append(_oracle_norm_full(s.grads[g], S, R_rep))
-        samp = [orc.bf16_bits_to_f64(bf16_bits(sy.normal_at(tidx, sy.stream_key(cfg["seed"], sy.KIND_GRAD, 1, g, k), cfg["grad_sigma"],
-                                                             sy.uniform_scale(cfg["seed"], g, k) if cfg["per_buffer_scale"] else 1.0,
-                                                             torch.bfloat16))) for k in range(K)]
-        gbar_s.append(orc.reduce_mean(samp, S, R_rep))
-        samp_last = samp
-    due = s.step()
+    z = np.zeros(idx.size, np.float32)
+    states = [orc.GroupState(th0.copy(), z.copy(), z.copy(), orc.f32_to_bf16_bits(th0)) for _ in range(G)]
+
+    def oracle_step(t):
+        norms, samp_last, gb_last = [], None, None
+        for g in range(G):
+            norms.append(_oracle_norm_full(s.grads[g], S, R_rep))
+            samp_last = _sample_grads(cfg, tidx, t, g, K)
+            gb_last = orc.reduce_mean(samp_last, S, R_rep)
+            c = orc.clip_coef(norms[g], hp.max_grad_norm)
+            assert c < 1.0
+            st = states[g]
+            st.theta, st.m, st.v, st.param_bf16 = orc.adamw(st.theta, st.m, st.v, gb_last, c, t, hp.lr, hp.beta1, hp.beta2, hp.eps,
+                                                           hp.weight_decay)
+        return norms, samp_last, gb_last
+
+    def check_state(tag):
+        for g in range(G):
+            assert_state_close(s.master[g][at].cpu().numpy(), states[g].theta, f"{tag} master[{g}]")
+            assert_state_close(s.m[g][at].cpu().numpy(), states[g].m, f"{tag} m[{g}]", 1e-5, "rms")
+            assert_state_close(s.v[g][at].cpu().numpy(), states[g].v, f"{tag} v[{g}]", 1e-5, "rms")
+            assert_bf16_close(bf16_bits(s.param_bf16[g][jt]), states[g].param_bf16, f"{tag} bf16[{g}]")
+
+    # step 1: plain step of every group
+    norms, samp_last, gb_last = oracle_step(1)
+    assert not s.step()
     torch.cuda.synchronize()
-    assert not due
     got_n = s.norms().cpu().numpy().astype(np.float64)
     assert np.allclose(got_n, norms, rtol=1e-6, atol=0), (got_n, norms)
     # fp32 running sum against the exactly rounded mean: identical except where a tiny addend loses bits
     got_g = s.reduced_grad()[at].cpu().numpy()
-    assert np.mean(got_g == gbar_s[G - 1]) > 0.999
-    assert np.all(np.abs(got_g.astype(np.float64) - gbar_s[G - 1]) <= 2.0 ** -24 * np.sum(np.abs(samp_last), axis=0))
-    states = []
-    for g in range(G):
-        c = orc.clip_coef(norms[g], hp.max_grad_norm)
-        assert c < 1.0
-        z = np.zeros(idx.size, np.float32)
-        th, m, v, bits = orc.adamw(th0, z, z, gbar_s[g], c, 1, hp.lr, hp.beta1, hp.beta2, hp.eps, hp.weight_decay)
-        states.append(orc.GroupState(th, m, v, bits))
-        assert_state_close(s.master[g][at].cpu().numpy(), th, f"master[{g}]")
-        assert_state_close(s.m[g][at].cpu().numpy(), m, f"m[{g}]", 1e-5, "rms")
-        assert_state_close(s.v[g][at].cpu().numpy(), v, f"v[{g}]", 1e-5, "rms")
-        assert_bf16_close(bf16_bits(s.param_bf16[g][jt]), bits, f"bf16[{g}]")
+    assert np.mean(got_g == gb_last) > 0.999
+    assert np.all(np.abs(got_g.astype(np.float64) - gb_last) <= 2.0 ** -24 * np.sum(np.abs(samp_last), axis=0))
+    check_state("step 1")
+    # step 2: new gradients, the step and the aggregation in the one fused call
+    _fill_grads_full_size(s, cfg, L, 2)
+    norms, _, _ = oracle_step(2)
     orc.fedavg(states, counts)
-    s.fedavg(counts)
+    s.step_fedavg(counts)
     torch.cuda.synchronize()
-    for g in range(G):
-        assert_state_close(s.master[g][at].cpu().numpy(), states[g].theta, f"fedavg master[{g}]")
-        assert_bf16_close(bf16_bits(s.param_bf16[g][jt]), states[g].param_bf16, f"fedavg bf16[{g}]")
+    assert s.t == 2
+    got_n = s.norms().cpu().numpy().astype(np.float64)
+    assert np.allclose(got_n, norms, rtol=1e-6, atol=0), (got_n, norms)
+    check_state("step 2 + FedAvg")
     assert torch.equal(s.master[0], s.master[G - 1]) and torch.equal(s.param_bf16[0], s.param_bf16[G - 1])
+    assert not torch.equal(s.m[0], s.m[G - 1])                            # parameters only: every group keeps its own moments
     assert s.status() == 0
     s.close()
 

@@ -1,7 +1,9 @@
-"""The only multi-rank logic of the benchmark (replicas only: no data-path collective) is the timing
-aggregation: the job's time is the slowest rank's.  Checked with two gloo ranks on CPU."""
+"""The only multi-rank logic of the benchmark (replicas only: no data-path collective) is starting the ranks
+and the timing aggregation: the job's time is the slowest rank's.  Checked with two gloo ranks on CPU."""
+import json
 import os
 import socket
+import subprocess
 import sys
 
 import torch
@@ -57,3 +59,29 @@ def test_reference_arm_runs_on_rank0_only(capsys, monkeypatch):
     class A: steps, warmup, gpus = 1, 0, 2
     bench.run_reference(A, sy.config_by_name("tiny_fl_fsdp"))
     assert capsys.readouterr().out == ""
+
+
+def test_gpus_flag_starts_the_ranks_itself():
+    """`bench.py --gpus 2` without a launcher re-runs itself as two ranks; with the stub workload (no GPU) rank r
+    takes 10*(r+1) ms per step, so the line must report two ranks and the slower rank's time."""
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--stub-workload", "--steps", "3", "--warmup", "3"],
+                         capture_output=True, text=True, cwd=ROOT, env=env, timeout=300)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1, out.stdout[-2000:]
+    d = json.loads(lines[0])
+    assert d["n_gpus"] == 2 and d["config"]["parallelism"] == "replicas only" and d["steps"] == 3
+    assert abs(d["ms_per_step"] - 20.0) < 1e-9 and abs(d["value"] - 2 * 1000 * 3 / 0.060) < 1e-6
+
+
+def test_under_a_launcher_the_flag_does_not_spawn_again(monkeypatch):
+    sys.path.insert(0, ROOT)
+    import bench
+    called = []
+    monkeypatch.setattr(bench, "spawn_ranks", lambda n, argv: called.append(n) or 0)
+    monkeypatch.setattr(bench, "run_stub", lambda args: called.append("stub"))
+    monkeypatch.setenv("WORLD_SIZE", "2")
+    monkeypatch.setattr(sys, "argv", ["bench.py", "--gpus", "2", "--stub-workload"])
+    bench.main()
+    assert called == ["stub"]
