@@ -140,7 +140,7 @@ int fls_plan_query(const fls_plan* plan, fls_layout* out);
  * FLS_ECUDA. */
 int fls_plan_bind(fls_plan* plan, const fls_buffers* buffers);
 
-/* One local training step of all G groups ("each federation group proceeds independently"), enqueued
+/* One local training step of all G groups (the groups train without waiting for one another), enqueued
  * on `cuda_stream` (a cudaStream_t; NULL = default stream).  Per group: mean of the K gradient buffers
  * in fp32, ascending buffer order inside a sharding group, then ascending replica order (reduce-scatter
  * over S, then all-reduce over R: Background FSDP/HSDP, Eq. 2), one multiply by 1/K; L2 norm of the mean
@@ -159,17 +159,17 @@ int fls_sync_step(fls_plan* plan, double lr, void* cuda_stream, int* fedavg_due)
 int fls_sync_step_host(fls_plan* plan, const void* const* host_grads, double lr, void* cuda_stream,
                        float* host_norms, int* fedavg_due);
 
-/* FedAvg: every group's parameters become sum_g w_g x_g, w_g = n_g / sum n ("a weighted average of all
- * locally trained models"; shard by shard across the federation groups, after which every shard equals
- * the average of its counterparts).  fp32 accumulation in ascending group order; all G master copies and
+/* FedAvg: every group's parameters become sum_g w_g x_g, w_g = n_g / sum n (the weighted mean of the
+ * locally trained models of Background "Federated Learning", taken shard by shard across the federation
+ * groups, Section FL+FSDP).  fp32 accumulation in ascending group order; all G master copies and
  * all G bf16 copies are rewritten; m and v too if the plan has FLS_AVG_OPT_STATE.  sample_counts: host,
  * G entries, NULL = equal weights.  The step counter is unchanged.
  * Errors: FLS_EINVAL if all counts are zero, FLS_ESTATE, FLS_ECUDA. */
 int fls_fedavg(fls_plan* plan, const uint64_t* sample_counts, void* cuda_stream);
 
 /* Aggregation with an outer optimizer (the FedOpt family of the paper's related work: AdamW inside the groups,
- * SGD with optional Nesterov momentum across them; "FedAvg as a base aggregation strategy, enabling easy
- * integration of more complex ones").  With xbar = sum_g w_g x_g as in fls_fedavg:
+ * SGD with optional Nesterov momentum across them; the paper presents FedAvg as the base strategy that others
+ * can replace).  With xbar = sum_g w_g x_g as in fls_fedavg:
  *   delta = x_global - xbar;  buf = momentum*buf + delta;  d = nesterov ? delta + momentum*buf : buf;
  *   x_global -= outer_lr * d;  every group's master = x_global, every bf16 copy = bf16(x_global).
  * outer_lr = 1, momentum = 0 is plain FedAvg (up to fp32 rounding of x - (x - xbar)).  global_params and
@@ -182,8 +182,8 @@ int fls_fedavg_outer(fls_plan* plan, const uint64_t* sample_counts, double outer
                      float* global_params, float* outer_momentum, void* cuda_stream);
 
 /* One local step of all groups immediately followed by FedAvg, i.e. exactly fls_sync_step then fls_fedavg
- * (same results bit for bit), for the steps on which aggregation is due ("after the local update every A
- * training steps").  With FLS_AVG_FUSED in the plan and G <= FLS_MAX_FUSED_GROUPS the aggregation is fused
+ * (same results bit for bit), for the steps on which aggregation is due (every A-th step, after
+ * its optimizer update).  With FLS_AVG_FUSED in the plan and G <= FLS_MAX_FUSED_GROUPS the aggregation is fused
  * into the optimizer kernel: after the G reductions one kernel applies AdamW to every group's element,
  * averages the G results in registers and writes the average to all G copies, which saves FedAvg's own
  * read and write of the parameters (10*G bytes per parameter).  Otherwise it runs the two calls one after the

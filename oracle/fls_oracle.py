@@ -19,7 +19,7 @@ The paper defines the communication pattern, not the arithmetic:
     average of the corresponding shards of all groups (Section "Augmenting
     Sharded DP Through FL"; FedAvg as described in Background, "Federated
     Learning").
-  * Optimiser: "AdamW, learning rate 3e-4", bf16 training (Experimental Setup).
+  * Optimiser: AdamW with learning rate 3e-4, training in bf16 (Experimental Setup).
   * Cost model: Table of symbols and Eq. 1-5.
 Everything numeric that the paper does not state (mean vs sum, order, clipping
 rule, AdamW variant, rounding) follows the readings listed beside each function.
@@ -146,7 +146,49 @@ def round_to_bf16(x: np.ndarray) -> np.ndarray:
     return bf16_bits_to_f64(f32_to_bf16_bits(np.asarray(x, dtype=np.float64).astype(np.float32)))
 
 
-def reduce_mean(grads: Sequence[np.ndarray], S: int, R_rep: int = 1, wire_bf16: bool = False) -> np.ndarray:
+def ring_positions(L: Layout, R_rep: int):
+    """For every logical element: (s, c) = the rank that ends up owning it after the reduce-scatter over the S
+    ranks of a sharding group, and the sub-chunk of that rank's slice it falls in when the slice is cut into
+    R_rep equal parts for the ring all-reduce across the replicas.  Element i of unit u: s = i div M_u; its
+    position inside the slice is p = i mod M_u and c = p div ceil(M_u / R_rep)."""
+    s_all, c_all = [], []
+    for n, M in zip(L.unit_numel, L.unit_shard_numel):
+        i = np.arange(n, dtype=np.int64)
+        sub = -(-M // R_rep)
+        s_all.append(i // M)
+        c_all.append((i % M) // sub)
+    return np.concatenate(s_all), np.concatenate(c_all)
+
+
+def ring_order(owner: int, n: int) -> List[int]:
+    """Order in which a ring reduce-scatter over n ranks adds the contributions to the chunk that rank `owner`
+    ends up with: the chunk starts on the next rank and travels once around the ring, every rank adding its own
+    part, so the owner's part is added last: owner+1, owner+2, ..., n-1, 0, ..., owner."""
+    return [(owner + 1 + q) % n for q in range(n)]
+
+
+def _sum_levels(grads, S: int, R_rep: int, sigma_order, rho_order, wire_bf16: bool) -> np.ndarray:
+    """Two-level sum in the given visiting orders, then one division by K; fp32 result."""
+    K = S * R_rep
+    if wire_bf16:
+        outer = np.zeros_like(np.asarray(grads[0], dtype=np.float64))
+        for rho in rho_order:
+            inner = np.zeros_like(outer)
+            for sigma in sigma_order:
+                inner = round_to_bf16((inner + np.asarray(grads[rho * S + sigma], dtype=np.float64)).astype(np.float32))
+            outer = round_to_bf16((outer + inner).astype(np.float32))
+        return round_to_bf16((outer / K).astype(np.float32)).astype(np.float32)
+    outer = None
+    for rho in rho_order:
+        inner = None
+        for sigma in sigma_order:
+            x = np.asarray(grads[rho * S + sigma], dtype=np.float64)
+            inner = x.copy() if inner is None else inner + x
+        outer = inner if outer is None else outer + inner
+    return (outer / K).astype(np.float32)
+
+
+def reduce_mean(grads: Sequence[np.ndarray], S: int, R_rep: int = 1, wire_bf16: bool = False, ring=None) -> np.ndarray:
     """Mean gradient of one group, stored as fp32.
 
     grads: K = R_rep*S float64 arrays (exact input values), buffer rho*S+sigma.
@@ -160,25 +202,25 @@ def reduce_mean(grads: Sequence[np.ndarray], S: int, R_rep: int = 1, wire_bf16: 
     bfloat16 and it attributes HSDP's different result to the order of floating-point
     operations): every partial sum and the final mean are rounded to bf16, so the
     two orders give different numbers.  Both levels start from zero, as on the GPU.
+
+    ring: None visits the buffers in ascending index at both levels.  Otherwise the pair of integer arrays
+    `ring_positions` returns (owner rank s and all-reduce sub-chunk c of every element): the order a ring
+    produces.  The shard level adds sigma = s+1, s+2, ..., s (mod S); the replicate level, a ring all-reduce
+    (reduce-scatter of R_rep sub-chunks, then all-gather), adds rho = c+1, ..., c (mod R_rep).  The sums are the
+    same mathematically; with bf16 partial sums the start of the ring changes the rounding.
     """
     K = len(grads)
     assert K == S * R_rep and K >= 1
-    if wire_bf16:
-        outer = np.zeros_like(np.asarray(grads[0], dtype=np.float64))
-        for rho in range(R_rep):
-            inner = np.zeros_like(outer)
-            for sigma in range(S):
-                inner = round_to_bf16((inner + np.asarray(grads[rho * S + sigma], dtype=np.float64)).astype(np.float32))
-            outer = round_to_bf16((outer + inner).astype(np.float32))
-        return round_to_bf16((outer / K).astype(np.float32)).astype(np.float32)
-    outer = None
-    for rho in range(R_rep):
-        inner = None
-        for sigma in range(S):
-            x = np.asarray(grads[rho * S + sigma], dtype=np.float64)
-            inner = x.copy() if inner is None else inner + x
-        outer = inner if outer is None else outer + inner
-    return (outer / K).astype(np.float32)
+    if ring is None:
+        return _sum_levels(grads, S, R_rep, range(S), range(R_rep), wire_bf16)
+    s_idx, c_idx = ring
+    out = np.zeros(np.asarray(grads[0]).shape, np.float32)
+    for s in range(S):
+        for c in range(R_rep):
+            sel = (s_idx == s) & (c_idx == c)
+            if sel.any():
+                out[sel] = _sum_levels([np.asarray(g)[sel] for g in grads], S, R_rep, ring_order(s, S), ring_order(c, R_rep), wire_bf16)
+    return out
 
 
 def grad_norm(gbar: np.ndarray) -> float:
@@ -238,14 +280,16 @@ class Hyper:
     weight_decay: float = 0.1
     max_grad_norm: float = 1.0
     wire_bf16: bool = False        # bf16 emulation of the two reduction levels (see reduce_mean)
+    ring: bool = False             # visit the buffers in the order a ring produces (see reduce_mean)
 
 
 def sync_step_group(st: GroupState, grads: Sequence[np.ndarray], S: int, R_rep: int, t_new: int,
-                    hp: Hyper, lr: Optional[float] = None):
+                    hp: Hyper, lr: Optional[float] = None, ring=None):
     """One local step of one group: reduce -> norm -> clip -> AdamW.  Returns
-    (norm, coef, gbar).  Each group "proceeds independently of the others"
-    (Section FL+FSDP)."""
-    gbar = reduce_mean(grads, S, R_rep, hp.wire_bf16)
+    (norm, coef, gbar).  Every federation group runs its steps on its own, without
+    waiting for the others (Section FL+FSDP).  `ring`: see reduce_mean (needed when hp.ring)."""
+    assert (ring is not None) == bool(hp.ring)
+    gbar = reduce_mean(grads, S, R_rep, hp.wire_bf16, ring)
     nrm = grad_norm(gbar)
     c = clip_coef(nrm, hp.max_grad_norm)
     st.theta, st.m, st.v, st.param_bf16 = adamw(
@@ -265,8 +309,8 @@ def fedavg_weights(sample_counts: Optional[Sequence[int]], G: int) -> np.ndarray
 
 def fedavg_array(copies: Sequence[np.ndarray], w: np.ndarray) -> np.ndarray:
     """Weighted average of G corresponding copies, double accumulate in ascending
-    group order, stored as fp32 (FedAvg: "a weighted average of all locally trained
-    models"; shard by shard over the F groups)."""
+    group order, stored as fp32 (FedAvg combines the locally trained models into one by a
+    weighted mean, Background "Federated Learning"; here shard by shard over the F groups)."""
     acc = None
     for g, x in enumerate(copies):
         term = w[g] * np.asarray(x, dtype=np.float32).astype(np.float64)
@@ -276,8 +320,8 @@ def fedavg_array(copies: Sequence[np.ndarray], w: np.ndarray) -> np.ndarray:
 
 def fedavg(states: Sequence[GroupState], sample_counts: Optional[Sequence[int]] = None,
            opt_state: bool = False) -> None:
-    """After aggregation "every shard is equal to the average of its corresponding
-    shards in all the other federation groups": every group receives the same
+    """After the aggregation each shard holds the mean of the shards it corresponds to in
+    the other federation groups (Section FL+FSDP): every group receives the same
     averaged parameters (and the bf16 copy of them).  Reading: w_g = n_g / sum n;
     m and v are averaged the same way only when `opt_state` is set."""
     G = len(states)
@@ -291,6 +335,35 @@ def fedavg(states: Sequence[GroupState], sample_counts: Optional[Sequence[int]] 
         s.theta = th.copy(); s.param_bf16 = bits.copy()
         if opt_state:
             s.m = m.copy(); s.v = v.copy()
+
+
+def sync_step_replicated(replicas: Sequence[GroupState], grads: Sequence[np.ndarray], S: int, R_rep: int, t_new: int,
+                         hp: Hyper, lr: Optional[float] = None, ring=None):
+    """FL+HSDP with one state copy per replica: after the shard-level reduce-scatter and the all-reduce across
+    the replicas every replica of the group holds the same mean gradient, and each applies the optimizer to its
+    own copy of the shard (Background, HSDP).  `replicas`: the R_rep state copies of one group."""
+    assert len(replicas) == R_rep
+    out = None
+    for st in replicas:
+        out = sync_step_group(st, grads, S, R_rep, t_new, hp, lr, ring)
+    return out
+
+
+def fedavg_replicated(groups: Sequence[Sequence[GroupState]], sample_counts: Optional[Sequence[int]] = None,
+                      opt_state: bool = False) -> None:
+    """FedAvg of FL+HSDP (Section FL+HSDP): only one replica of every federation group takes part in the
+    aggregation across the groups, after which it broadcasts the new parameters to the other replicas of its
+    group.  groups[g][rho]; replica 0 of each group is the one that aggregates.  The broadcast copies the
+    aggregated replica's parameters (and, with `opt_state`, its averaged m and v); without `opt_state` every
+    replica keeps the moments of its own optimizer."""
+    firsts = [reps[0] for reps in groups]
+    fedavg(firsts, sample_counts, opt_state)
+    for reps in groups:
+        src = reps[0]
+        for st in reps[1:]:
+            st.theta = src.theta.copy(); st.param_bf16 = src.param_bf16.copy()
+            if opt_state:
+                st.m = src.m.copy(); st.v = src.v.copy()
 
 
 def fedavg_outer(states: Sequence[GroupState], x_global: np.ndarray, buf: np.ndarray, sample_counts=None,
@@ -320,8 +393,8 @@ def fedavg_outer(states: Sequence[GroupState], x_global: np.ndarray, buf: np.nda
 # --------------------------------------------------------------------------- driver loop
 def run(states: List[GroupState], grads_for_step, S: int, R_rep: int, H: int, n_steps: int, hp: Hyper,
         sample_counts=None, opt_state: bool = False, t0: int = 0):
-    """for step: every group takes one local step; after every H-th step FedAvg
-    ("every A training steps", "after the local update").  grads_for_step(step, g)
+    """for step: every group takes one local step; after every H-th step FedAvg (the
+    aggregation period A of Section FL+FSDP; it follows that step's optimizer update).  grads_for_step(step, g)
     returns that group's K float64 gradient arrays (logical).  The step counter
     is global and is not reset by FedAvg.  Returns the per-step list of norms."""
     norms = []
@@ -360,7 +433,7 @@ def comm_costs(unit_shard_bytes: Sequence[float], S: int, R: int, F: int, A: int
     """Eq. 1-5 written as the sums of collectives they are defined by (the left-hand
     forms), with the uniform M*L replaced by a sum over units.  With all
     bandwidths 1 the values are bytes per step; with real bandwidths, seconds.
-    FL+HSDP with R = 1 "falls back to FL+FSDP" (Section FL+HSDP)."""
+    FL+HSDP with R = 1 costs what FL+FSDP costs (the fallback stated in Section FL+HSDP)."""
     fsdp = hsdp = fl = bc = 0.0
     for M in unit_shard_bytes:
         f = 2 * cost_all_gather(M, S, B_S) + cost_reduce_scatter(M, S, B_S)

@@ -181,6 +181,75 @@ def test_bf16_wire_makes_the_two_orders_differ():
     assert np.allclose(a, b, rtol=2 ** -5, atol=1e-5)
 
 
+def _ring_token_sum(values, owner, add):
+    """A ring reduce-scatter written as message passing: the chunk that rank `owner` will hold starts as the
+    value of the next rank, is handed from rank to rank once around the ring, and every rank it reaches adds its
+    own value with `add`; the owner is reached last."""
+    n = len(values)
+    rank = (owner + 1) % n
+    token = add(Fraction(0), values[rank])
+    while rank != owner:
+        rank = (rank + 1) % n
+        token = add(token, values[rank])
+    return token
+
+
+@pytest.mark.parametrize("S,R_rep", [(2, 1), (3, 1), (4, 1), (2, 2), (3, 2), (4, 2)])
+@pytest.mark.parametrize("wire", [True, False])
+def test_reduce_mean_ring_order_brute_force_p17(S, R_rep, wire):
+    """Ring order on P = 17 (padded shards of ceil(17/S) elements): element j belongs to rank s = j div M; inside
+    that rank's slice it lies in sub-chunk c of R_rep for the all-reduce across replicas.  The expected value is
+    the message-passing ring above in exact rationals, with the nearest-even rounding of the worked-case
+    generator after every add when the wire is bf16; with fp32 partial sums it is the exactly rounded mean."""
+    from tests.golden.make_worked_cases import _round_to_bits
+    r32 = lambda q: _round_to_bits(q, 23, -126)
+    rb = lambda q: _round_to_bits(r32(q), 7, -126)
+    rng = np.random.default_rng(500 + S * 10 + R_rep)
+    K = S * R_rep
+    bits = [rng_bf16_bits(rng, 17, 1.0) for _ in range(K)]
+    L = orc.plan([17], S, 1)
+    ring = orc.ring_positions(L, R_rep)
+    M = -(-17 // S)
+    sub = -(-M // R_rep)
+    got = orc.reduce_mean([orc.bf16_bits_to_f64(b) for b in bits], S, R_rep, wire_bf16=wire, ring=ring)
+    add = (lambda a, b: rb(a + b)) if wire else (lambda a, b: a + b)
+    for j in range(17):
+        s, c = j // M, (j % M) // sub
+        assert (ring[0][j], ring[1][j]) == (s, c)
+        per_replica = [_ring_token_sum([frac_of_bf16(bits[rho * S + sigma][j]) for sigma in range(S)], s, add) for rho in range(R_rep)]
+        total = _ring_token_sum(per_replica, c, add)
+        want = rb(total / K) if wire else total / K
+        assert (Fraction(float(got[j])) == want) if wire else (got[j] == f32_of_fraction(want)), (j, s, c)
+    if wire:
+        asc = orc.reduce_mean([orc.bf16_bits_to_f64(b) for b in bits], S, R_rep, wire_bf16=True)
+        assert np.allclose(got, asc, rtol=2 ** -6, atol=0.03)           # same sum, other rounding
+
+
+def test_ring_order_changes_bf16_sums_but_not_fp32_sums():
+    rng = np.random.default_rng(78)
+    g = [orc.bf16_bits_to_f64(rng_bf16_bits(rng, 4096, 1e-3)) for _ in range(8)]
+    for S, R_rep in ((8, 1), (4, 2)):
+        ring = orc.ring_positions(orc.plan([4096], S, 8), R_rep)
+        assert np.array_equal(orc.reduce_mean(g, S, R_rep, ring=ring), orc.reduce_mean(g, S, R_rep))
+        a, b = orc.reduce_mean(g, S, R_rep, True, ring), orc.reduce_mean(g, S, R_rep, True)
+        # rank S-1 of the shard level (and sub-chunk R_rep-1) visits the buffers in ascending order anyway
+        last = (ring[0] == S - 1) & (ring[1] == R_rep - 1)
+        assert np.array_equal(a[last], b[last]) and 0.02 < np.mean(a[~last] != b[~last]) < 0.9
+    assert orc.ring_order(2, 4) == [3, 0, 1, 2] and orc.ring_order(0, 1) == [0] and orc.ring_order(3, 4) == [0, 1, 2, 3]
+
+
+def test_ring_positions_on_several_units():
+    L = orc.plan([10, 3, 8], 2, 1)          # shard lengths 5, 2, 4
+    s, c = orc.ring_positions(L, 2)
+    want_s, want_c = [], []
+    for n, M in zip([10, 3, 8], [5, 2, 4]):
+        for i in range(n):
+            want_s.append(i // M)
+            want_c.append((i % M) // (-(-M // 2)))
+    assert s.tolist() == want_s and c.tolist() == want_c
+    assert max(want_c) == 1 and c[:10].tolist() == [0, 0, 0, 1, 1, 0, 0, 0, 1, 1]
+
+
 def test_reduce_special_cases():
     rng = np.random.default_rng(7)
     g = [orc.bf16_bits_to_f64(rng_bf16_bits(rng, 1000)) for _ in range(8)]
@@ -355,6 +424,42 @@ def test_fedavg_identity_cases():
     s2 = [orc.GroupState(y.copy(), None, None, None) for y in ys[::-1]]
     orc.fedavg(s1); orc.fedavg(s2)
     assert np.allclose(s1[0].theta, s2[0].theta, rtol=2e-7, atol=0)
+
+
+def test_replicated_state_copies_stay_identical_and_match_the_single_copy():
+    """FL+HSDP with one state copy per replica: every replica of a group applies the same mean gradient, so the
+    copies stay bit-identical; the aggregation reads one replica per group and its broadcast makes all R_rep
+    copies of every group equal to what plain FedAvg over one copy per group gives."""
+    rng = np.random.default_rng(41)
+    G, S, R_rep, n = 3, 2, 2, 300
+    hp = orc.Hyper(max_grad_norm=0.01)
+    th0 = rng.normal(0, 0.02, n).astype(np.float32)
+    z = np.zeros(n, np.float32)
+    single = [orc.GroupState(th0.copy(), z.copy(), z.copy(), None) for _ in range(G)]
+    repl = [[orc.GroupState(th0.copy(), z.copy(), z.copy(), None) for _ in range(R_rep)] for _ in range(G)]
+    counts = [3, 1, 5]
+    for opt_state in (False, True):
+        for t in (1, 2):
+            for g in range(G):
+                grads = [orc.bf16_bits_to_f64(rng_bf16_bits(rng, n)) for _ in range(S * R_rep)]
+                a = orc.sync_step_group(single[g], grads, S, R_rep, t, hp)
+                b = orc.sync_step_replicated(repl[g], grads, S, R_rep, t, hp)
+                assert a[0] == b[0] and a[1] == b[1]
+                for st in repl[g]:
+                    assert np.array_equal(st.theta, single[g].theta) and np.array_equal(st.v, single[g].v)
+        assert not np.array_equal(repl[0][1].theta, repl[1][1].theta)      # groups have diverged
+        orc.fedavg(single, counts, opt_state)
+        orc.fedavg_replicated(repl, counts, opt_state)
+        for g in range(G):
+            for st in repl[g]:
+                assert np.array_equal(st.theta, single[g].theta) and np.array_equal(st.param_bf16, single[g].param_bf16)
+                assert np.array_equal(st.m, single[g].m) and np.array_equal(st.v, single[g].v)
+        assert np.array_equal(repl[0][1].theta, repl[2][0].theta)
+        assert np.array_equal(repl[0][1].m, repl[2][0].m) == opt_state     # moments are shared only when averaged
+    # a replica that did not take part must still receive the broadcast: corrupt one, aggregate, all equal again
+    repl[1][1].theta = repl[1][1].theta + 1.0
+    orc.fedavg_replicated(repl, counts, False)
+    assert all(np.array_equal(st.theta, repl[0][0].theta) for reps in repl for st in reps)
 
 
 def test_fedavg_outer_special_case_and_torch_sgd():
