@@ -294,6 +294,8 @@ def measure_workload(args, cfg, fls, Session, rank, world, local, with_e2e, samp
         fls.fls_plan_tune(sess.plan, fls.FLS_KERNEL_ADAMW, 0, 0)
     if args.no_overlap:
         fls.fls_plan_set_overlap(sess.plan, False)
+    if args.l2_keep_mb is not None:
+        fls.fls_plan_set_l2_keep(sess.plan, int(args.l2_keep_mb * 2 ** 20))
     fill_session(sess, cfg)
     stream = torch.cuda.current_stream()
 
@@ -632,6 +634,7 @@ def main():
     ap.add_argument("--descending-adamw", action="store_true")
     ap.add_argument("--ascending-adamw", action="store_true")
     ap.add_argument("--no-overlap", action="store_true", help="plain launches instead of programmatic dependent launch")
+    ap.add_argument("--l2-keep-mb", type=float, default=None, help="MiB at the end of the reduced gradient stored with L2 evict-last (library default: 64)")
     # slices of a workload, for profiler captures that must stay small (same kernels, fewer bytes)
     ap.add_argument("--n-params", type=int, default=0, help="override P (single flat unit)")
     ap.add_argument("--groups", type=int, default=0, help="override G")

@@ -43,6 +43,8 @@ typedef struct fls_plan fls_plan; /* opaque, created by fls_plan_create, freed b
 enum { FLS_OK = 0, FLS_EINVAL = 1, FLS_EALIGN = 2, FLS_EPTR = 3, FLS_ESIZE = 4, FLS_ECUDA = 5, FLS_ESTATE = 6 };
 enum { FLS_GRAD_BF16 = 0, FLS_GRAD_F32 = 1 };
 enum { FLS_WIRE_F32 = 0, FLS_WIRE_BF16 = 1 };          /* reduce_wire */
+enum { FLS_ORDER_ASCENDING = 0, FLS_ORDER_RING = 1 };  /* reduce_order */
+enum { FLS_STATE_PER_GROUP = 0, FLS_STATE_PER_REPLICA = 1 }; /* state_copies */
 enum { FLS_AVG_PARAMS = 1, FLS_AVG_OPT_STATE = 2, FLS_AVG_FUSED = 4 }; /* fedavg_what bit mask */
 enum { FLS_KERNEL_REDUCE = 0, FLS_KERNEL_ADAMW = 1, FLS_KERNEL_FEDAVG = 2, FLS_KERNEL_ADAMW_FEDAVG = 3, FLS_KERNEL_COUNT = 4 };
 enum { FLS_STATUS_NONFINITE_NORM = 1 }; /* sticky bits of the device status word */
@@ -50,6 +52,7 @@ enum { FLS_STATUS_NONFINITE_NORM = 1 }; /* sticky bits of the device status word
 #define FLS_MAX_GROUPS 64        /* G <= 64 */
 #define FLS_MAX_GRAD_BUFFERS 64  /* K = shard_dim * replicate_dim <= 64 */
 #define FLS_MAX_FUSED_GROUPS 16  /* fls_sync_step_fedavg fuses the aggregation for G up to this */
+#define FLS_MAX_STATE_COPIES 64  /* G * R_rep <= 64 with FLS_STATE_PER_REPLICA */
 #define FLS_BUFFER_ALIGN 32      /* every device buffer must start on a 32-byte boundary */
 #define FLS_NOALLOC_MAX_ELEMS 536870912ull /* 2^29: largest n_elems fls_reduce_norm_noalloc accepts */
 
@@ -75,6 +78,19 @@ typedef struct {
                                  to bf16, emulating collectives that run in bf16 -- the setting in which the
                                  paper observes that the FSDP and HSDP orders give different numbers.  Slower
                                  (generic kernel); meant for numerical experiments                         */
+  uint32_t reduce_order;      /* FLS_ORDER_ASCENDING (default): buffers are added in ascending index at both levels.
+                                 FLS_ORDER_RING: in the order ring collectives produce.  The elements rank s owns
+                                 after the reduce-scatter are summed sigma = s+1, s+2, ..., s (mod S): the chunk
+                                 starts on the next rank and its owner adds last.  The all-reduce across replicas
+                                 is a ring reduce-scatter + all-gather over R_rep equal sub-chunks of every
+                                 rank's slice of a unit (ceil(M_u/R_rep) elements each): sub-chunk c is summed
+                                 rho = c+1, ..., c (mod R_rep).  Same sums, other rounding order: visible with
+                                 FLS_WIRE_BF16, within rounding with fp32 partial sums.  Generic kernel (slower) */
+  uint32_t state_copies;      /* FLS_STATE_PER_GROUP (default): one master/m/v/bf16 copy per group.
+                                 FLS_STATE_PER_REPLICA: one per replica, G*R_rep in all (FL+HSDP as it runs: every
+                                 replica of a group applies the same mean gradient to its own copy; only one replica
+                                 per group takes part in FedAvg and then broadcasts the result inside its group, the
+                                 C_BC term of Eq. 5).  Needs G*R_rep <= FLS_MAX_STATE_COPIES                       */
   double lr, beta1, beta2, eps, weight_decay;
   double max_grad_norm;       /* <= 0 disables clipping (the norm is still computed)                    */
 } fls_plan_desc;
@@ -95,6 +111,9 @@ typedef struct {
   uint64_t workspace_bytes;          /* size the caller must provide in fls_buffers.workspace           */
   uint32_t n_segments;               /* contiguous (unit, shard) runs the kernels walk                  */
   uint32_t vector_path;              /* 1 if every segment is 8-element aligned in both orders          */
+  uint32_t n_state_copies;           /* entries of fls_buffers.master / m / v / param_bf16: G, or G*R_rep with
+                                        FLS_STATE_PER_REPLICA                                            */
+  uint32_t reserved;
 } fls_layout;
 
 /* Device buffers, all caller-owned, each N_pad elements, FLS_BUFFER_ALIGN-aligned, non-overlapping.
@@ -102,7 +121,8 @@ typedef struct {
 typedef struct {
   const void* const* grads; /* host array of G*K device pointers, index g*K + rho*S + sigma; bf16 or fp32;
                                unsharded order; read-only to the library, never cleared by it            */
-  float* const* master;     /* host array of G device pointers: fp32 parameters, shard order, in/out     */
+  float* const* master;     /* host array of n_state_copies device pointers (G; with FLS_STATE_PER_REPLICA G*R_rep,
+                               index g*R_rep + rho): fp32 parameters, shard order, in/out                   */
   float* const* m;          /* same: first moment                                                        */
   float* const* v;          /* same: second moment                                                       */
   void* const* param_bf16;  /* host array of G device pointers: bf16 copy, unsharded order, output       */
@@ -119,16 +139,21 @@ typedef struct {
   fls_cost5 wire_bytes;  /* bytes one rank sends per step when D of all-gather / reduce-scatter is the whole
                             unit (S*M_u), the convention of the NCCL performance notes the paper cites        */
   fls_cost5 seconds;     /* Eq. 1-5 with B_S, B_R, B_F; NaN when no bandwidths were given                     */
-  double hbm_bytes_sync_step; /* bytes one fls_sync_step must move in this library: G*N_pad*(K*e_g + 34), or
-                                 G*N_pad*(2*K*e_g + 26) when K*e_g < 8 (gradients read twice, nothing stored),
-                                 or G*N_pad*(K*e_g + 26) without clipping (single pass)                        */
-  double hbm_bytes_fedavg;    /* bytes one fls_fedavg must move: G*N_pad*10, or *26 with optimizer state      */
+  double hbm_bytes_sync_step; /* bytes one fls_sync_step must move on the route the plan is set to at the time of the
+                                 call: G*N_pad*(K*e_g + 34) (store and reread), G*N_pad*(2*K*e_g + 26) (recompute,
+                                 the default when K*e_g < 8), G*N_pad*(K*e_g + 26) (single pass: no clipping, or a
+                                 speculative step that is kept).  With FLS_STATE_PER_REPLICA: G*N_pad*(K*e_g + 4 +
+                                 30*R_rep)                                                                     */
+  double hbm_bytes_fedavg;    /* bytes one fls_fedavg must move: G*N_pad*10, or *26 with optimizer state; with
+                                 FLS_STATE_PER_REPLICA the broadcast adds 6 (14) per extra copy: G*N_pad*(4 + 6*R_rep),
+                                 or G*N_pad*(12 + 14*R_rep)                                                    */
 } fls_comm_costs;
 
 /* Layout planner + validation (flat-buffer layout: padding to the shard multiple, per-unit offsets).
  * Host only: touches no GPU.  Errors: FLS_EINVAL for a null argument, G, S, R_rep, H or Q = 0, G or K
  * above the maxima, sum(unit_numel) != n_params, a zero-length unit, beta outside [0,1), eps <= 0, lr < 0,
- * an unknown dtype, FLS_WIRE_BF16 with fp32 gradients, or fedavg_what without FLS_AVG_PARAMS.  On error *out is NULL. */
+ * an unknown dtype, order or state_copies value, FLS_WIRE_BF16 with fp32 gradients, G*R_rep above
+ * FLS_MAX_STATE_COPIES with FLS_STATE_PER_REPLICA, or fedavg_what without FLS_AVG_PARAMS.  On error *out is NULL. */
 int fls_plan_create(const fls_plan_desc* desc, fls_plan** out);
 
 /* Copies the layout summary into *out (host). */
@@ -232,6 +257,34 @@ int fls_plan_set_recompute(fls_plan* plan, int mode);
  * (FLS_ESTATE if the plan clips or uses FLS_WIRE_BF16), -1 restores the default.  master, m, v and the bf16 copy
  * are identical either way; after a single-pass step fls_get_reduced_grad has nothing to offer (FLS_ESTATE). */
 int fls_plan_set_single_pass(fls_plan* plan, int mode);
+
+/* Speculative single pass for plans that clip.  When the norm usually stays below max_grad_norm, the two passes
+ * of a step (norm first, then AdamW) can be replaced by one that guesses "clip coefficient = 1": one kernel per
+ * group forms the mean gradient, applies AdamW with coefficient 1 and computes the norm; a second, normally empty
+ * kernel looks at the coefficient and, only if it is not 1, redoes the step with it.  K*e_g + 26 bytes per element
+ * when the guess holds, twice that when it does not (the default route costs K*e_g + 34 either way), so it pays
+ * only on workloads that rarely clip; it is never on by default.  Results are bit-identical to the default route.
+ * The first kernel must not overwrite its own input, so the plan needs a second set of state buffers:
+ * fls_plan_bind_shadow gives it G device pointers each for master, m and v (host arrays; N_pad floats each,
+ * FLS_BUFFER_ALIGN-aligned, caller-owned, overlapping nothing bound).  Every speculative step reads the current set
+ * and writes the other one, which then becomes current: after each fls_sync_step ask fls_get_state where group g's
+ * state is now.  fls_plan_set_speculative(plan, 1) turns it on: FLS_ESTATE without shadow buffers, for plans that do
+ * not clip, for FLS_WIRE_BF16, FLS_ORDER_RING or FLS_STATE_PER_REPLICA plans; 0 turns it off (the state stays where
+ * it is).  The fused aggregation of fls_sync_step_fedavg steps in place and does not speculate.
+ * fls_get_spec_stats: device pointer to two uint32 counters, [0] group-steps whose guess held, [1] group-steps that
+ * were redone; valid once the steps have completed on their stream. */
+int fls_plan_bind_shadow(fls_plan* plan, float* const* master, float* const* m, float* const* v);
+int fls_plan_set_speculative(fls_plan* plan, int enabled);
+int fls_get_spec_stats(const fls_plan* plan, const uint32_t** dev_counts);
+
+/* Current device pointers of state copy `copy` (0 .. n_state_copies-1): what was bound, except on speculative
+ * plans, where every step moves the state to the other buffer set.  Any output may be NULL. */
+int fls_get_state(const fls_plan* plan, uint32_t copy, float** master, float** m, float** v);
+
+/* How many bytes at the end of the reduced gradient the reduce kernel stores with the "evict last" L2 policy (the
+ * AdamW kernel walks the reduced gradient backwards, so it reads that part first and finds it in L2); the rest is
+ * stored "evict first" like every other stream.  Default 64 MiB.  Scheduling only: results do not change. */
+int fls_plan_set_l2_keep(fls_plan* plan, uint64_t bytes);
 
 /* enabled != 0 (the default): inside one call every kernel but the first is launched so that its first CTAs may
  * start during the tail of the kernel before it (programmatic dependent launch); they fetch what that kernel does

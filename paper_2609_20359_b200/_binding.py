@@ -13,12 +13,15 @@ LIB_PATH = os.environ.get("FLS_LIBRARY") or os.path.join(_PKG, "libfls.so")
 FLS_OK, FLS_EINVAL, FLS_EALIGN, FLS_EPTR, FLS_ESIZE, FLS_ECUDA, FLS_ESTATE = range(7)
 FLS_GRAD_BF16, FLS_GRAD_F32 = 0, 1
 FLS_WIRE_F32, FLS_WIRE_BF16 = 0, 1
+FLS_ORDER_ASCENDING, FLS_ORDER_RING = 0, 1
+FLS_STATE_PER_GROUP, FLS_STATE_PER_REPLICA = 0, 1
 FLS_AVG_PARAMS, FLS_AVG_OPT_STATE, FLS_AVG_FUSED = 1, 2, 4
 FLS_KERNEL_REDUCE, FLS_KERNEL_ADAMW, FLS_KERNEL_FEDAVG, FLS_KERNEL_ADAMW_FEDAVG, FLS_KERNEL_COUNT = 0, 1, 2, 3, 4
 FLS_STATUS_NONFINITE_NORM = 1
 FLS_MAX_GROUPS = 64
 FLS_MAX_GRAD_BUFFERS = 64
 FLS_MAX_FUSED_GROUPS = 16
+FLS_MAX_STATE_COPIES = 64
 FLS_BUFFER_ALIGN = 32
 FLS_NOALLOC_MAX_ELEMS = 1 << 29
 
@@ -26,6 +29,7 @@ EXPORTS = [
     "fls_plan_create", "fls_plan_query", "fls_plan_bind", "fls_sync_step", "fls_sync_step_host", "fls_fedavg",
     "fls_sync_step_fedavg", "fls_fedavg_outer",
     "fls_get_norms", "fls_get_reduced_grad", "fls_get_status", "fls_get_step", "fls_set_step", "fls_comm_report",
+    "fls_plan_bind_shadow", "fls_plan_set_speculative", "fls_get_spec_stats", "fls_get_state", "fls_plan_set_l2_keep",
     "fls_plan_tune", "fls_plan_set_recompute", "fls_plan_set_single_pass", "fls_plan_set_overlap", "fls_set_profiling", "fls_get_kernel_ms", "fls_get_launch_count", "fls_plan_destroy",
     "fls_last_error", "fls_reduce_norm_noalloc",
 ]
@@ -42,6 +46,7 @@ class fls_plan_desc(C.Structure):
                 ("groups", C.c_uint32), ("shard_dim", C.c_uint32), ("replicate_dim", C.c_uint32),
                 ("sync_period", C.c_uint32), ("grad_dtype", C.c_uint32), ("align_elems", C.c_uint32),
                 ("fedavg_what", C.c_uint32), ("reduce_wire", C.c_uint32),
+                ("reduce_order", C.c_uint32), ("state_copies", C.c_uint32),
                 ("lr", C.c_double), ("beta1", C.c_double), ("beta2", C.c_double), ("eps", C.c_double),
                 ("weight_decay", C.c_double), ("max_grad_norm", C.c_double)]
 
@@ -50,7 +55,8 @@ class fls_layout(C.Structure):
     _fields_ = [("n_padded", C.c_uint64), ("shard_numel", C.c_uint64), ("n_units", C.c_uint32),
                 ("grad_buffers", C.c_uint32), ("unit_offset", C.POINTER(C.c_uint64)),
                 ("unit_shard_numel", C.POINTER(C.c_uint64)), ("unit_shard_offset", C.POINTER(C.c_uint64)),
-                ("workspace_bytes", C.c_uint64), ("n_segments", C.c_uint32), ("vector_path", C.c_uint32)]
+                ("workspace_bytes", C.c_uint64), ("n_segments", C.c_uint32), ("vector_path", C.c_uint32),
+                ("n_state_copies", C.c_uint32), ("reserved", C.c_uint32)]
 
 
 class fls_buffers(C.Structure):
@@ -92,6 +98,11 @@ def _load() -> C.CDLL:
     lib.fls_set_step.argtypes = [P, C.c_uint64]
     lib.fls_comm_report.argtypes = [P, C.POINTER(C.c_double), C.POINTER(fls_comm_costs)]
     lib.fls_plan_tune.argtypes = [P, C.c_uint32, C.c_int, C.c_int]
+    lib.fls_plan_bind_shadow.argtypes = [P, C.POINTER(C.c_void_p), C.POINTER(C.c_void_p), C.POINTER(C.c_void_p)]
+    lib.fls_plan_set_speculative.argtypes = [P, C.c_int]
+    lib.fls_get_spec_stats.argtypes = [P, C.POINTER(P)]
+    lib.fls_get_state.argtypes = [P, C.c_uint32, C.POINTER(P), C.POINTER(P), C.POINTER(P)]
+    lib.fls_plan_set_l2_keep.argtypes = [P, C.c_uint64]
     lib.fls_plan_set_recompute.argtypes = [P, C.c_int]
     lib.fls_plan_set_single_pass.argtypes = [P, C.c_int]
     lib.fls_plan_set_overlap.argtypes = [P, C.c_int]
@@ -136,7 +147,8 @@ def fls_plan_create(n_params: int, unit_numel: Optional[Sequence[int]] = None, g
                     replicate_dim: int = 1, sync_period: int = 1, grad_dtype: int = FLS_GRAD_BF16, align_elems: int = 8,
                     fedavg_what: int = FLS_AVG_PARAMS, lr: float = 3e-4, beta1: float = 0.9, beta2: float = 0.95,
                     eps: float = 1e-8, weight_decay: float = 0.1, max_grad_norm: float = 1.0,
-                    reduce_wire: int = FLS_WIRE_F32) -> int:
+                    reduce_wire: int = FLS_WIRE_F32, reduce_order: int = FLS_ORDER_ASCENDING,
+                    state_copies: int = FLS_STATE_PER_GROUP) -> int:
     """Returns the opaque plan handle."""
     d = fls_plan_desc()
     d.n_params = n_params
@@ -145,6 +157,7 @@ def fls_plan_create(n_params: int, unit_numel: Optional[Sequence[int]] = None, g
         d.n_units, d.unit_numel = len(unit_numel), arr
     d.groups, d.shard_dim, d.replicate_dim, d.sync_period = groups, shard_dim, replicate_dim, sync_period
     d.grad_dtype, d.align_elems, d.fedavg_what, d.reduce_wire = grad_dtype, align_elems, fedavg_what, reduce_wire
+    d.reduce_order, d.state_copies = reduce_order, state_copies
     d.lr, d.beta1, d.beta2, d.eps, d.weight_decay, d.max_grad_norm = lr, beta1, beta2, eps, weight_decay, max_grad_norm
     out = C.c_void_p()
     _check(lib.fls_plan_create(C.byref(d), C.byref(out)))
@@ -159,12 +172,14 @@ def fls_plan_query(plan: int) -> dict:
                 unit_offset=[lay.unit_offset[i] for i in range(n)],
                 unit_shard_numel=[lay.unit_shard_numel[i] for i in range(n)],
                 unit_shard_offset=[lay.unit_shard_offset[i] for i in range(n)],
-                workspace_bytes=lay.workspace_bytes, n_segments=lay.n_segments, vector_path=bool(lay.vector_path))
+                workspace_bytes=lay.workspace_bytes, n_segments=lay.n_segments, vector_path=bool(lay.vector_path),
+                n_state_copies=lay.n_state_copies)
 
 
 def fls_plan_bind(plan: int, grads: Sequence, master: Sequence, m: Sequence, v: Sequence, param_bf16: Sequence,
                   workspace, workspace_bytes: Optional[int] = None) -> None:
-    """grads: G*K tensors (index g*K + rho*S + sigma); master/m/v/param_bf16: G tensors; workspace: a byte tensor."""
+    """grads: G*K tensors (index g*K + rho*S + sigma); master/m/v/param_bf16: n_state_copies tensors (G, or G*R_rep
+    with one state copy per replica, index g*R_rep + rho); workspace: a byte tensor."""
     b = fls_buffers()
     keep = [_ptr_array(grads), _ptr_array(master), _ptr_array(m), _ptr_array(v), _ptr_array(param_bf16)]
     b.grads, b.master, b.m, b.v, b.param_bf16 = keep
@@ -248,6 +263,33 @@ def fls_comm_report(plan: int, bw_bytes_per_s: Optional[Sequence[float]] = None)
 
 def fls_plan_tune(plan: int, kernel: int, ctas_per_sm: int = 0, descending: int = -1) -> None:
     _check(lib.fls_plan_tune(plan, kernel, ctas_per_sm, descending))
+
+
+def fls_plan_bind_shadow(plan: int, master: Sequence, m: Sequence, v: Sequence) -> None:
+    """Second set of state buffers (G tensors each) that speculative steps write to."""
+    _check(lib.fls_plan_bind_shadow(plan, _ptr_array(master), _ptr_array(m), _ptr_array(v)))
+
+
+def fls_plan_set_speculative(plan: int, enabled: bool) -> None:
+    _check(lib.fls_plan_set_speculative(plan, int(enabled)))
+
+
+def fls_get_spec_stats(plan: int) -> int:
+    """Device address of two uint32 counters: group-steps kept, group-steps redone."""
+    a = C.c_void_p()
+    _check(lib.fls_get_spec_stats(plan, C.byref(a)))
+    return a.value
+
+
+def fls_get_state(plan: int, copy: int):
+    """(master, m, v) device addresses of state copy `copy` as they are now."""
+    a, b, c = C.c_void_p(), C.c_void_p(), C.c_void_p()
+    _check(lib.fls_get_state(plan, copy, C.byref(a), C.byref(b), C.byref(c)))
+    return a.value, b.value, c.value
+
+
+def fls_plan_set_l2_keep(plan: int, nbytes: int) -> None:
+    _check(lib.fls_plan_set_l2_keep(plan, nbytes))
 
 
 def fls_plan_set_recompute(plan: int, mode: int) -> None:

@@ -38,6 +38,13 @@ struct TimedLaunch {
   int kernel;
 };
 
+struct Range {
+  uintptr_t lo, hi;
+  const char* what;
+  int index;
+  bool output;
+};
+
 }  // namespace
 
 struct fls_plan {
@@ -45,6 +52,9 @@ struct fls_plan {
   std::vector<uint64_t> units;
   Layout lay;
   uint32_t K = 0;
+  uint32_t R_state = 1;     // state copies per group: R_rep with FLS_STATE_PER_REPLICA, else 1
+  uint32_t n_copies = 0;    // G * R_state: entries of master / m / v / pbf16
+  bool ring = false;
   uint64_t end_mask = 0;
   uint32_t fold_mask = 0;
   int reduce_sg = -1;
@@ -53,8 +63,12 @@ struct fls_plan {
   int device = -1;
   int sm_count = 0;
   std::vector<const void*> grads;
-  std::vector<float*> master, m, v;
+  std::vector<float*> master, m, v;      // current state of every copy (index g*R_state + rho)
   std::vector<uint16_t*> pbf16;
+  std::vector<float*> master2, m2, v2;   // second buffer set of a speculative plan (the one not current)
+  std::vector<Range> ranges;             // everything bound, for overlap checks of later additions
+  bool speculative = false;
+  uint64_t l2_keep_bytes = 64ull << 20;  // tail of the reduced gradient stored with L2 evict-last
   char* ws = nullptr;
 
   uint64_t step = 0;
@@ -81,8 +95,16 @@ struct fls_plan {
   float* d_coefs() const { return reinterpret_cast<float*>(ws + kWsCoefs); }
   double* d_normsq() const { return reinterpret_cast<double*>(ws + kWsNormSq); }
   double* d_partials() const { return reinterpret_cast<double*>(ws + lay.ws_partials_offset); }
+  double* d_chunk_partials() const { return reinterpret_cast<double*>(ws + lay.ws_chunk_partials_offset); }
+  uint32_t* d_chunk_count() const { return reinterpret_cast<uint32_t*>(ws + lay.ws_chunk_count_offset); }
   uint32_t* d_status() const { return reinterpret_cast<uint32_t*>(ws + kWsStatus); }
   uint32_t* d_ticket() const { return reinterpret_cast<uint32_t*>(ws + kWsStatus) + 1; }
+  uint32_t* d_spec_counts() const { return reinterpret_cast<uint32_t*>(ws + kWsStatus) + 2; }
+  // how fls_sync_step currently gets from the gradients to the new state (for the HBM byte count)
+  // the routes that form the mean gradient inside the AdamW kernel exist for fp32 partial sums in ascending order
+  // and one state copy per group
+  bool plain_reduce() const { return desc.reduce_wire == FLS_WIRE_F32 && !ring && R_state == 1; }
+  int route() const { return speculative || single_pass ? 2 : (recompute ? 1 : 0); }
 
   SegIndex seg_index() const {
     SegIndex ix{};
@@ -115,13 +137,6 @@ struct fls_plan {
 };
 
 namespace {
-
-struct Range {
-  uintptr_t lo, hi;
-  const char* what;
-  int index;
-  bool output;
-};
 
 // Brackets one kernel launch with events when profiling is on.
 template <typename F>
@@ -160,6 +175,11 @@ AdamScalars adam_scalars(const fls_plan_desc& d, double lr, uint64_t t_new) {
   return s;
 }
 
+void set_adam_scalars(AdamArgs* aa, const AdamScalars& sc) {
+  aa->decay = sc.decay; aa->beta1 = sc.beta1; aa->omb1 = sc.omb1; aa->beta2 = sc.beta2; aa->omb2 = sc.omb2;
+  aa->step_size = sc.step_size; aa->inv_sqrt_bc2 = sc.inv_sqrt_bc2; aa->eps = sc.eps;
+}
+
 // One group's reduce (+ AdamW) launches.  chain: the previous operation on `st` is a kernel of this same call,
 // so this group's first kernel may overlap its tail.  slot: which reduced-gradient buffer of the workspace
 // receives the mean gradient; with_adamw = false stops after the reduction (the fused aggregation applies AdamW
@@ -167,6 +187,7 @@ AdamScalars adam_scalars(const fls_plan_desc& d, double lr, uint64_t t_new) {
 int run_group(fls_plan* p, uint32_t g, double lr, uint64_t t_new, cudaStream_t st, bool chain, uint32_t slot = 0,
               bool with_adamw = true) {
   const fls_plan_desc& d = p->desc;
+  const uint32_t c0 = g * p->R_state;      // the group's first state copy
   ReduceArgs ra{};
   for (uint32_t k = 0; k < p->K; ++k) ra.grad[k] = p->grads[size_t(g) * p->K + k];
   ra.gbar = p->d_gbar(slot);
@@ -179,60 +200,121 @@ int run_group(fls_plan* p, uint32_t g, double lr, uint64_t t_new, cudaStream_t s
   ra.fold_mask = p->fold_mask;
   ra.end_mask = p->end_mask;
   ra.partials = p->d_partials();
+  ra.chunk_partials = p->d_chunk_partials();
+  ra.chunk_count = p->d_chunk_count();
   ra.ticket = p->d_ticket();
   ra.norm_out = p->d_norms() + g;
   ra.coef_out = p->d_coefs() + g;
   ra.normsq_out = p->d_normsq() + g;
   ra.status = p->d_status();
   ra.max_grad_norm = d.max_grad_norm;
-  const bool single = p->single_pass && with_adamw;
+  ra.ring = p->ring ? 1u : 0u;
+  ra.S = d.shard_dim;
+  ra.R = d.replicate_dim;
+  ra.spec_counts = nullptr;
+  // the AdamW kernel walks the reduced gradient from its end: keep that end in L2, stream the rest
+  const uint64_t keep_tiles = std::min<uint64_t>(p->lay.n_tiles, p->l2_keep_bytes / (uint64_t(kTile) * 4));
+  ra.keep_from_tile = with_adamw && p->descending[FLS_KERNEL_ADAMW] ? uint32_t(p->lay.n_tiles - keep_tiles) : uint32_t(p->lay.n_tiles);
+  const bool speculate = p->speculative && with_adamw;
+  const bool single = (p->single_pass || speculate) && with_adamw;
   const bool recompute = p->recompute && with_adamw && !single;   // the fused aggregation needs the stored gradients
   ra.store_gbar = (recompute || single) ? 0 : 1;
   p->gbar_valid = ra.store_gbar != 0;
   const bool f32 = d.grad_dtype == FLS_GRAD_F32;
   const bool overlap = p->overlap && !p->profiling;   // event records between kernels would serialise anyway
+  const AdamScalars sc = adam_scalars(d, lr, t_new);
+  AdamArgs aa{};
+  aa.gbar = p->d_gbar(slot);
+  aa.theta = aa.theta_out = p->master[c0];
+  aa.m = aa.m_out = p->m[c0];
+  aa.v = aa.v_out = p->v[c0];
+  aa.pbf16 = p->pbf16[c0];
+  aa.idx = ra.idx;
+  aa.descending = p->descending[FLS_KERNEL_ADAMW];
+  aa.coef = p->d_coefs() + g;
+  set_adam_scalars(&aa, sc);
   if (single) {
-    // no clipping: the coefficient is 1 before the norm is known, so one kernel does the whole step of the group
-    const AdamScalars sc1 = adam_scalars(d, lr, t_new);
+    // The coefficient is 1 (no clipping) or guessed to be 1 (speculative): one kernel does the whole step of the
+    // group.  A speculative step writes the other buffer set and is followed by a kernel that redoes the step with
+    // the real coefficient if the guess was wrong; either way the other set holds the new state afterwards.
     ReduceAdamArgs rp{};
     rp.r = ra;
-    rp.a.theta = p->master[g];
-    rp.a.m = p->m[g];
-    rp.a.v = p->v[g];
-    rp.a.pbf16 = p->pbf16[g];
-    rp.a.idx = ra.idx;
-    rp.a.decay = sc1.decay; rp.a.beta1 = sc1.beta1; rp.a.omb1 = sc1.omb1; rp.a.beta2 = sc1.beta2; rp.a.omb2 = sc1.omb2;
-    rp.a.step_size = sc1.step_size; rp.a.inv_sqrt_bc2 = sc1.inv_sqrt_bc2; rp.a.eps = sc1.eps;
+    rp.a = aa;
+    if (speculate) {
+      rp.r.spec_counts = p->d_spec_counts();
+      rp.a.theta_out = p->master2[g];
+      rp.a.m_out = p->m2[g];
+      rp.a.v_out = p->v2[g];
+    }
     cudaError_t e1 = timed_launch(p, FLS_KERNEL_ADAMW, st, [&] { return launch_step_noclip(rp, f32, p->reduce_sg, st, overlap && chain); });
     if (e1 != cudaSuccess) return cuda_fail(e1, "single-pass step kernel launch");
+    if (speculate) {
+      rp.r.spec_counts = nullptr;
+      rp.skip_if_unclipped = 1;
+      const unsigned grid = unsigned(std::min<uint64_t>(p->lay.n_tiles, uint64_t(std::max(p->sm_count, 1)) * 8));
+      e1 = timed_launch(p, FLS_KERNEL_ADAMW, st, [&] { return launch_reduce_adamw(rp, f32, p->reduce_sg, grid, st, overlap); });
+      if (e1 != cudaSuccess) return cuda_fail(e1, "speculative redo kernel launch");
+      std::swap(p->master[g], p->master2[g]);
+      std::swap(p->m[g], p->m2[g]);
+      std::swap(p->v[g], p->v2[g]);
+    }
     return FLS_OK;
   }
   cudaError_t e = timed_launch(p, FLS_KERNEL_REDUCE, st, [&] { return launch_reduce(ra, f32, p->reduce_sg, st, overlap && chain); });
   if (e != cudaSuccess) return cuda_fail(e, "reduce kernel launch");
   if (!with_adamw) return FLS_OK;
 
-  const AdamScalars sc = adam_scalars(d, lr, t_new);
-  AdamArgs aa{};
-  aa.gbar = p->d_gbar(slot);
-  aa.theta = p->master[g];
-  aa.m = p->m[g];
-  aa.v = p->v[g];
-  aa.pbf16 = p->pbf16[g];
-  aa.idx = ra.idx;
-  aa.descending = p->descending[FLS_KERNEL_ADAMW];
-  aa.coef = p->d_coefs() + g;
-  aa.decay = sc.decay; aa.beta1 = sc.beta1; aa.omb1 = sc.omb1; aa.beta2 = sc.beta2; aa.omb2 = sc.omb2;
-  aa.step_size = sc.step_size; aa.inv_sqrt_bc2 = sc.inv_sqrt_bc2; aa.eps = sc.eps;
   if (recompute) {
     ReduceAdamArgs rp{};
     rp.r = ra;
     rp.a = aa;
     e = timed_launch(p, FLS_KERNEL_ADAMW, st,
                      [&] { return launch_reduce_adamw(rp, f32, p->reduce_sg, p->grid_for(FLS_KERNEL_ADAMW), st, overlap); });
-  } else {
-    e = timed_launch(p, FLS_KERNEL_ADAMW, st, [&] { return launch_adamw(aa, p->grid_for(FLS_KERNEL_ADAMW), st, overlap); });
+    if (e != cudaSuccess) return cuda_fail(e, "adamw kernel launch");
+    return FLS_OK;
   }
-  if (e != cudaSuccess) return cuda_fail(e, "adamw kernel launch");
+  // every state copy of the group (one, or one per replica) takes the same update; consecutive passes over the
+  // reduced gradient alternate direction so that each starts where the one before stopped
+  for (uint32_t r = 0; r < p->R_state; ++r) {
+    aa.theta = aa.theta_out = p->master[c0 + r];
+    aa.m = aa.m_out = p->m[c0 + r];
+    aa.v = aa.v_out = p->v[c0 + r];
+    aa.pbf16 = p->pbf16[c0 + r];
+    aa.descending = p->descending[FLS_KERNEL_ADAMW] ^ int(r & 1u);
+    e = timed_launch(p, FLS_KERNEL_ADAMW, st, [&] { return launch_adamw(aa, p->grid_for(FLS_KERNEL_ADAMW), st, overlap); });
+    if (e != cudaSuccess) return cuda_fail(e, "adamw kernel launch");
+  }
+  return FLS_OK;
+}
+
+// Every range must be non-null, aligned device memory of the current device.  Outputs may overlap nothing;
+// gradient buffers may only overlap each other (a caller may feed one buffer to several replicas).
+int check_ranges(const std::vector<Range>& ranges, int dev) {
+  for (const Range& r : ranges) {
+    if (r.lo == 0) return fail(FLS_EPTR, "%s[%d] is null", r.what, r.index);
+    if (r.lo % FLS_BUFFER_ALIGN != 0) return fail(FLS_EALIGN, "%s[%d] is not %d-byte aligned", r.what, r.index, FLS_BUFFER_ALIGN);
+    cudaPointerAttributes attr{};
+    cudaError_t e = cudaPointerGetAttributes(&attr, reinterpret_cast<const void*>(r.lo));
+    if (e != cudaSuccess) {
+      cudaGetLastError();
+      return fail(FLS_EPTR, "%s[%d]: %s", r.what, r.index, cudaGetErrorString(e));
+    }
+    if (attr.type != cudaMemoryTypeDevice && attr.type != cudaMemoryTypeManaged)
+      return fail(FLS_EPTR, "%s[%d] is not device memory", r.what, r.index);
+    if (attr.type == cudaMemoryTypeDevice && attr.device != dev)
+      return fail(FLS_EPTR, "%s[%d] lives on device %d, current device is %d", r.what, r.index, attr.device, dev);
+  }
+  std::vector<size_t> order(ranges.size());
+  for (size_t i = 0; i < order.size(); ++i) order[i] = i;
+  std::sort(order.begin(), order.end(), [&](size_t x, size_t y) { return ranges[x].lo < ranges[y].lo; });
+  for (size_t q = 0; q < order.size(); ++q) {
+    const Range& r0 = ranges[order[q]];
+    for (size_t w = q + 1; w < order.size() && ranges[order[w]].lo < r0.hi; ++w) {
+      const Range& r1 = ranges[order[w]];
+      if (r0.output || r1.output)
+        return fail(FLS_EPTR, "%s[%d] overlaps %s[%d]", r0.what, r0.index, r1.what, r1.index);
+    }
+  }
   return FLS_OK;
 }
 
@@ -267,6 +349,12 @@ int fls_plan_create(const fls_plan_desc* desc, fls_plan** out) {
   if (d.reduce_wire != FLS_WIRE_F32 && d.reduce_wire != FLS_WIRE_BF16) return fail(FLS_EINVAL, "unknown reduce_wire %u", d.reduce_wire);
   if (d.reduce_wire == FLS_WIRE_BF16 && d.grad_dtype != FLS_GRAD_BF16)
     return fail(FLS_EINVAL, "FLS_WIRE_BF16 needs bf16 gradients");
+  if (d.reduce_order != FLS_ORDER_ASCENDING && d.reduce_order != FLS_ORDER_RING) return fail(FLS_EINVAL, "unknown reduce_order %u", d.reduce_order);
+  if (d.state_copies != FLS_STATE_PER_GROUP && d.state_copies != FLS_STATE_PER_REPLICA)
+    return fail(FLS_EINVAL, "unknown state_copies %u", d.state_copies);
+  if (d.state_copies == FLS_STATE_PER_REPLICA && uint64_t(d.groups) * d.replicate_dim > FLS_MAX_STATE_COPIES)
+    return fail(FLS_EINVAL, "groups*replicate_dim = %llu exceeds %d state copies", (unsigned long long)(uint64_t(d.groups) * d.replicate_dim),
+                FLS_MAX_STATE_COPIES);
   if (!(d.beta1 >= 0.0 && d.beta1 < 1.0) || !(d.beta2 >= 0.0 && d.beta2 < 1.0)) return fail(FLS_EINVAL, "betas must lie in [0, 1)");
   if (!(d.eps > 0.0) || !std::isfinite(d.eps)) return fail(FLS_EINVAL, "eps must be positive");
   if (!(d.lr >= 0.0) || !std::isfinite(d.lr)) return fail(FLS_EINVAL, "lr must be finite and >= 0");
@@ -291,8 +379,12 @@ int fls_plan_create(const fls_plan_desc* desc, fls_plan** out) {
   p->units = units;
   p->desc.unit_numel = nullptr;   // the caller's table is not kept; p->units is the copy
   p->desc.n_units = uint32_t(units.size());
-  const bool fused = (d.fedavg_what & FLS_AVG_FUSED) && d.groups <= FLS_MAX_FUSED_GROUPS;
-  const std::string msg = build_layout(units, d.shard_dim, d.align_elems, fused ? d.groups : 1, &p->lay);
+  p->ring = d.reduce_order == FLS_ORDER_RING;
+  p->R_state = d.state_copies == FLS_STATE_PER_REPLICA ? d.replicate_dim : 1;
+  p->n_copies = d.groups * p->R_state;
+  const bool fused = (d.fedavg_what & FLS_AVG_FUSED) && d.groups <= FLS_MAX_FUSED_GROUPS &&
+                     uint64_t(d.groups) * (p->R_state - 1) <= uint64_t(FLS_MAX_FUSED_EXTRA);
+  const std::string msg = build_layout(units, d.shard_dim, d.align_elems, fused ? d.groups : 1, p->ring ? d.replicate_dim : 0, &p->lay);
   if (!msg.empty()) {
     delete p;
     return fail(FLS_EINVAL, "layout: %s", msg.c_str());
@@ -311,11 +403,12 @@ int fls_plan_create(const fls_plan_desc* desc, fls_plan** out) {
   } else {
     p->reduce_sg = -1;
   }
+  if (p->ring) p->reduce_sg = -1;                          // generic kernel: the visiting order depends on the element
   if (d.reduce_wire == FLS_WIRE_BF16) p->reduce_sg = -2;   // generic kernel, bf16 rounding after every sum
   // fewer than 8 gradient bytes per element: a second read of the gradients costs less than the fp32 round trip
-  p->recompute = d.reduce_wire == FLS_WIRE_F32 && K * (d.grad_dtype == FLS_GRAD_F32 ? 4 : 2) < 8;
+  p->recompute = p->plain_reduce() && K * (d.grad_dtype == FLS_GRAD_F32 ? 4 : 2) < 8;
   // without clipping the coefficient is 1 whatever the norm: the step needs no second pass at all
-  p->single_pass = d.reduce_wire == FLS_WIRE_F32 && !(d.max_grad_norm > 0.0);
+  p->single_pass = p->plain_reduce() && !(d.max_grad_norm > 0.0);
   *out = p;
   return FLS_OK;
 }
@@ -332,6 +425,8 @@ int fls_plan_query(const fls_plan* plan, fls_layout* out) {
   out->workspace_bytes = plan->lay.workspace_bytes;
   out->n_segments = uint32_t(plan->lay.segments.size());
   out->vector_path = plan->lay.vector_path ? 1u : 0u;
+  out->n_state_copies = plan->n_copies;
+  out->reserved = 0;
   return FLS_OK;
 }
 
@@ -342,7 +437,7 @@ int fls_plan_bind(fls_plan* p, const fls_buffers* b) {
   if (b->workspace_bytes < p->lay.workspace_bytes)
     return fail(FLS_ESIZE, "workspace has %llu bytes, %llu needed", (unsigned long long)b->workspace_bytes,
                 (unsigned long long)p->lay.workspace_bytes);
-  const uint32_t G = p->desc.groups, K = p->K;
+  const uint32_t G = p->desc.groups, K = p->K, C = p->n_copies;
   const uint64_t N = p->lay.n_padded;
   const uint64_t eg = p->desc.grad_dtype == FLS_GRAD_F32 ? 4 : 2;
 
@@ -351,7 +446,7 @@ int fls_plan_bind(fls_plan* p, const fls_buffers* b) {
     ranges.push_back(Range{reinterpret_cast<uintptr_t>(ptr), reinterpret_cast<uintptr_t>(ptr) + bytes, what, idx, output});
   };
   for (uint32_t i = 0; i < G * K; ++i) add(b->grads[i], N * eg, "grads", int(i), false);
-  for (uint32_t g = 0; g < G; ++g) {
+  for (uint32_t g = 0; g < C; ++g) {
     add(b->master[g], N * 4, "master", int(g), true);
     add(b->m[g], N * 4, "m", int(g), true);
     add(b->v[g], N * 4, "v", int(g), true);
@@ -362,33 +457,8 @@ int fls_plan_bind(fls_plan* p, const fls_buffers* b) {
   int dev = -1;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
-  for (const Range& r : ranges) {
-    if (r.lo == 0) return fail(FLS_EPTR, "%s[%d] is null", r.what, r.index);
-    if (r.lo % FLS_BUFFER_ALIGN != 0) return fail(FLS_EALIGN, "%s[%d] is not %d-byte aligned", r.what, r.index, FLS_BUFFER_ALIGN);
-    cudaPointerAttributes attr{};
-    e = cudaPointerGetAttributes(&attr, reinterpret_cast<const void*>(r.lo));
-    if (e != cudaSuccess) {
-      cudaGetLastError();
-      return fail(FLS_EPTR, "%s[%d]: %s", r.what, r.index, cudaGetErrorString(e));
-    }
-    if (attr.type != cudaMemoryTypeDevice && attr.type != cudaMemoryTypeManaged)
-      return fail(FLS_EPTR, "%s[%d] is not device memory", r.what, r.index);
-    if (attr.type == cudaMemoryTypeDevice && attr.device != dev)
-      return fail(FLS_EPTR, "%s[%d] lives on device %d, current device is %d", r.what, r.index, attr.device, dev);
-  }
-  // outputs may overlap nothing; gradient buffers may only overlap each other exactly (a caller may
-  // feed one buffer to several replicas) but never an output
-  std::vector<size_t> order(ranges.size());
-  for (size_t i = 0; i < order.size(); ++i) order[i] = i;
-  std::sort(order.begin(), order.end(), [&](size_t x, size_t y) { return ranges[x].lo < ranges[y].lo; });
-  for (size_t q = 0; q < order.size(); ++q) {
-    const Range& r0 = ranges[order[q]];
-    for (size_t w = q + 1; w < order.size() && ranges[order[w]].lo < r0.hi; ++w) {
-      const Range& r1 = ranges[order[w]];
-      if (r0.output || r1.output)
-        return fail(FLS_EPTR, "%s[%d] overlaps %s[%d]", r0.what, r0.index, r1.what, r1.index);
-    }
-  }
+  int rc = check_ranges(ranges, dev);
+  if (rc != FLS_OK) return rc;
 
   int sms = 0;
   e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -396,15 +466,20 @@ int fls_plan_bind(fls_plan* p, const fls_buffers* b) {
   p->device = dev;
   p->sm_count = sms;
   p->grads.assign(b->grads, b->grads + size_t(G) * K);
-  p->master.assign(b->master, b->master + G);
-  p->m.assign(b->m, b->m + G);
-  p->v.assign(b->v, b->v + G);
-  p->pbf16.resize(G);
-  for (uint32_t g = 0; g < G; ++g) p->pbf16[g] = static_cast<uint16_t*>(b->param_bf16[g]);
+  p->master.assign(b->master, b->master + C);
+  p->m.assign(b->m, b->m + C);
+  p->v.assign(b->v, b->v + C);
+  p->pbf16.resize(C);
+  for (uint32_t g = 0; g < C; ++g) p->pbf16[g] = static_cast<uint16_t*>(b->param_bf16[g]);
   p->ws = static_cast<char*>(b->workspace);
+  p->ranges = ranges;
+  p->master2.clear(); p->m2.clear(); p->v2.clear();   // a new binding drops the second buffer set
+  p->speculative = false;
 
   e = cudaMemset(p->ws, 0, size_t(kWsSegments));
   if (e != cudaSuccess) return cuda_fail(e, "cudaMemset(workspace head)");
+  e = cudaMemset(p->ws + p->lay.ws_chunk_count_offset, 0, size_t(p->lay.ws_chunk_count_bytes));
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMemset(norm counters)");
   e = cudaMemcpy(p->ws + kWsSegments, p->lay.segments.data(), p->lay.segments.size() * sizeof(Segment), cudaMemcpyHostToDevice);
   if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(segment table)");
   e = cudaDeviceSynchronize();
@@ -497,10 +572,18 @@ int fedavg_impl(fls_plan* p, const uint64_t* sample_counts, void* cuda_stream, c
   fa.G = G;
   fa.descending = p->descending[FLS_KERNEL_FEDAVG];
   const int n_arrays = (p->desc.fedavg_what & FLS_AVG_OPT_STATE) ? 3 : 1;
+  // with one state copy per replica only the first replica of every group aggregates; the others receive the result
+  const uint32_t R = p->R_state;
+  fa.n_extra = G * (R - 1);
   for (int arr = 0; arr < n_arrays; ++arr) {
+    const std::vector<float*>& src = arr == 0 ? p->master : (arr == 1 ? p->m : p->v);
     for (uint32_t g = 0; g < G; ++g) {
-      fa.x[g] = arr == 0 ? p->master[g] : (arr == 1 ? p->m[g] : p->v[g]);
-      fa.pbf16[g] = p->pbf16[g];
+      fa.x[g] = src[g * R];
+      fa.pbf16[g] = p->pbf16[g * R];
+      for (uint32_t r = 1; r < R; ++r) {
+        fa.x_extra[g * (R - 1) + r - 1] = src[g * R + r];
+        fa.pbf16_extra[g * (R - 1) + r - 1] = p->pbf16[g * R + r];
+      }
     }
     fa.write_bf16 = arr == 0 ? 1 : 0;
     const bool use_outer = outer && arr == 0;       // the outer optimizer acts on the parameters only
@@ -556,13 +639,22 @@ int fls_sync_step_fedavg(fls_plan* p, double lr, const uint64_t* sample_counts, 
   }
   const AdamScalars sc = adam_scalars(p->desc, lr, t_new);
   FusedArgs fa{};
+  const uint32_t R = p->R_state;
+  fa.replicas = R;
   for (uint32_t g = 0; g < G; ++g) {
     fa.gbar[g] = p->d_gbar(g);
-    fa.theta[g] = p->master[g];
-    fa.m[g] = p->m[g];
-    fa.v[g] = p->v[g];
-    fa.pbf16[g] = p->pbf16[g];
+    fa.theta[g] = p->master[g * R];
+    fa.m[g] = p->m[g * R];
+    fa.v[g] = p->v[g * R];
+    fa.pbf16[g] = p->pbf16[g * R];
     fa.w[g] = float((sample_counts ? double(sample_counts[g]) : 1.0) / double(total));
+    for (uint32_t r = 1; r < R; ++r) {
+      const uint32_t i = g * (R - 1) + r - 1;
+      fa.theta_extra[i] = p->master[g * R + r];
+      fa.m_extra[i] = p->m[g * R + r];
+      fa.v_extra[i] = p->v[g * R + r];
+      fa.pbf16_extra[i] = p->pbf16[g * R + r];
+    }
   }
   fa.coefs = p->d_coefs();
   fa.idx = p->seg_index();
@@ -619,7 +711,7 @@ int fls_comm_report(const fls_plan* p, const double* bw, fls_comm_costs* out) {
   if (bw)
     for (int i = 0; i < 3; ++i)
       if (!(bw[i] > 0.0)) return fail(FLS_EINVAL, "fls_comm_report: bandwidths must be positive");
-  comm_report(p->lay, p->desc, bw, out);
+  comm_report(p->lay, p->desc, p->route(), bw, out);
   return FLS_OK;
 }
 
@@ -635,17 +727,78 @@ int fls_plan_set_recompute(fls_plan* p, int mode) {
   if (!p) return fail(FLS_EINVAL, "fls_plan_set_recompute: null plan");
   const fls_plan_desc& d = p->desc;
   const bool small = uint64_t(p->K) * (d.grad_dtype == FLS_GRAD_F32 ? 4 : 2) < 8;
-  if (mode > 0 && (!small || d.reduce_wire != FLS_WIRE_F32))
-    return fail(FLS_ESTATE, "fls_plan_set_recompute: only for K*e_g < 8 bytes and fp32 partial sums");
-  p->recompute = mode > 0 || (mode < 0 && small && d.reduce_wire == FLS_WIRE_F32);
+  if (mode > 0 && (!small || !p->plain_reduce()))
+    return fail(FLS_ESTATE, "fls_plan_set_recompute: only for K*e_g < 8 bytes, fp32 partial sums in ascending order and one state copy per group");
+  p->recompute = mode > 0 || (mode < 0 && small && p->plain_reduce());
   return FLS_OK;
 }
 
 int fls_plan_set_single_pass(fls_plan* p, int mode) {
   if (!p) return fail(FLS_EINVAL, "fls_plan_set_single_pass: null plan");
-  const bool can = p->desc.reduce_wire == FLS_WIRE_F32 && !(p->desc.max_grad_norm > 0.0);
-  if (mode > 0 && !can) return fail(FLS_ESTATE, "fls_plan_set_single_pass: only for plans without clipping and with fp32 partial sums");
+  const bool can = p->plain_reduce() && !(p->desc.max_grad_norm > 0.0);
+  if (mode > 0 && !can)
+    return fail(FLS_ESTATE, "fls_plan_set_single_pass: only for plans without clipping, with fp32 partial sums in ascending order and one state copy per group");
   p->single_pass = mode > 0 || (mode < 0 && can);
+  return FLS_OK;
+}
+
+int fls_plan_bind_shadow(fls_plan* p, float* const* master, float* const* m, float* const* v) {
+  if (!p || !master || !m || !v) return fail(FLS_EINVAL, "fls_plan_bind_shadow: null argument");
+  if (!p->bound) return fail(FLS_ESTATE, "fls_plan_bind_shadow: bind the plan's buffers first");
+  if (p->R_state != 1) return fail(FLS_ESTATE, "fls_plan_bind_shadow: not for plans with one state copy per replica");
+  const uint32_t G = p->desc.groups;
+  const uint64_t N = p->lay.n_padded;
+  std::vector<Range> ranges = p->ranges;
+  for (uint32_t g = 0; g < G; ++g) {
+    const float* ptrs[3] = {master[g], m[g], v[g]};
+    const char* names[3] = {"shadow master", "shadow m", "shadow v"};
+    for (int i = 0; i < 3; ++i)
+      ranges.push_back(Range{reinterpret_cast<uintptr_t>(ptrs[i]), reinterpret_cast<uintptr_t>(ptrs[i]) + N * 4, names[i], int(g), true});
+  }
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+  if (dev != p->device) return fail(FLS_ESTATE, "fls_plan_bind_shadow: the plan was bound on device %d, current device is %d", p->device, dev);
+  const int rc = check_ranges(ranges, dev);
+  if (rc != FLS_OK) return rc;
+  p->master2.assign(master, master + G);
+  p->m2.assign(m, m + G);
+  p->v2.assign(v, v + G);
+  return FLS_OK;
+}
+
+int fls_plan_set_speculative(fls_plan* p, int enabled) {
+  if (!p) return fail(FLS_EINVAL, "fls_plan_set_speculative: null plan");
+  if (enabled) {
+    if (!p->bound || p->master2.empty()) return fail(FLS_ESTATE, "fls_plan_set_speculative: needs fls_plan_bind_shadow first");
+    if (!(p->desc.max_grad_norm > 0.0)) return fail(FLS_ESTATE, "fls_plan_set_speculative: the plan does not clip (it already runs a single pass)");
+    if (!p->plain_reduce())
+      return fail(FLS_ESTATE, "fls_plan_set_speculative: only with fp32 partial sums in ascending order and one state copy per group");
+  }
+  p->speculative = enabled != 0;
+  return FLS_OK;
+}
+
+int fls_get_spec_stats(const fls_plan* p, const uint32_t** dev_counts) {
+  if (!p || !dev_counts) return fail(FLS_EINVAL, "fls_get_spec_stats: null argument");
+  if (!p->bound) return fail(FLS_ESTATE, "fls_get_spec_stats: plan has no buffers bound");
+  *dev_counts = p->d_spec_counts();
+  return FLS_OK;
+}
+
+int fls_get_state(const fls_plan* p, uint32_t copy, float** master, float** m, float** v) {
+  if (!p) return fail(FLS_EINVAL, "fls_get_state: null plan");
+  if (!p->bound) return fail(FLS_ESTATE, "fls_get_state: plan has no buffers bound");
+  if (copy >= p->n_copies) return fail(FLS_EINVAL, "fls_get_state: copy %u of %u", copy, p->n_copies);
+  if (master) *master = p->master[copy];
+  if (m) *m = p->m[copy];
+  if (v) *v = p->v[copy];
+  return FLS_OK;
+}
+
+int fls_plan_set_l2_keep(fls_plan* p, uint64_t bytes) {
+  if (!p) return fail(FLS_EINVAL, "fls_plan_set_l2_keep: null plan");
+  p->l2_keep_bytes = bytes;
   return FLS_OK;
 }
 

@@ -3,15 +3,16 @@
 // and 256-bit (fp32) global accesses.  By default the grid covers the whole buffer in one pass (no
 // grid-stride loop): the hardware scheduler hands out CTAs in order, so the tiles in flight form a
 // compact window that moves through memory and the SMs stay balanced, which measured 5-15 % faster
-// than persistent grid-stride CTAs.  The kernels are kept small in registers (32-66) so that 1024-2048
+// than persistent grid-stride CTAs.  The kernels are kept small in registers (32-72) so that 768-2048
 // threads are resident per SM; that, not unrolling, is what keeps enough loads in flight.
 // No shared-memory staging and no tensor cores: nothing here is a contraction, and each byte is touched
 // once.
 //
-//   fls_reduce_kernel  : K gradient buffers -> mean gradient (fp32, shard order) + squared-norm partials;
-//                        the last CTA to finish adds the partials in index order and writes the group's
-//                        norm and clip coefficient (no floating-point atomics: the result does not depend
-//                        on which CTA is last).
+//   fls_reduce_kernel  : K gradient buffers -> mean gradient (fp32, shard order) + squared-norm partials,
+//                        added up over a fixed tree (warp, CTA, chunk of CTAs, grid) by whoever arrives last
+//                        at each level; the last of all writes the group's norm and clip coefficient (no
+//                        floating-point atomics, no block-wide barrier: the result does not depend on the
+//                        order of arrival).
 //   fls_adamw_kernel   : clip + AdamW on master/m/v in place + bf16 copy in unsharded order.
 //   fls_fedavg_kernel  : weighted average of G copies written back to all G (+ bf16 copies).
 #include <cuda_bf16.h>
@@ -50,7 +51,8 @@ __device__ __forceinline__ F8 ld8_keep(const float* p) {
 __device__ __forceinline__ void st8_stream(float* p, const F8& r) {
   asm volatile("st.global.L1::no_allocate.L2::evict_first.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" :: "l"(p), FLS_U8(r) : "memory");
 }
-// the reduced gradient is the one stream that is read again (by the next kernel): ask L2 to evict it last
+// the reduced gradient is the one stream that is read again (by the next kernel): its last part, which that
+// kernel reads first, is stored with "evict last" so that it is still in L2 by then
 __device__ __forceinline__ void st8_keep(float* p, const F8& r) {
   asm volatile("st.global.L2::evict_last.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" :: "l"(p), FLS_U8(r) : "memory");
 }
@@ -117,7 +119,7 @@ __device__ __forceinline__ uint32_t find_segment(const SegIndex& ix, uint32_t ti
 
 // Per-thread slice of a tile: n = number of valid elements (0..8), vec = whole 8 on the vector path.
 // `lane` is the thread's index inside the 256-thread group that owns the tile.
-struct Slice { uint64_t j, a; uint32_t n; bool vec; };
+struct Slice { uint64_t j, a, e; uint32_t n; bool vec; };   // e: position of the first element inside its segment
 __device__ __forceinline__ Slice slice_of(const Segment* sg, uint32_t tile, uint32_t lane) {
   Slice r;
   const uint64_t e0 = (uint64_t(tile) - __ldg(&sg->tile_begin)) * kTile + lane * kVec;
@@ -127,6 +129,7 @@ __device__ __forceinline__ Slice slice_of(const Segment* sg, uint32_t tile, uint
   r.vec = __ldg(&sg->aligned) && r.n == kVec;
   r.j = __ldg(&sg->j0) + e0;
   r.a = __ldg(&sg->a0) + e0;
+  r.e = e0;
   return r;
 }
 
@@ -148,23 +151,11 @@ struct Walker {
   }
 };
 
-// Fixed-shape block sum of one double per thread (shuffle tree inside a warp, then warp 0 over the
-// per-warp results): same order every run.  Result valid in thread 0.
-template <int THREADS>
-__device__ __forceinline__ double block_sum(double x, double* sh) {
+// Sum over the lanes of a warp in a fixed (butterfly) order: every lane ends with the same bits.
+__device__ __forceinline__ double warp_sum(double x) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, o);
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  __syncthreads();
-  if (lane == 0) sh[warp] = x;
-  __syncthreads();
-  double t = 0.0;
-  if (warp == 0) {
-    t = lane < THREADS / 32 ? sh[lane] : 0.0;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, o);
-  }
-  return t;
+  return x;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -212,7 +203,19 @@ __device__ __forceinline__ void unpack(const Raw<1, true>& x, float (&f)[1]) { f
 //   SG = 1, 2, 4 : S == SG, a batch holds whole groups of SG buffers.
 //   SG = -1 : any other shape; bit k of end_mask says that buffer k closes a group.
 //   SG = -2 : as -1, with every partial sum and the final mean rounded to bf16 (the bf16-wire emulation).
+// Ring order (SG < 0 only, a.ring set): the q-th buffer visited is not buffer q but the one a ring would add
+// q-th.  For an element owned by rank s after the reduce-scatter and lying in sub-chunk c of the all-reduce
+// across replicas (sc = s | c << 16), the shard level adds sigma = s+1, s+2, ..., s (mod S) inside each replica
+// and the replicate level adds rho = c+1, ..., c (mod R): the owner's contribution comes last at both levels.
 __device__ __forceinline__ float round_bf16(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
+
+__device__ __forceinline__ uint32_t ring_buffer(const ReduceArgs& a, uint32_t sc, uint32_t q) {
+  const uint32_t lvl = q / a.S, pos = q - lvl * a.S;
+  uint32_t sigma = (sc & 0xFFFFu) + 1 + pos, rho = (sc >> 16) + 1 + lvl;
+  if (sigma >= a.S) sigma -= a.S;
+  if (rho >= a.R) rho -= a.R;
+  return rho * a.S + sigma;
+}
 
 // one scaling by 1/K after the last level: a multiply when 1/K is exact, else an IEEE division
 template <int N>
@@ -266,7 +269,7 @@ __device__ __forceinline__ void combine_loaded(const ReduceArgs& a, const Raw<N,
 }
 
 template <int N, bool F32, int KT, int SG>
-__device__ __forceinline__ void reduce_elems(const ReduceArgs& a, uint64_t j, float (&mean)[N]) {
+__device__ __forceinline__ void reduce_elems(const ReduceArgs& a, uint64_t j, float (&mean)[N], uint32_t sc = 0) {
   if constexpr (KT > 0 && SG >= 0) {
     Raw<N, F32> raw[KT];
 #pragma unroll
@@ -281,9 +284,15 @@ __device__ __forceinline__ void reduce_elems(const ReduceArgs& a, uint64_t j, fl
 #pragma unroll 1
     for (uint32_t k0 = 0; k0 < K; k0 += 8) {
       Raw<N, F32> raw[8];
+      if (SG < 0 && a.ring) {
 #pragma unroll
-      for (int b = 0; b < 8; ++b)
-        if (k0 + b < K) load_raw(raw[b], a.grad[k0 + b], j);
+        for (int b = 0; b < 8; ++b)
+          if (k0 + b < K) load_raw(raw[b], a.grad[ring_buffer(a, sc, k0 + b)], j);
+      } else {
+#pragma unroll
+        for (int b = 0; b < 8; ++b)
+          if (k0 + b < K) load_raw(raw[b], a.grad[k0 + b], j);
+      }
       if constexpr (SG == 0) {
 #pragma unroll
         for (int b = 0; b < 8; ++b) {
@@ -342,76 +351,134 @@ __device__ __forceinline__ void reduce_elems(const ReduceArgs& a, uint64_t j, fl
 
 // element-wise path of one thread's slice (unaligned runs and ragged tails); kept out of line so that
 // it does not cost the vector path registers
+// ring order (a.ring): seg is the slice's segment (it names the owning rank and the all-reduce sub-chunk length) and
+// pos the position of the slice's first element inside it; otherwise both are ignored
 template <bool F32, bool WIRE>
-__device__ __noinline__ float reduce_slice_scalar(const ReduceArgs& a, uint64_t j, uint64_t addr, uint32_t n) {
+__device__ __noinline__ float reduce_slice_scalar(const ReduceArgs& a, uint64_t j, uint64_t addr, uint32_t n, const Segment* seg,
+                                                  uint64_t pos) {
   float sq = 0.f;
+  uint32_t shard = 0;
+  uint64_t sub_len = 1;
+  if (a.ring) {
+    shard = uint32_t(__ldg(&seg->shard));
+    sub_len = __ldg(&seg->sub_len);
+  }
   for (uint32_t e = 0; e < n; ++e) {
     float g[1];
-    reduce_elems<1, F32, 0, WIRE ? -2 : -1>(a, j + e, g);
+    const uint32_t sc = a.ring ? (shard | uint32_t((pos + e) / sub_len) << 16) : 0u;
+    reduce_elems<1, F32, 0, WIRE ? -2 : -1>(a, j + e, g, sc);
     if (a.store_gbar) a.gbar[addr + e] = g[0];
     sq = fmaf(g[0], g[0], sq);
   }
   return sq;
 }
 
-// End of every kernel that computes the norm: CTA partial -> workspace; the CTA that takes the last ticket adds
-// all partials in index order (so the norm does not depend on the order in which CTAs finish), then writes the
-// group's norm and clip coefficient and re-arms the ticket.  Must be reached by all threads of the CTA.
+// End of every kernel that computes the norm.  The squared norm is added up over a fixed tree, so the result
+// does not depend on the order in which warps or CTAs finish (no floating-point atomics), and without any
+// block-wide barrier, so that a warp that is done never waits for the slowest warp of its CTA:
+//   thread: fp32 sum of its 8 squares -> warp: butterfly in double -> CTA: the LAST WARP TO ARRIVE (a shared
+//   counter) adds the warp sums in index order -> chunk of kNormChunk consecutive CTAs: the last CTA of the chunk
+//   to arrive (one global counter per chunk) adds the chunk's CTA partials in index order -> grid: the last chunk
+//   to arrive (the ticket) adds the chunk sums in index order, writes the group's norm and clip coefficient and
+//   re-arms the ticket; every chunk counter is re-armed by the warp that closes the chunk.
+// The caller must have zeroed *arrived (shared) behind a __syncthreads() at the start of the kernel.
+constexpr unsigned kNormChunk = kNormChunkCtas;
+
 template <int THREADS>
-__device__ __forceinline__ void finish_norm(const ReduceArgs& a, float sq) {
-  __shared__ double sh[THREADS / 32];
-  __shared__ bool is_last;
-  double total = block_sum<THREADS>(double(sq), sh);
-  if (threadIdx.x == 0) {
-    a.partials[blockIdx.x] = total;
-    __threadfence();
-    const uint32_t ticket = atomicAdd(a.ticket, 1u);
-    is_last = (ticket == gridDim.x - 1);
+__device__ __forceinline__ void finish_norm(const ReduceArgs& a, float sq, unsigned* arrived) {
+  constexpr int W = THREADS / 32;
+  __shared__ double sh[W];
+  const double x = warp_sum(double(sq));
+  const unsigned lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+  unsigned t = 0;
+  if (lane == 0) {
+    sh[warp] = x;
+    __threadfence_block();
+    t = atomicAdd(arrived, 1u);
   }
-  __syncthreads();
-  if (!is_last) return;
+  if (__shfl_sync(0xFFFFFFFFu, t, 0) != W - 1) return;
+  __threadfence_block();
+  const double cta = warp_sum(lane < W ? sh[lane] : 0.0);
+  const unsigned chunk = blockIdx.x / kNormChunk, n_chunks = (gridDim.x + kNormChunk - 1) / kNormChunk;
+  const unsigned chunk_size = min(kNormChunk, gridDim.x - chunk * kNormChunk);
+  if (lane == 0) {
+    a.partials[blockIdx.x] = cta;
+    __threadfence();
+    t = atomicAdd(a.chunk_count + chunk, 1u);
+  }
+  if (__shfl_sync(0xFFFFFFFFu, t, 0) != chunk_size - 1) return;
   __threadfence();
-  double s = 0.0;
-  for (uint32_t i = threadIdx.x; i < gridDim.x; i += THREADS) s += __ldcg(a.partials + i);
-  total = block_sum<THREADS>(s, sh);
-  if (threadIdx.x == 0) {
+  double c = 0.0;
+  for (unsigned i = lane; i < chunk_size; i += 32) c += __ldcg(a.partials + size_t(chunk) * kNormChunk + i);
+  c = warp_sum(c);
+  if (lane == 0) {
+    a.chunk_partials[chunk] = c;
+    a.chunk_count[chunk] = 0u;           // ready for the next launch (stream order)
+    __threadfence();
+    t = atomicAdd(a.ticket, 1u);
+  }
+  if (__shfl_sync(0xFFFFFFFFu, t, 0) != n_chunks - 1) return;
+  __threadfence();
+  double total = 0.0;
+  for (unsigned i = lane; i < n_chunks; i += 32) total += __ldcg(a.chunk_partials + i);
+  total = warp_sum(total);
+  if (lane == 0) {
     const double nrm = sqrt(total);
-    double c = 1.0;
+    double c1 = 1.0;
     if (a.max_grad_norm > 0.0) {
-      c = a.max_grad_norm / (nrm + 1e-6);
-      if (c >= 1.0) c = 1.0;            // NaN compares false and stays NaN: non-finite norms propagate
+      c1 = a.max_grad_norm / (nrm + 1e-6);
+      if (c1 >= 1.0) c1 = 1.0;          // NaN compares false and stays NaN: non-finite norms propagate
     }
     *a.normsq_out = total;
     *a.norm_out = float(nrm);
-    *a.coef_out = float(c);
+    *a.coef_out = float(c1);
     if (!isfinite(nrm)) atomicOr(a.status, uint32_t(FLS_STATUS_NONFINITE_NORM));
+    if (a.spec_counts) atomicAdd(a.spec_counts + (float(c1) == 1.0f ? 0 : 1), 1u);   // speculative step: kept / redone
     *a.ticket = 0u;                      // ready for the next launch (stream order)
   }
 }
 
+// Start of the same kernels: arm the CTA's arrival counter.
+__device__ __forceinline__ void begin_norm(unsigned* arrived) {
+  if (threadIdx.x == 0) *arrived = 0u;
+  __syncthreads();
+}
+
 // One pass, no loop: a CTA of THREADS threads owns U * THREADS/256 consecutive tiles (each group of 256
 // threads takes every (THREADS/256)-th of them, U in all) and the grid covers the whole buffer.  MINB resident
-// CTAs per SM fix the register budget: 1024 x 2 (32 registers) for the flat order with K = 4 or 8, 512 x 3 (42
+// CTAs per SM fix the register budget: 256 x 8 (32 registers) for the flat order with K = 4 or 8, 256 x 6 (40
 // registers) for the two-level orders, which carry a second set of accumulators, 256 x 2 for a run-time K.
+// Small CTAs turn over independently (no warp waits for the slowest of 32); they became the fastest shape once
+// the norm epilogue lost its block-wide barriers.
 // With K = 1 or 2 a thread would have only one or two 16-byte loads in flight, so those shapes take U > 1 tiles
 // per thread (512 x 2 CTAs) and issue the loads of all of them before the first add.
 template <bool F32, int KT, int SG>
 __device__ __forceinline__ float reduce_one_tile(const ReduceArgs& a, uint32_t tile, uint32_t lane) {
   float sq = 0.f;
-  const Slice s = slice_of(a.idx.segs + find_segment(a.idx, tile), tile, lane);
-  if (s.vec) {
+  const Segment* seg = a.idx.segs + find_segment(a.idx, tile);
+  const Slice s = slice_of(seg, tile, lane);
+  bool vec = s.vec;
+  uint32_t sc = 0;
+  if (SG < 0 && a.ring) {
+    // the eight elements of a vector access must share one all-reduce sub-chunk, else they go one by one
+    const uint64_t sub_len = __ldg(&seg->sub_len);
+    const uint64_t c0 = s.e / sub_len;
+    vec = vec && (s.e + kVec - 1) / sub_len == c0;
+    sc = uint32_t(__ldg(&seg->shard)) | uint32_t(c0) << 16;
+  }
+  if (vec) {
     float g[8];
-    reduce_elems<8, F32, KT, SG>(a, s.j, g);
+    reduce_elems<8, F32, KT, SG>(a, s.j, g, sc);
     F8 o;
 #pragma unroll
     for (int e = 0; e < 8; ++e) { o.v[e] = g[e]; sq = fmaf(g[e], g[e], sq); }
     if (a.store_gbar) {
       dep_wait();                        // the previous group's AdamW kernel may still be reading the scratch
-      st8_keep(a.gbar + s.a, o);
+      if (tile >= a.keep_from_tile) st8_keep(a.gbar + s.a, o); else st8_stream(a.gbar + s.a, o);
     }
   } else if (s.n) {
     dep_wait();
-    sq = reduce_slice_scalar<F32, SG == -2>(a, s.j, s.a, s.n);
+    sq = reduce_slice_scalar<F32, SG == -2>(a, s.j, s.a, s.n, seg, s.e);
   }
   return sq;
 }
@@ -419,6 +486,8 @@ __device__ __forceinline__ float reduce_one_tile(const ReduceArgs& a, uint32_t t
 template <bool F32, int KT, int SG, int THREADS, int MINB, int U>
 __global__ void __launch_bounds__(THREADS, MINB) fls_reduce_kernel(const __grid_constant__ ReduceArgs a) {
   constexpr uint32_t T = THREADS / kThreads;
+  __shared__ unsigned arrived;
+  begin_norm(&arrived);
   const uint32_t lane = threadIdx.x % kThreads;
   const uint32_t first = blockIdx.x * (T * U) + threadIdx.x / kThreads;   // this thread's tiles: first + u*T
   float sq = 0.f;
@@ -458,7 +527,9 @@ __global__ void __launch_bounds__(THREADS, MINB) fls_reduce_kernel(const __grid_
 #pragma unroll
         for (int e = 0; e < 8; ++e) { o.v[e] = g[e]; s8 = fmaf(g[e], g[e], s8); }
         sq += s8;
-        if (a.store_gbar) st8_keep(a.gbar + a0 + u * stride, o);
+        if (a.store_gbar) {
+          if (first + u * T >= a.keep_from_tile) st8_keep(a.gbar + a0 + u * stride, o); else st8_stream(a.gbar + a0 + u * stride, o);
+        }
       }
     } else {
       for (int u = 0; u < U; ++u) {
@@ -469,7 +540,7 @@ __global__ void __launch_bounds__(THREADS, MINB) fls_reduce_kernel(const __grid_
   }
   dep_wait();                            // partials, ticket and the norm slots belong to the predecessor until now
   dep_launch();
-  finish_norm<THREADS>(a, sq);
+  finish_norm<THREADS>(a, sq, &arrived);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -535,11 +606,15 @@ __device__ __noinline__ void reduce_adamw_slice_scalar(const ReduceAdamArgs& p, 
     reduce_elems<1, F32, 0, -1>(p.r, j + e, g);
     float th = a.theta[addr + e], m = a.m[addr + e], v = a.v[addr + e];
     adamw_one(a, c, g[0], th, m, v);
-    a.theta[addr + e] = th; a.m[addr + e] = m; a.v[addr + e] = v;
+    a.theta_out[addr + e] = th; a.m_out[addr + e] = m; a.v_out[addr + e] = v;
     a.pbf16[j + e] = to_bf16_bits(th);
   }
 }
 
+// skip_if_unclipped: this launch is the second kernel of a speculative step.  The first one applied AdamW with
+// coefficient 1 while it computed the norm; if the coefficient turned out to be 1 its result stands and this
+// kernel has nothing to do; otherwise it redoes the step with the real coefficient, reading the same (untouched)
+// input state and overwriting the same output buffers.
 template <bool F32, int KT, int SG>
 __global__ void __launch_bounds__(kThreads, KT == 0 ? 2 : 4) fls_reduce_adamw_kernel(const __grid_constant__ ReduceAdamArgs p) {
   const AdamArgs& a = p.a;
@@ -547,6 +622,13 @@ __global__ void __launch_bounds__(kThreads, KT == 0 ? 2 : 4) fls_reduce_adamw_ke
   if (blockIdx.x >= n_tiles) { dep_wait(); dep_launch(); return; }
   float c = 0.f;
   bool waited = false;
+  if (p.skip_if_unclipped) {
+    dep_wait();
+    dep_launch();
+    c = __ldcg(a.coef);
+    waited = true;
+    if (c == 1.0f) return;
+  }
   Walker w;
   w.init(a.idx, a.descending ? n_tiles - 1 - blockIdx.x : blockIdx.x);
   for (uint32_t lin = blockIdx.x; lin < n_tiles; lin += gridDim.x) {
@@ -562,9 +644,9 @@ __global__ void __launch_bounds__(kThreads, KT == 0 ? 2 : 4) fls_reduce_adamw_ke
       if (!waited) { dep_wait(); dep_launch(); c = __ldcg(a.coef); waited = true; }
 #pragma unroll
       for (int e = 0; e < 8; ++e) adamw_one(a, c, g[e], th.v[e], m.v[e], v.v[e]);
-      st8_stream(a.theta + s.a, th);
-      st8_stream(a.m + s.a, m);
-      st8_stream(a.v + s.a, v);
+      st8_stream(a.theta_out + s.a, th);
+      st8_stream(a.m_out + s.a, m);
+      st8_stream(a.v_out + s.a, v);
       st_b128_stream(a.pbf16 + s.j, pack_bf16x8(th));
     } else if (s.n) {
       if (!waited) { dep_wait(); dep_launch(); c = __ldcg(a.coef); waited = true; }
@@ -575,13 +657,18 @@ __global__ void __launch_bounds__(kThreads, KT == 0 ? 2 : 4) fls_reduce_adamw_ke
 }
 
 // Whole step in one pass, for plans without clipping: the clip coefficient is 1 whatever the norm turns out
-// to be, so AdamW does not have to wait for it.  One 256-thread CTA per tile forms the mean gradient, applies
+// to be, so AdamW does not have to wait for it.  Plans that clip use the same kernel as the first half of a
+// speculative step: it writes the new state to the plan's second buffer set (theta_out, m_out, v_out) and the
+// coefficient it computes at the end tells the follow-up kernel whether the guess "1" held.  One 256-thread CTA per tile forms the mean gradient, applies
 // AdamW and contributes to the norm (still reported): K*e_g + 26 bytes per element instead of K*e_g + 34.
 // theta, m and v come out bit-identical to the two-pass route (there the gradient is multiplied by exactly 1).
-// (4 CTAs per SM measured best: 2 and 3 leave loads in flight on the table, 5 and 6 spill)
+// (4 CTAs per SM measured best for a static K: 2 and 3 leave loads in flight on the table, 5 and 6 spill; the
+// run-time-K form holds a batch of eight raw loads next to the state and needs the registers of 2 CTAs per SM)
 template <bool F32, int KT, int SG>
-__global__ void __launch_bounds__(kThreads, 4) fls_step_noclip_kernel(const __grid_constant__ ReduceAdamArgs p) {
+__global__ void __launch_bounds__(kThreads, KT == 0 ? 2 : 4) fls_step_noclip_kernel(const __grid_constant__ ReduceAdamArgs p) {
   const AdamArgs& a = p.a;
+  __shared__ unsigned arrived;
+  begin_norm(&arrived);
   float sq = 0.f;
   const uint32_t tile = blockIdx.x;        // the grid covers every tile exactly once
   const Slice s = slice_of(a.idx.segs + find_segment(a.idx, tile), tile, threadIdx.x);
@@ -598,9 +685,9 @@ __global__ void __launch_bounds__(kThreads, 4) fls_step_noclip_kernel(const __gr
       adamw_one(a, 1.0f, g[e], th.v[e], m.v[e], v.v[e]);
     }
     dep_wait();
-    st8_stream(a.theta + s.a, th);
-    st8_stream(a.m + s.a, m);
-    st8_stream(a.v + s.a, v);
+    st8_stream(a.theta_out + s.a, th);
+    st8_stream(a.m_out + s.a, m);
+    st8_stream(a.v_out + s.a, v);
     st_b128_stream(a.pbf16 + s.j, pack_bf16x8(th));
   } else if (s.n) {
     dep_wait();
@@ -610,13 +697,13 @@ __global__ void __launch_bounds__(kThreads, 4) fls_step_noclip_kernel(const __gr
       sq = fmaf(g[0], g[0], sq);
       float th = a.theta[s.a + e], m = a.m[s.a + e], v = a.v[s.a + e];
       adamw_one(a, 1.0f, g[0], th, m, v);
-      a.theta[s.a + e] = th; a.m[s.a + e] = m; a.v[s.a + e] = v;
+      a.theta_out[s.a + e] = th; a.m_out[s.a + e] = m; a.v_out[s.a + e] = v;
       a.pbf16[s.j + e] = to_bf16_bits(th);
     }
   }
   dep_wait();
   dep_launch();
-  finish_norm<kThreads>(p.r, sq);
+  finish_norm<kThreads>(p.r, sq, &arrived);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -643,9 +730,11 @@ __device__ __noinline__ void fedavg_slice_scalar(const FedavgArgs& a, uint64_t j
       a.outer_buf[addr + e] = b;
     }
     for (uint32_t g = 0; g < a.G; ++g) a.x[g][addr + e] = acc;
+    for (uint32_t i = 0; i < a.n_extra; ++i) a.x_extra[i][addr + e] = acc;
     if (a.write_bf16) {
       const uint16_t b = to_bf16_bits(acc);
       for (uint32_t g = 0; g < a.G; ++g) a.pbf16[g][j + e] = b;
+      for (uint32_t i = 0; i < a.n_extra; ++i) a.pbf16_extra[i][j + e] = b;
     }
   }
 }
@@ -696,6 +785,8 @@ __global__ void __launch_bounds__(kThreads, MINB) fls_fedavg_kernel(const __grid
       } else {
         for (uint32_t g = 0; g < G; ++g) st8_stream(a.x[g] + s.a, acc);
       }
+      // the broadcast inside each group: the other replicas' copies receive the same values
+      for (uint32_t i = 0; i < a.n_extra; ++i) st8_stream(a.x_extra[i] + s.a, acc);
       if (a.write_bf16) {
         const uint4 p = pack_bf16x8(acc);
         if constexpr (GT != 0) {
@@ -704,6 +795,7 @@ __global__ void __launch_bounds__(kThreads, MINB) fls_fedavg_kernel(const __grid
         } else {
           for (uint32_t g = 0; g < G; ++g) st_b128_stream(a.pbf16[g] + s.j, p);
         }
+        for (uint32_t i = 0; i < a.n_extra; ++i) st_b128_stream(a.pbf16_extra[i] + s.j, p);
       }
     } else if (s.n) {
       fedavg_slice_scalar(a, s.j, s.a, s.n);
@@ -735,13 +827,24 @@ __device__ __noinline__ void fused_slice_scalar(const FusedArgs& a, uint64_t j, 
       adamw_one_f(a, __ldcg(a.coefs + g), a.gbar[g][addr + e], th, m, v);
       ath = fmaf(a.w[g], th, ath);
       if (a.avg_opt_state) { am = fmaf(a.w[g], m, am); av = fmaf(a.w[g], v, av); }
-      else { a.m[g][addr + e] = m; a.v[g][addr + e] = v; }
+      else {
+        a.m[g][addr + e] = m; a.v[g][addr + e] = v;
+        for (uint32_t r = 0; r + 1 < a.replicas; ++r) {
+          const uint32_t i = g * (a.replicas - 1) + r;
+          a.m_extra[i][addr + e] = m; a.v_extra[i][addr + e] = v;
+        }
+      }
     }
     const uint16_t b = to_bf16_bits(ath);
     for (uint32_t g = 0; g < a.G; ++g) {
       a.theta[g][addr + e] = ath;
       a.pbf16[g][j + e] = b;
       if (a.avg_opt_state) { a.m[g][addr + e] = am; a.v[g][addr + e] = av; }
+    }
+    for (uint32_t i = 0; i < a.G * (a.replicas - 1); ++i) {
+      a.theta_extra[i][addr + e] = ath;
+      a.pbf16_extra[i][j + e] = b;
+      if (a.avg_opt_state) { a.m_extra[i][addr + e] = am; a.v_extra[i][addr + e] = av; }
     }
   }
 }
@@ -775,13 +878,25 @@ __global__ void __launch_bounds__(kThreads, 3) fls_adamw_fedavg_kernel(const __g
           ath.v[e] = fmaf(wg, th.v[e], ath.v[e]);
           if (OPT) { am.v[e] = fmaf(wg, m.v[e], am.v[e]); av.v[e] = fmaf(wg, v.v[e], av.v[e]); }
         }
-        if (!OPT) { st8_stream(a.m[g] + s.a, m); st8_stream(a.v[g] + s.a, v); }
+        if (!OPT) {
+          st8_stream(a.m[g] + s.a, m); st8_stream(a.v[g] + s.a, v);
+          // the group's other replicas ran the same update on the same gradient: they get the same moments
+          for (uint32_t r = 0; r + 1 < a.replicas; ++r) {
+            const uint32_t i = g * (a.replicas - 1) + r;
+            st8_stream(a.m_extra[i] + s.a, m); st8_stream(a.v_extra[i] + s.a, v);
+          }
+        }
       }
       const uint4 p = pack_bf16x8(ath);
       for (uint32_t g = 0; g < a.G; ++g) {
         st8_stream(a.theta[g] + s.a, ath);
         st_b128_stream(a.pbf16[g] + s.j, p);
         if (OPT) { st8_stream(a.m[g] + s.a, am); st8_stream(a.v[g] + s.a, av); }
+      }
+      for (uint32_t i = 0; i < a.G * (a.replicas - 1); ++i) {     // the broadcast to the other replicas of every group
+        st8_stream(a.theta_extra[i] + s.a, ath);
+        st_b128_stream(a.pbf16_extra[i] + s.j, p);
+        if (OPT) { st8_stream(a.m_extra[i] + s.a, am); st8_stream(a.v_extra[i] + s.a, av); }
       }
     } else if (s.n) {
       if (!waited) { dep_wait(); dep_launch(); waited = true; }
@@ -795,12 +910,12 @@ __global__ void __launch_bounds__(kThreads, 3) fls_adamw_fedavg_kernel(const __g
 // Launchers.
 // ------------------------------------------------------------------------------------------------
 #ifndef FLS_FLAT_THREADS
-#define FLS_FLAT_THREADS 1024
-#define FLS_FLAT_MINB 2
+#define FLS_FLAT_THREADS 256
+#define FLS_FLAT_MINB 8
 #endif
 #ifndef FLS_LEVEL_THREADS
-#define FLS_LEVEL_THREADS 512
-#define FLS_LEVEL_MINB 3
+#define FLS_LEVEL_THREADS 256
+#define FLS_LEVEL_MINB 6
 #endif
 constexpr int kFlatThreads = FLS_FLAT_THREADS, kFlatMinB = FLS_FLAT_MINB;       // SG == 0 with a static K
 constexpr int kLevelThreads = FLS_LEVEL_THREADS, kLevelMinB = FLS_LEVEL_MINB;   // two-level orders with a static K
@@ -922,10 +1037,17 @@ cudaError_t launch_step_noclip(const ReduceAdamArgs& a, bool f32, int sg, cudaSt
 }
 
 cudaError_t launch_reduce_adamw(const ReduceAdamArgs& a, bool f32, int sg, unsigned grid, cudaStream_t st, bool overlap) {
-  // the recompute plan exists for K * e_g < 8: bf16 with K <= 3, fp32 with K = 1
+  // static shapes for the recompute plan (K * e_g < 8: bf16 with K <= 3, fp32 with K = 1); any other K, which only
+  // the redo of a speculative step brings here, takes the run-time-K form
   const uint32_t K = a.r.K;
-  if (f32) {
+  if (f32 && K == 1) {
     launch_k(fls_reduce_adamw_kernel<true, 1, 0>, a, grid, kThreads, st, overlap);
+  } else if (f32 && sg == 0) {
+    launch_k(fls_reduce_adamw_kernel<true, 0, 0>, a, grid, kThreads, st, overlap);
+  } else if (f32 && sg == 1) {
+    launch_k(fls_reduce_adamw_kernel<true, 0, 1>, a, grid, kThreads, st, overlap);
+  } else if (f32) {
+    launch_k(fls_reduce_adamw_kernel<true, 0, -1>, a, grid, kThreads, st, overlap);
   } else if (K == 1) {
     launch_k(fls_reduce_adamw_kernel<false, 1, 0>, a, grid, kThreads, st, overlap);
   } else if (K == 2 && sg == 0) {

@@ -6,6 +6,8 @@
 
 namespace fls {
 
+constexpr int FLS_MAX_FUSED_EXTRA = 32;    // extra state copies (G*(R_rep-1)) the fused aggregation kernel can serve
+
 // Where the tiles of each segment end, for the tile -> segment search.  Small tables (the usual case)
 // are also copied here so that the search runs out of the kernel parameters (constant bank) instead of
 // global memory; the segment record itself is then one global load.
@@ -24,9 +26,13 @@ struct ReduceArgs {
   uint32_t K;
   float k_float, inv_k;                    // K and 1/K as float: the mean is scaled by 1/K once
   uint32_t k_is_pow2;                      // 1/K exact: multiply; otherwise divide
+  uint32_t keep_from_tile;                 // tiles from this one on store the mean gradient with L2::evict_last (the
+                                           // AdamW kernel reads them first), the others with evict_first
   uint32_t fold_mask;                      // bit i set: the i-th batch of 8 buffers closes a sharding group
   uint64_t end_mask;                       // bit k set: buffer k closes a sharding group
   double* partials;                        // device, one per CTA
+  double* chunk_partials;                  // device, one per chunk of 256 CTAs
+  uint32_t* chunk_count;                   // device, one per chunk, zero between launches
   uint32_t* ticket;                        // device, zero between launches
   float* norm_out;
   float* coef_out;
@@ -34,11 +40,17 @@ struct ReduceArgs {
   uint32_t* status;
   double max_grad_norm;
   int store_gbar;                          // 0: norm only (the recompute plan: the mean gradient is formed again in AdamW)
+  // ring order (generic kernels only): visit the buffers as a ring reduce-scatter / all-reduce would
+  uint32_t ring;                           // 0: ascending buffer index at both levels
+  uint32_t S, R;                           // shard_dim, replicate_dim (used by the ring order)
+  uint32_t* spec_counts;                   // device, 2 counters (coefficient == 1, != 1) or null: speculative steps only
 };
 
 struct AdamArgs {
   const float* gbar;
-  float *theta, *m, *v;
+  float *theta, *m, *v;                    // state read (and, in fls_adamw_kernel, updated in place)
+  float *theta_out, *m_out, *v_out;        // where the kernels that form the gradient themselves store the new state
+                                           // (the same three pointers, or the other buffer set of a speculative plan)
   uint16_t* pbf16;
   SegIndex idx;
   int descending;
@@ -50,12 +62,18 @@ struct AdamArgs {
 struct ReduceAdamArgs {
   ReduceArgs r;                            // gradient pointers, level structure, 1/K (its outputs are not used)
   AdamArgs a;                              // state pointers, scalars (its gbar is not used)
+  int skip_if_unclipped;                   // second kernel of a speculative step: return at once if the coefficient is 1
 };
 
 struct FedavgArgs {
   float* x[FLS_MAX_GROUPS];                // device, the G copies (in/out)
   uint16_t* pbf16[FLS_MAX_GROUPS];         // device, the G bf16 copies (out), used if write_bf16
   float w[FLS_MAX_GROUPS];
+  // plans with one state copy per replica: x[] holds replica 0 of every group (the one that aggregates); the
+  // average is also stored ("broadcast") to the other copies listed here
+  float* x_extra[FLS_MAX_GROUPS];
+  uint16_t* pbf16_extra[FLS_MAX_GROUPS];
+  uint32_t n_extra;
   SegIndex idx;
   uint32_t G;
   int write_bf16;
@@ -75,6 +93,13 @@ struct FusedArgs {
   float* v[FLS_MAX_FUSED_GROUPS];
   uint16_t* pbf16[FLS_MAX_FUSED_GROUPS];
   float w[FLS_MAX_FUSED_GROUPS];
+  // plans with one state copy per replica: the arrays above hold replica 0 of every group; copy r >= 1 of group g
+  // is entry g*(R-1) + r-1 of the arrays below (R = replicas)
+  float* theta_extra[FLS_MAX_FUSED_EXTRA];
+  float* m_extra[FLS_MAX_FUSED_EXTRA];
+  float* v_extra[FLS_MAX_FUSED_EXTRA];
+  uint16_t* pbf16_extra[FLS_MAX_FUSED_EXTRA];
+  uint32_t replicas;                       // 1: no extra copies
   const float* coefs;                      // device, G clip coefficients written by the reduce kernels
   SegIndex idx;
   uint32_t G;

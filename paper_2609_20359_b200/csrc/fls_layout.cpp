@@ -9,7 +9,8 @@
 
 namespace fls {
 
-std::string build_layout(const std::vector<uint64_t>& unit_numel, uint32_t S, uint32_t Q, uint32_t scratch_slots, Layout* out) {
+std::string build_layout(const std::vector<uint64_t>& unit_numel, uint32_t S, uint32_t Q, uint32_t scratch_slots,
+                         uint32_t ring_replicas, Layout* out) {
   if (unit_numel.empty()) return "empty unit table";
   if (S == 0 || Q == 0) return "shard_dim and align_elems must be >= 1";
   Layout& L = *out;
@@ -36,14 +37,17 @@ std::string build_layout(const std::vector<uint64_t>& unit_numel, uint32_t S, ui
   L.shard_numel = soff;
 
   // Segments in shard-address order: for each rank, for each unit.  Neighbours that are adjacent in
-  // both orders are merged (a single unit collapses to one segment covering the whole buffer).
+  // both orders are merged (a single unit collapses to one segment covering the whole buffer), except for
+  // ring-order plans, whose kernels need to know the rank and the position inside the rank's slice.
   for (uint32_t s = 0; s < S; ++s) {
     for (size_t u = 0; u < n_units; ++u) {
       Segment g{};
       g.j0 = L.unit_offset[u] + uint64_t(s) * L.unit_shard_numel[u];
       g.a0 = uint64_t(s) * L.shard_numel + L.unit_shard_offset[u];
       g.len = L.unit_shard_numel[u];
-      if (!L.segments.empty()) {
+      g.shard = s;
+      g.sub_len = ring_replicas ? (g.len + ring_replicas - 1) / ring_replicas : g.len;
+      if (!L.segments.empty() && !ring_replicas) {
         Segment& p = L.segments.back();
         if (p.j0 + p.len == g.j0 && p.a0 + p.len == g.a0) {
           p.len += g.len;
@@ -69,7 +73,12 @@ std::string build_layout(const std::vector<uint64_t>& unit_numel, uint32_t S, ui
   const uint64_t seg_bytes = L.segments.size() * sizeof(Segment);
   if (L.n_tiles >= (1ull << 32)) return "plan too large";
   L.ws_partials_offset = (kWsSegments + seg_bytes + 255) / 256 * 256;
-  L.ws_scratch_offset = (L.ws_partials_offset + 8 * L.n_tiles + 255) / 256 * 256;   // at most one partial per tile
+  // norm tree: at most one partial per tile, then one sum and one arrival counter per chunk of kNormChunkCtas partials
+  const uint64_t n_chunks = (L.n_tiles + kNormChunkCtas - 1) / kNormChunkCtas;
+  L.ws_chunk_partials_offset = (L.ws_partials_offset + 8 * L.n_tiles + 255) / 256 * 256;
+  L.ws_chunk_count_offset = (L.ws_chunk_partials_offset + 8 * n_chunks + 255) / 256 * 256;
+  L.ws_chunk_count_bytes = 4 * n_chunks;
+  L.ws_scratch_offset = (L.ws_chunk_count_offset + L.ws_chunk_count_bytes + 255) / 256 * 256;
   L.scratch_slots = scratch_slots ? scratch_slots : 1;
   L.scratch_stride = (4ull * L.n_padded + 255) / 256 * 256;
   L.workspace_bytes = L.ws_scratch_offset + L.scratch_stride * L.scratch_slots;

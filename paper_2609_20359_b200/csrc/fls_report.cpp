@@ -45,7 +45,7 @@ fls_cost5 eval(const Layout& lay, double elem_bytes, double S, double R, double 
 
 }  // namespace
 
-void comm_report(const Layout& lay, const fls_plan_desc& d, const double* bw, fls_comm_costs* out) {
+void comm_report(const Layout& lay, const fls_plan_desc& d, int route, const double* bw, fls_comm_costs* out) {
   const double e = d.grad_dtype == FLS_GRAD_F32 ? 4.0 : 2.0;
   const double S = d.shard_dim, R = d.replicate_dim, F = d.groups, A = d.sync_period;
   out->paper_bytes = eval(lay, e, S, R, F, A, 1, 1, 1, false);
@@ -57,15 +57,16 @@ void comm_report(const Layout& lay, const fls_plan_desc& d, const double* bw, fl
     out->seconds = fls_cost5{nan, nan, nan, nan, nan};
   }
   const double K = S * R;
-  // store-and-reread moves K*e_g + 34 bytes per element; with K*e_g < 8 the library reads the gradients twice
-  // instead and moves 2*K*e_g + 26
-  // ... and without clipping one pass does everything: K*e_g + 26
-  const bool f32_sums = d.reduce_wire == FLS_WIRE_F32;
-  const double per_elem = (f32_sums && !(d.max_grad_norm > 0.0)) ? K * e + 26.0
-                          : (f32_sums && K * e < 8.0)            ? 2.0 * K * e + 26.0
-                                                                 : K * e + 34.0;
+  // HBM bytes per element of one group's step.  Store and reread: K*e_g read + 4 written by the reduction, then per
+  // state copy 16 read (mean gradient, theta, m, v) + 14 written (theta, m, v, bf16).  Recompute: the gradients are
+  // read twice and nothing is stored.  Single pass: one kernel, the gradients read once.
+  const double copies = d.state_copies == FLS_STATE_PER_REPLICA ? R : 1.0;
+  const double per_elem = route == 2 ? K * e + 26.0 : route == 1 ? 2.0 * K * e + 26.0 : K * e + 4.0 + 30.0 * copies;
   out->hbm_bytes_sync_step = F * double(lay.n_padded) * per_elem;
-  out->hbm_bytes_fedavg = F * double(lay.n_padded) * ((d.fedavg_what & FLS_AVG_OPT_STATE) ? 26.0 : 10.0);
+  // FedAvg reads one copy per group and writes every copy (4 + 2 bytes for the parameters and their bf16 copy,
+  // 4 + 4 for m and v when they are averaged too)
+  const bool opt = (d.fedavg_what & FLS_AVG_OPT_STATE) != 0;
+  out->hbm_bytes_fedavg = F * double(lay.n_padded) * ((opt ? 12.0 : 4.0) + (opt ? 14.0 : 6.0) * copies);
 }
 
 }  // namespace fls

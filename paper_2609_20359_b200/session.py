@@ -20,7 +20,8 @@ class Session:
                  replicate_dim: int = 1, sync_period: int = 1, grad_dtype: str = "bf16", align_elems: int = 8,
                  opt_state: bool = False, lr: float = 3e-4, beta1: float = 0.9, beta2: float = 0.95, eps: float = 1e-8,
                  weight_decay: float = 0.1, max_grad_norm: float = 1.0, device: str = "cuda:0", guard_bytes: int = 0,
-                 alloc_grads: bool = True, fused: bool = False, wire_bf16: bool = False):
+                 alloc_grads: bool = True, fused: bool = False, wire_bf16: bool = False, ring: bool = False,
+                 state_per_replica: bool = False, speculative: bool = False):
         if not torch.cuda.is_available():
             raise RuntimeError("libfls needs a CUDA device; there is no CPU path")
         self.device = torch.device(device)
@@ -34,16 +35,25 @@ class Session:
             n_params, unit_numel, groups, shard_dim, replicate_dim, sync_period,
             fls.FLS_GRAD_F32 if grad_dtype == "f32" else fls.FLS_GRAD_BF16, align_elems,
             fls.FLS_AVG_PARAMS | (fls.FLS_AVG_OPT_STATE if opt_state else 0) | (fls.FLS_AVG_FUSED if fused else 0),
-            lr, beta1, beta2, eps, weight_decay, max_grad_norm, fls.FLS_WIRE_BF16 if wire_bf16 else fls.FLS_WIRE_F32)
+            lr, beta1, beta2, eps, weight_decay, max_grad_norm, fls.FLS_WIRE_BF16 if wire_bf16 else fls.FLS_WIRE_F32,
+            fls.FLS_ORDER_RING if ring else fls.FLS_ORDER_ASCENDING,
+            fls.FLS_STATE_PER_REPLICA if state_per_replica else fls.FLS_STATE_PER_GROUP)
         self.layout = fls.fls_plan_query(self.plan)
         N = self.layout["n_padded"]
         self.n_padded, self.n_params = N, n_params
+        # state copies: one per group, or one per replica (index g*R_rep + rho)
+        self.n_copies = self.layout["n_state_copies"]
         self.grads = [[self._alloc(N, self.grad_torch_dtype) for _ in range(self.K)] for _ in range(groups)] if alloc_grads else None
-        self.master = [self._alloc(N, torch.float32) for _ in range(groups)]
-        self.m = [self._alloc(N, torch.float32) for _ in range(groups)]
-        self.v = [self._alloc(N, torch.float32) for _ in range(groups)]
-        self.param_bf16 = [self._alloc(N, torch.bfloat16) for _ in range(groups)]
+        self._state = {"master": [self._alloc(N, torch.float32) for _ in range(self.n_copies)],
+                       "m": [self._alloc(N, torch.float32) for _ in range(self.n_copies)],
+                       "v": [self._alloc(N, torch.float32) for _ in range(self.n_copies)]}
+        self.param_bf16 = [self._alloc(N, torch.bfloat16) for _ in range(self.n_copies)]
         self.workspace = self._alloc(self.layout["workspace_bytes"], torch.uint8, zero=False)
+        self.speculative = speculative
+        self._shadow = None
+        if speculative:
+            # the second buffer set that speculative steps write to; which set is current changes with every step
+            self._shadow = {k: [self._alloc(N, torch.float32) for _ in range(groups)] for k in ("master", "m", "v")}
         if alloc_grads:
             self.bind()
 
@@ -73,7 +83,37 @@ class Session:
         if grads is not None:
             self.grads = grads
         flat = [t for row in self.grads for t in row]
-        fls.fls_plan_bind(self.plan, flat, self.master, self.m, self.v, self.param_bf16, self.workspace)
+        st = self._state
+        fls.fls_plan_bind(self.plan, flat, st["master"], st["m"], st["v"], self.param_bf16, self.workspace)
+        if self._shadow is not None:
+            sh = self._shadow
+            fls.fls_plan_bind_shadow(self.plan, sh["master"], sh["m"], sh["v"])
+            fls.fls_plan_set_speculative(self.plan, True)
+
+    def _current(self, which: str):
+        """The tensors that hold `which` ("master", "m", "v") of every state copy right now."""
+        if self._shadow is None:
+            return self._state[which]
+        by_ptr = {t.data_ptr(): t for t in self._state[which] + self._shadow[which]}
+        i = ("master", "m", "v").index(which)
+        return [by_ptr[fls.fls_get_state(self.plan, c)[i]] for c in range(self.n_copies)]
+
+    @property
+    def master(self):
+        return self._current("master")
+
+    @property
+    def m(self):
+        return self._current("m")
+
+    @property
+    def v(self):
+        return self._current("v")
+
+    def spec_stats(self):
+        """(group-steps whose guess held, group-steps redone) of a speculative plan so far."""
+        t = self._ws_view(fls.fls_get_spec_stats(self.plan), 2, torch.int32).cpu()
+        return int(t[0]), int(t[1])
 
     # ------------------------------------------------------------------ calls
     def step(self, lr: float = math.nan, stream=None) -> bool:

@@ -65,7 +65,7 @@ class Case:
 
     def __init__(self, units, G, S, R_rep=1, H=1, Q=8, grad_dtype="bf16", opt_state=False, seed=1234,
                  grad_sigma=1e-3, master_sigma=0.02, per_buffer_scale=False, hp: orc.Hyper = None, guard=4096,
-                 same_grads_all_groups=False, fused=False):
+                 same_grads_all_groups=False, fused=False, state_per_replica=False, speculative=False):
         from paper_2609_20359_b200.session import Session
         self.units, self.G, self.S, self.R_rep, self.H, self.Q = list(units), G, S, R_rep, H, Q
         self.K = S * R_rep
@@ -77,14 +77,20 @@ class Case:
         self.L = orc.plan(units, S, Q)
         th0 = sy.normal_fill_(torch.empty(self.P), sy.stream_key(seed, sy.KIND_MASTER), master_sigma).numpy()
         z = np.zeros(self.P, np.float32)
-        self.states = [orc.GroupState(th0.copy(), z.copy(), z.copy(), orc.f32_to_bf16_bits(th0)) for _ in range(G)]
+        # state copies per group: one, or one per replica (FL+HSDP as it runs); states[g] is the first copy of group g
+        self.R_state = R_rep if state_per_replica else 1
+        self.copies = [[orc.GroupState(th0.copy(), z.copy(), z.copy(), orc.f32_to_bf16_bits(th0)) for _ in range(self.R_state)]
+                       for _ in range(G)]
+        self.states = [c[0] for c in self.copies]
+        self.ring = orc.ring_positions(self.L, R_rep) if self.hp.ring else None
         self.sess = Session(self.P, units, G, S, R_rep, H, grad_dtype, Q, opt_state, self.hp.lr, self.hp.beta1,
                             self.hp.beta2, self.hp.eps, self.hp.weight_decay, self.hp.max_grad_norm, guard_bytes=guard, fused=fused,
-                            wire_bf16=self.hp.wire_bf16)
+                            wire_bf16=self.hp.wire_bf16, ring=self.hp.ring, state_per_replica=state_per_replica, speculative=speculative)
         self.fused = fused
         lay = self.sess.layout
         assert lay["n_padded"] == self.L.n_padded and lay["shard_numel"] == self.L.shard_numel
-        for g in range(G):
+        assert lay["n_state_copies"] == G * self.R_state
+        for g in range(G * self.R_state):
             self.sess.master[g].copy_(torch.from_numpy(orc.pack_sharded(self.L, th0)))
             self.sess.param_bf16[g].copy_(torch.from_numpy(orc.pack_unsharded(self.L, th0)).to(torch.bfloat16))
         self.t = 0
@@ -123,21 +129,30 @@ class Case:
         grads = self.load_grads(self.t, override)
         row = []
         for g in range(self.G):
-            nrm, c, _ = orc.sync_step_group(self.states[g], grads[g], self.S, self.R_rep, self.t, self.hp, lr)
+            if self.R_state > 1:
+                nrm, c, _ = orc.sync_step_replicated(self.copies[g], grads[g], self.S, self.R_rep, self.t, self.hp, lr, self.ring)
+            else:
+                nrm, c, _ = orc.sync_step_group(self.states[g], grads[g], self.S, self.R_rep, self.t, self.hp, lr, self.ring)
             row.append((nrm, c))
         self.norms.append(row)
         due = self.t % self.H == 0
         if due and fedavg and self.fused:
             # the single call that does the step and the aggregation
-            orc.fedavg(self.states, counts, self.opt_state)
+            self.oracle_fedavg(counts)
             self.sess.step_fedavg(counts, float("nan") if lr is None else lr)
         else:
             assert self.sess.step(float("nan") if lr is None else lr) == due
             if due and fedavg:
-                orc.fedavg(self.states, counts, self.opt_state)
+                self.oracle_fedavg(counts)
                 self.sess.fedavg(counts)
         torch.cuda.synchronize()
         return row
+
+    def oracle_fedavg(self, counts):
+        if self.R_state > 1:
+            orc.fedavg_replicated(self.copies, counts, self.opt_state)
+        else:
+            orc.fedavg(self.states, counts, self.opt_state)
 
     def compare(self, check_norms=True):
         torch.cuda.synchronize()
@@ -148,14 +163,15 @@ class Case:
             for g, (nrm, c) in enumerate(self.norms[-1]):
                 assert abs(got_n[g] - nrm) <= 1e-6 * max(nrm, 1e-30), (g, got_n[g], nrm)
                 assert abs(got_c[g] - c) <= 1e-6 * c, (g, got_c[g], c)
-        for g, st in enumerate(self.states):
-            assert_state_close(self.sess.master[g].cpu().numpy(), orc.pack_sharded(self.L, st.theta), f"master[{g}]")
-            assert_state_close(self.sess.m[g].cpu().numpy(), orc.pack_sharded(self.L, st.m), f"m[{g}]", REL_M, ABS_M)
-            assert_state_close(self.sess.v[g].cpu().numpy(), orc.pack_sharded(self.L, st.v), f"v[{g}]", REL_V, ABS_V)
+        master, m, v = self.sess.master, self.sess.m, self.sess.v
+        for g, st in enumerate(c for grp in self.copies for c in grp):       # copy index g*R_state + rho
+            assert_state_close(master[g].cpu().numpy(), orc.pack_sharded(self.L, st.theta), f"master[{g}]")
+            assert_state_close(m[g].cpu().numpy(), orc.pack_sharded(self.L, st.m), f"m[{g}]", REL_M, ABS_M)
+            assert_state_close(v[g].cpu().numpy(), orc.pack_sharded(self.L, st.v), f"v[{g}]", REL_V, ABS_V)
             assert_bf16_close(bf16_bits(self.sess.param_bf16[g]), orc.pack_unsharded(self.L, st.param_bf16), f"param_bf16[{g}]")
             # and the copy is exactly the nearest-even rounding of the GPU's own fp32 master
-            own = orc.unpack_sharded(self.L, bf16_bits(self.sess.master[g].to(torch.bfloat16)))
-            assert np.array_equal(orc.unpack_unsharded(self.L, bf16_bits(self.sess.param_bf16[g])), own), f"bf16 copy of group {g} is not RNE(master)"
+            own = orc.unpack_sharded(self.L, bf16_bits(master[g].to(torch.bfloat16)))
+            assert np.array_equal(orc.unpack_unsharded(self.L, bf16_bits(self.sess.param_bf16[g])), own), f"bf16 copy {g} is not RNE(master)"
 
     def close(self):
         self.sess.close()

@@ -209,6 +209,58 @@ def test_bf16_wire_orders_differ_on_the_gpu_too(fls):
     assert 0.02 < (res[(True, 8)] != res[(True, 4)]).float().mean().item() < 0.9
 
 
+@pytest.mark.parametrize("units,G,S,R_rep,Q,dtype,wire", [
+    ([40000, 30011], 2, 8, 1, 8, "bf16", True),         # reduce-scatter ring only
+    ([40000, 30011], 2, 4, 2, 8, "bf16", True),         # ring at both levels, sub-chunks of M/2
+    ([70001, 33], 1, 3, 2, 1, "bf16", True),            # unaligned shards and sub-chunks: element-wise path
+    ([17], 2, 2, 2, 1, "bf16", True),                   # the brute-force size
+    ([40000, 30011], 2, 4, 3, 8, "bf16", True),         # K = 12, sub-chunk length not a multiple of 8
+    ([40000, 30011], 2, 4, 2, 8, "bf16", False),        # ring order with fp32 partial sums
+    ([40000, 30011], 1, 2, 2, 8, "f32", False),         # fp32 gradients
+])
+def test_ring_order_reduction(fls, units, G, S, R_rep, Q, dtype, wire):
+    """reduce_order = FLS_ORDER_RING: every rank's slice is summed starting on the next rank, every all-reduce
+    sub-chunk starting on the next replica.  With bf16 partial sums the reduced gradient is bit-identical to the
+    oracle's; with fp32 partial sums it equals the exactly rounded mean up to the rounding of the fp32 adds."""
+    hp = orc.Hyper(max_grad_norm=0.05, wire_bf16=wire, ring=True)
+    c = Case(units, G, S, R_rep, H=2, Q=Q, grad_dtype=dtype, hp=hp, per_buffer_scale=True)
+    for t in range(1, 3):
+        grads = c.load_grads(t)
+        want = orc.pack_sharded(c.L, orc.reduce_mean(grads[G - 1], S, R_rep, wire_bf16=wire, ring=c.ring))
+        c.step()
+        got = c.sess.reduced_grad().cpu().numpy()
+        if wire:
+            assert np.array_equal(got, want)
+        else:
+            bound = orc.pack_sharded(c.L, 2.0 ** -24 * np.sum(np.abs(grads[G - 1]), axis=0))
+            assert np.all(np.abs(got.astype(np.float64) - want) <= bound)
+        c.compare()
+    assert c.sess.status() == 0
+    c.close()
+
+
+def test_ring_start_changes_bf16_sums_and_not_fp32_sums(fls):
+    """Same 8 buffers, ascending order against ring order, flat (8 x 1) and two-level (4 x 2): with bf16 partial
+    sums a measurable share of the elements differs (all but those owned by the last rank / last sub-chunk, whose
+    ring order is the ascending one); with fp32 partial sums of bf16 inputs the two orders agree."""
+    res = {}
+    for wire in (False, True):
+        for S, R_rep in ((8, 1), (4, 2)):
+            for ring in (False, True):
+                c = Case([65536], 1, S, R_rep, H=10, Q=8, hp=orc.Hyper(max_grad_norm=10.0, wire_bf16=wire, ring=ring))
+                c.load_grads(1)
+                c.sess.step()
+                torch.cuda.synchronize()
+                res[(wire, S, ring)] = c.sess.reduced_grad().clone()
+                c.close()
+    for S in (8, 4):
+        assert (res[(False, S, False)] != res[(False, S, True)]).float().mean().item() < 1e-3
+        assert 0.02 < (res[(True, S, False)] != res[(True, S, True)]).float().mean().item() < 0.9
+    # the last rank's slice of the flat plan: ring order = ascending order, bit for bit
+    M = 65536 // 8
+    assert torch.equal(res[(True, 8, False)][7 * M:], res[(True, 8, True)][7 * M:])
+
+
 def test_two_level_order_differs_from_flat_where_fp32_rounds(fls):
     """fp32 gradients spanning many binades: the shard-then-replicate order and the flat order round
     differently; each matches the oracle run in the same order (to fp32 rounding of the sum)."""
@@ -299,6 +351,120 @@ def test_fused_step_fedavg_matches_oracle_and_unfused(fls, units, G, S, R_rep, Q
         outs.append([x.clone() for x in c.sess.master + c.sess.m + c.sess.v + c.sess.param_bf16])
         c.close()
     assert all(torch.equal(x, y) for x, y in zip(*outs))
+
+
+@pytest.mark.parametrize("units,G,S,R_rep,Q,dtype,opt_state,fused", [
+    ([50000, 1234, 4096], 2, 2, 2, 8, "bf16", False, False),
+    ([50000, 1234, 4096], 2, 2, 2, 8, "bf16", False, True),
+    ([50000, 1234, 4096], 3, 4, 3, 8, "bf16", True, True),
+    ([70001], 2, 2, 2, 1, "f32", True, False),           # unaligned tail
+    ([70001], 2, 1, 2, 1, "bf16", False, True),          # K = 2: the recompute route is not taken with replica copies
+    ([30000, 517], 16, 2, 3, 8, "bf16", False, True),    # 32 extra copies: the most the fused kernel serves
+    ([30000, 517], 16, 2, 4, 8, "bf16", True, True),     # 48 extra copies: the fused call falls back to step + FedAvg
+    ([17], 2, 2, 2, 1, "bf16", True, True),
+])
+def test_state_copy_per_replica(fls, units, G, S, R_rep, Q, dtype, opt_state, fused):
+    """FLS_STATE_PER_REPLICA: G*R_rep state copies.  Every replica of a group applies the group's mean gradient to
+    its own copy; FedAvg reads one replica per group and its result is broadcast to all copies.  Against the
+    oracle, copy by copy; all copies of a group stay bit-identical; after an aggregation all copies of all groups
+    hold the same parameters."""
+    counts = [sy.sample_count(23, g) for g in range(G)]
+    c = Case(units, G, S, R_rep, H=2, Q=Q, grad_dtype=dtype, opt_state=opt_state, hp=orc.Hyper(max_grad_norm=0.05), fused=fused,
+             state_per_replica=True)
+    assert len(c.sess.master) == G * R_rep
+    for t in range(1, 5):
+        c.step(counts)
+        c.compare()
+        for g in range(G):
+            for r in range(1, R_rep):
+                a, b = g * R_rep, g * R_rep + r
+                assert torch.equal(c.sess.master[a], c.sess.master[b]) and torch.equal(c.sess.m[a], c.sess.m[b])
+                assert torch.equal(c.sess.v[a], c.sess.v[b]) and torch.equal(c.sess.param_bf16[a], c.sess.param_bf16[b])
+        if t % 2 == 0:
+            assert all(torch.equal(c.sess.master[0], x) for x in c.sess.master)
+            assert all(torch.equal(c.sess.param_bf16[0], x) for x in c.sess.param_bf16)
+            assert all(torch.equal(c.sess.m[0], x) for x in c.sess.m) == (opt_state or G == 1)
+    rep = fls.fls_comm_report(c.sess.plan)
+    N, K, eg = c.L.n_padded, S * R_rep, 4 if dtype == "f32" else 2
+    assert rep["hbm_bytes_sync_step"] == G * N * (K * eg + 4 + 30 * R_rep)
+    assert rep["hbm_bytes_fedavg"] == G * N * ((12 + 14 * R_rep) if opt_state else (4 + 6 * R_rep))
+    c.close()
+
+
+def test_state_copy_per_replica_equals_one_copy_per_group(fls):
+    """The replica copies change where the numbers live, not the numbers: copy 0 of every group is bit-identical to
+    the state of the same plan with one copy per group."""
+    outs = []
+    for per_replica in (False, True):
+        c = Case([40000, 30011], 2, 4, 2, H=2, Q=8, opt_state=True, hp=orc.Hyper(max_grad_norm=0.05), fused=True,
+                 state_per_replica=per_replica)
+        for _ in range(4):
+            c.step([5, 2])
+        R = 2 if per_replica else 1
+        outs.append([x.clone() for lst in (c.sess.master, c.sess.m, c.sess.v, c.sess.param_bf16) for x in lst[::R]])
+        c.close()
+    assert all(torch.equal(x, y) for x, y in zip(*outs))
+
+
+@pytest.mark.parametrize("units,G,S,R_rep,Q,dtype,clip", [
+    ([40000, 30011], 2, 8, 1, 8, "bf16", 10.0),          # never clips: every guess holds
+    ([40000, 30011], 2, 4, 2, 8, "bf16", 0.02),          # always clips: every step is redone
+    ([70001], 2, 3, 2, 1, "bf16", 10.0),                 # unaligned shards
+    ([40000, 30011], 2, 2, 1, 8, "f32", 0.02),
+    ([17], 1, 4, 1, 1, "bf16", 10.0),
+])
+def test_speculative_single_pass(fls, units, G, S, R_rep, Q, dtype, clip):
+    """Speculative steps (guess: clip coefficient 1) against the oracle and, bit for bit, against the default
+    two-pass route; the state moves to the other buffer set with every step; kept / redone counts are reported."""
+    outs = []
+    for spec in (True, False):
+        c = Case(units, G, S, R_rep, H=2, Q=Q, grad_dtype=dtype, hp=orc.Hyper(max_grad_norm=clip), per_buffer_scale=True, speculative=spec)
+        seen = set()
+        for t in range(1, 5):
+            c.step([2, 1][:G])
+            c.compare()
+            seen.add(c.sess.master[0].data_ptr())
+        outs.append([x.clone() for x in c.sess.master + c.sess.m + c.sess.v + c.sess.param_bf16] + [c.sess.norms().clone(), c.sess.coefs().clone()])
+        if spec:
+            assert len(seen) == 2                              # the two buffer sets take turns
+            kept, redone = c.sess.spec_stats()
+            assert (kept, redone) == ((4 * G, 0) if clip > 1 else (0, 4 * G))
+            rep = fls.fls_comm_report(c.sess.plan)
+            assert rep["hbm_bytes_sync_step"] == G * c.L.n_padded * (S * R_rep * (4 if dtype == "f32" else 2) + 26)
+        assert c.sess.status() == 0
+        c.close()
+    assert all(torch.equal(x, y) for x, y in zip(*outs[:1] + outs[1:]))
+
+
+def test_speculative_mixed_hits_and_misses_and_errors(fls):
+    """A threshold between the norms of the two groups: group 0's guess holds, group 1 is redone, in the same call."""
+    c = Case([40000, 30011], 2, 4, 1, H=100, Q=8, hp=orc.Hyper(max_grad_norm=1.0), speculative=True)
+    big = lambda t, g, k: c.grad_logical(t, g, k) * (1.0 if g == 0 else 16.0)       # norms about 0.13 and 2.1
+    for _ in range(3):
+        row = c.step(override=big)
+        assert row[0][1] == 1.0 and row[1][1] < 1.0
+        c.compare()
+    assert c.sess.spec_stats() == (3, 3)
+    fls.fls_plan_set_speculative(c.sess.plan, False)        # back to two passes, in place, wherever the state is now
+    c.step(override=big)
+    c.compare()
+    assert c.sess.spec_stats() == (3, 3)
+    c.close()
+    plain = Case([4096], 1, 8, 1, H=2, Q=8)
+    with pytest.raises(fls.FlsError) as e:
+        fls.fls_plan_set_speculative(plain.sess.plan, True)                          # no second buffer set bound
+    assert e.value.code == fls.FLS_ESTATE
+    with pytest.raises(fls.FlsError) as e:
+        fls.fls_plan_bind_shadow(plain.sess.plan, plain.sess.master, plain.sess.m, plain.sess.v)   # overlaps the bound state
+    assert e.value.code == fls.FLS_EPTR
+    plain.close()
+    noclip = Case([4096], 1, 8, 1, H=2, Q=8, hp=orc.Hyper(max_grad_norm=0.0))
+    extra = [torch.zeros(noclip.L.n_padded, device="cuda") for _ in range(3)]
+    fls.fls_plan_bind_shadow(noclip.sess.plan, extra[:1], extra[1:2], extra[2:])
+    with pytest.raises(fls.FlsError) as e:
+        fls.fls_plan_set_speculative(noclip.sess.plan, True)                         # nothing to guess: the plan does not clip
+    assert e.value.code == fls.FLS_ESTATE
+    noclip.close()
 
 
 @pytest.mark.parametrize("G,nesterov,opt_state,units,Q", [(4, True, False, [30000, 517], 8), (3, False, True, [70001], 1), (9, True, False, [999], 8)])

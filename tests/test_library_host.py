@@ -33,8 +33,8 @@ def test_library_exports_every_declared_symbol(fls):
 
 def test_struct_sizes_match_header_layout(fls):
     # natural alignment of the C structs in include/fls.h
-    assert ctypes.sizeof(fls.fls_plan_desc) == 8 + 8 + 8 + 8 * 4 + 6 * 8
-    assert ctypes.sizeof(fls.fls_layout) == 8 + 8 + 4 + 4 + 3 * 8 + 8 + 4 + 4
+    assert ctypes.sizeof(fls.fls_plan_desc) == 8 + 8 + 8 + 10 * 4 + 6 * 8
+    assert ctypes.sizeof(fls.fls_layout) == 8 + 8 + 4 + 4 + 3 * 8 + 8 + 4 + 4 + 4 + 4
     assert ctypes.sizeof(fls.fls_buffers) == 7 * 8
     assert ctypes.sizeof(fls.fls_comm_costs) == 15 * 8 + 16
 
@@ -69,6 +69,26 @@ def test_planner_matches_oracle_on_random_unit_tables(fls):
         fls.fls_plan_destroy(p)
 
 
+def test_ring_order_plans_keep_one_segment_per_rank_and_unit(fls):
+    """Ring-order kernels need the owning rank and the position inside the rank's slice, so the planner does not
+    merge neighbouring runs for them; everything else about the layout is unchanged."""
+    for units, S in (([4096], 4), ([40000, 30011], 4), ([7, 9, 64, 3], 8)):
+        a = fls.fls_plan_create(sum(units), units, groups=2, shard_dim=S, replicate_dim=2, align_elems=8)
+        b = fls.fls_plan_create(sum(units), units, groups=2, shard_dim=S, replicate_dim=2, align_elems=8, reduce_order=fls.FLS_ORDER_RING)
+        la, lb = fls.fls_plan_query(a), fls.fls_plan_query(b)
+        assert lb["n_segments"] == len(units) * S >= la["n_segments"]
+        for k in ("n_padded", "shard_numel", "unit_offset", "unit_shard_numel", "unit_shard_offset", "n_state_copies"):
+            assert la[k] == lb[k]
+        fls.fls_plan_destroy(a); fls.fls_plan_destroy(b)
+    c = fls.fls_plan_create(4096, None, groups=3, shard_dim=2, replicate_dim=4, state_copies=fls.FLS_STATE_PER_REPLICA)
+    assert fls.fls_plan_query(c)["n_state_copies"] == 12
+    for call in (lambda: fls.fls_plan_set_recompute(c, 1), lambda: fls.fls_plan_set_single_pass(c, 1), lambda: fls.fls_plan_set_speculative(c, 1)):
+        with pytest.raises(fls.FlsError) as e:
+            call()
+        assert e.value.code == fls.FLS_ESTATE
+    fls.fls_plan_destroy(c)
+
+
 def test_single_unit_default_table(fls):
     p = fls.fls_plan_create(1000, None, groups=1, shard_dim=4, align_elems=8)
     lay = fls.fls_plan_query(p)
@@ -81,7 +101,8 @@ def test_single_unit_default_table(fls):
                                 dict(eps=0.0), dict(lr=-1.0), dict(lr=float("nan")), dict(grad_dtype=7), dict(fedavg_what=2),
                                 dict(fedavg_what=0), dict(unit_numel=[10, 5]), dict(unit_numel=[16, 0]),
                                 dict(max_grad_norm=float("nan")), dict(weight_decay=-0.5),
-                                dict(reduce_wire=2), dict(reduce_wire=1, grad_dtype=1), dict(fedavg_what=8)])
+                                dict(reduce_wire=2), dict(reduce_wire=1, grad_dtype=1), dict(fedavg_what=8),
+                                dict(reduce_order=2), dict(state_copies=2), dict(groups=33, replicate_dim=2, state_copies=1)])
 def test_plan_create_rejects_bad_arguments(fls, kw):
     args = dict(n_params=16, unit_numel=None, groups=2, shard_dim=2)
     args.update(kw)
