@@ -283,7 +283,7 @@ def measure_workload(args, cfg, fls, Session, rank, world, local, with_e2e, samp
     fused = not args.unfused and G <= fls.FLS_MAX_FUSED_GROUPS
     sess = Session(P, cfg["unit_numel"], G, cfg["shard_dim"], cfg["replicate_dim"], cfg["sync_period"], cfg["grad_dtype"], 8,
                    args.opt_state, cfg["lr"], cfg["beta1"], cfg["beta2"], cfg["eps"], cfg["weight_decay"], cfg["max_grad_norm"],
-                   device=f"cuda:{local}", fused=fused)
+                   device=f"cuda:{local}", fused=fused, speculative=args.speculative)
     H = cfg["sync_period"]
     for kern, val in (("reduce", args.ctas_reduce), ("adamw", args.ctas_adamw), ("fedavg", args.ctas_fedavg)):
         if val:
@@ -363,6 +363,10 @@ def measure_workload(args, cfg, fls, Session, rank, world, local, with_e2e, samp
     ms_prof, _ = timed(args.steps, True, sampler)
     kms, kn = fls.fls_get_kernel_ms(sess.plan)
     fls.fls_set_profiling(sess.plan, False)
+    spec = None
+    if args.speculative:
+        kept, redone = sess.spec_stats()          # all group-steps so far: warm-up, timed and profiled passes
+        spec = {"group_steps_kept": kept, "group_steps_redone": redone, "hit_rate": kept / max(1, kept + redone)}
 
     # end to end: gradients start in pinned host memory, norms come back to the host, every step
     e2e = None
@@ -410,6 +414,11 @@ def measure_workload(args, cfg, fls, Session, rank, world, local, with_e2e, samp
             # small K: nothing is stored by the norm pass and AdamW reads the gradients again
             per_launch.update(reduce=N * kbytes, adamw=N * (kbytes + 26))
             traffic_key.update(reduce=("norm_only", kbytes), adamw=("reduce_adamw", kbytes))
+        if spec is not None:
+            # two launches per group-step, both timed under "adamw": the guessing kernel always moves K*e_g + 26 B per
+            # element, the follow-up kernel nothing when the guess held and the same again when it redoes the step
+            per_launch.update(adamw=N * (kbytes + 26) * (1 + 1 - spec["hit_rate"]) / 2)
+            traffic_key.update(adamw=("step_noclip", kbytes))
         kernels = {}
         for i, name in enumerate(("reduce", "adamw", "fedavg", "adamw_fedavg")):
             if kn[i]:
@@ -424,6 +433,8 @@ def measure_workload(args, cfg, fls, Session, rank, world, local, with_e2e, samp
         # bytes the timed steps had to move: every sync step, plus the FedAvg calls that fell inside the region
         # (the fused aggregation moves no bytes of its own: an aggregation step costs what a plain step costs)
         step_bytes = rep["hbm_bytes_sync_step"] + (0 if fused else rep["hbm_bytes_fedavg"] * fedavg_calls / args.steps)
+        if spec is not None:
+            step_bytes += rep["hbm_bytes_sync_step"] * (1 - spec["hit_rate"])       # a redone group-step moves its bytes twice
         ms_step = ms_total / args.steps
         out = {
             "value": world * G * P * args.steps / (ms_total / 1e3), "ms_per_step": ms_step,
@@ -440,6 +451,8 @@ def measure_workload(args, cfg, fls, Session, rank, world, local, with_e2e, samp
             "kernels": kernels, "ms_per_step_profiled": ms_prof / args.steps,
             "gpu_launches": launches, "samples_in_timed_region": in_region, "e2e": e2e,
         }
+        if spec is not None:
+            out["config"]["speculative_single_pass"] = spec
     sess.close()
     del sess, flush_buf
     torch.cuda.empty_cache()
@@ -634,6 +647,7 @@ def main():
     ap.add_argument("--descending-adamw", action="store_true")
     ap.add_argument("--ascending-adamw", action="store_true")
     ap.add_argument("--no-overlap", action="store_true", help="plain launches instead of programmatic dependent launch")
+    ap.add_argument("--speculative", action="store_true", help="speculative single pass (guess: clip coefficient 1) with a second set of state buffers")
     ap.add_argument("--l2-keep-mb", type=float, default=None, help="MiB at the end of the reduced gradient stored with L2 evict-last (library default: 64)")
     # slices of a workload, for profiler captures that must stay small (same kernels, fewer bytes)
     ap.add_argument("--n-params", type=int, default=0, help="override P (single flat unit)")
@@ -660,7 +674,7 @@ def main():
         return
     cfg = sy.config_by_name(args.config)
     sliced = any([args.n_params, args.groups, args.sync_period, args.shard_dim, args.replicate_dim, args.clip is not None, args.grad_dtype])
-    if sliced or args.config != DEFAULT_CONFIG:
+    if sliced or args.config != DEFAULT_CONFIG or args.speculative:
         args.others = False
     if args.n_params and args.keep_units:
         # same unit table, every unit scaled by n_params / P and rounded to a multiple of 64 elements

@@ -411,17 +411,20 @@ __device__ __forceinline__ void finish_norm(const ReduceArgs& a, float sq, unsig
   double c = 0.0;
   for (unsigned i = lane; i < chunk_size; i += 32) c += __ldcg(a.partials + size_t(chunk) * kNormChunk + i);
   c = warp_sum(c);
-  if (lane == 0) {
-    a.chunk_partials[chunk] = c;
-    a.chunk_count[chunk] = 0u;           // ready for the next launch (stream order)
+  if (lane == 0) a.chunk_count[chunk] = 0u;   // ready for the next launch (stream order)
+  double total = c;
+  if (n_chunks > 1) {                    // (a grid of one chunk is complete here: its sum is the total)
+    if (lane == 0) {
+      a.chunk_partials[chunk] = c;
+      __threadfence();
+      t = atomicAdd(a.ticket, 1u);
+    }
+    if (__shfl_sync(0xFFFFFFFFu, t, 0) != n_chunks - 1) return;
     __threadfence();
-    t = atomicAdd(a.ticket, 1u);
+    total = 0.0;
+    for (unsigned i = lane; i < n_chunks; i += 32) total += __ldcg(a.chunk_partials + i);
+    total = warp_sum(total);
   }
-  if (__shfl_sync(0xFFFFFFFFu, t, 0) != n_chunks - 1) return;
-  __threadfence();
-  double total = 0.0;
-  for (unsigned i = lane; i < n_chunks; i += 32) total += __ldcg(a.chunk_partials + i);
-  total = warp_sum(total);
   if (lane == 0) {
     const double nrm = sqrt(total);
     double c1 = 1.0;

@@ -677,22 +677,30 @@ def _random_cases(n, seed=20260920):
         R_rep = int(rng.choice([1, 1, 2, 3]))
         wire = bool(rng.integers(0, 4) == 0)
         dtype = "bf16" if wire or rng.integers(0, 3) else "f32"
+        ring = bool(rng.integers(0, 4) == 0)
+        per_replica = bool(R_rep > 1 and rng.integers(0, 3) == 0)
+        clip = float(rng.choice([0.0, 0.02, 10.0]))
+        spec = bool(clip > 0 and not (wire or ring or per_replica) and rng.integers(0, 2) == 0)
         out.append(dict(units=units, G=int(rng.choice([1, 2, 3, 4, 8])), S=S, R_rep=R_rep, Q=int(rng.choice([1, 4, 8, 16])),
-                        dtype=dtype, opt_state=bool(rng.integers(0, 2)), fused=bool(rng.integers(0, 2)), wire=wire,
-                        H=int(rng.choice([1, 2, 3])), clip=float(rng.choice([0.0, 0.02, 10.0])),
-                        ctas=int(rng.choice([0, 0, 1, 5])), desc=int(rng.integers(0, 2)), overlap=bool(rng.integers(0, 2)), idx=i))
+                        dtype=dtype, opt_state=bool(rng.integers(0, 2)), fused=bool(rng.integers(0, 2)), wire=wire, ring=ring,
+                        per_replica=per_replica, spec=spec, H=int(rng.choice([1, 2, 3])), clip=clip,
+                        ctas=int(rng.choice([0, 0, 1, 5])), desc=int(rng.integers(0, 2)), overlap=bool(rng.integers(0, 2)),
+                        keep_mb=float(rng.choice([0.0, 0.05, 64.0])), idx=i))
     return out
 
 
-@pytest.mark.parametrize("p", _random_cases(40), ids=lambda p: f"case{p['idx']}")
+@pytest.mark.parametrize("p", _random_cases(60), ids=lambda p: f"case{p['idx']}")
 def test_random_combinations(fls, p):
-    """Random unit tables, mesh shapes, alignment quanta, dtypes, FedAvg options and launch shapes, 3 steps each."""
-    hp = orc.Hyper(max_grad_norm=p["clip"], wire_bf16=p["wire"])
+    """Random unit tables, mesh shapes, alignment quanta, dtypes, reduction wire and order, state copies per group or per
+    replica, speculative steps, FedAvg options and launch shapes, 3 steps each."""
+    hp = orc.Hyper(max_grad_norm=p["clip"], wire_bf16=p["wire"], ring=p["ring"])
     c = Case(p["units"], p["G"], p["S"], p["R_rep"], H=p["H"], Q=p["Q"], grad_dtype=p["dtype"], opt_state=p["opt_state"],
-             hp=hp, fused=p["fused"], per_buffer_scale=True, seed=1000 + p["idx"])
+             hp=hp, fused=p["fused"], per_buffer_scale=True, seed=1000 + p["idx"], state_per_replica=p["per_replica"],
+             speculative=p["spec"])
     for kern in (fls.FLS_KERNEL_ADAMW, fls.FLS_KERNEL_FEDAVG, fls.FLS_KERNEL_ADAMW_FEDAVG):
         fls.fls_plan_tune(c.sess.plan, kern, p["ctas"], p["desc"])
     fls.fls_plan_set_overlap(c.sess.plan, p["overlap"])
+    fls.fls_plan_set_l2_keep(c.sess.plan, int(p["keep_mb"] * 2 ** 20))
     counts = [sy.sample_count(p["idx"], g) for g in range(p["G"])]
     for _ in range(3):
         c.step(counts)
