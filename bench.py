@@ -296,6 +296,8 @@ def measure_workload(args, cfg, fls, Session, rank, world, local, with_e2e, samp
         fls.fls_plan_set_overlap(sess.plan, False)
     if args.l2_keep_mb is not None:
         fls.fls_plan_set_l2_keep(sess.plan, int(args.l2_keep_mb * 2 ** 20))
+    if args.batching is not None:
+        fls.fls_plan_set_batching(sess.plan, args.batching)
     fill_session(sess, cfg)
     stream = torch.cuda.current_stream()
 
@@ -361,6 +363,7 @@ def measure_workload(args, cfg, fls, Session, rank, world, local, with_e2e, samp
     # second pass over the same number of steps with events around every kernel: per-kernel durations
     # (the clocks keep being sampled: an NVML reading can take as long as a short timed region)
     ms_prof, _ = timed(args.steps, True, sampler)
+    batched = fls.fls_plan_get_batching(sess.plan)
     kms, kn = fls.fls_get_kernel_ms(sess.plan)
     fls.fls_set_profiling(sess.plan, False)
     spec = None
@@ -419,6 +422,10 @@ def measure_workload(args, cfg, fls, Session, rank, world, local, with_e2e, samp
             # element, the follow-up kernel nothing when the guess held and the same again when it redoes the step
             per_launch.update(adamw=N * (kbytes + 26) * (1 + 1 - spec["hit_rate"]) / 2)
             traffic_key.update(adamw=("step_noclip", kbytes))
+        if batched:
+            # all groups in one grid: a reduce or AdamW launch covers G times the elements
+            per_launch.update(reduce=G * per_launch["reduce"], adamw=G * per_launch["adamw"])
+            units.update(reduce=N * G, adamw=N * G)
         kernels = {}
         for i, name in enumerate(("reduce", "adamw", "fedavg", "adamw_fedavg")):
             if kn[i]:
@@ -440,7 +447,7 @@ def measure_workload(args, cfg, fls, Session, rank, world, local, with_e2e, samp
             "value": world * G * P * args.steps / (ms_total / 1e3), "ms_per_step": ms_step,
             "config": {"workload": cfg["name"], "n_params": P, "groups": G, "shard_dim": cfg["shard_dim"],
                        "replicate_dim": cfg["replicate_dim"], "sync_period": cfg["sync_period"], "grad_dtype": cfg["grad_dtype"],
-                       "fedavg_opt_state": bool(args.opt_state), "fused_aggregation": bool(fused),
+                       "fedavg_opt_state": bool(args.opt_state), "fused_aggregation": bool(fused), "groups_share_a_grid": bool(batched),
                        "fedavg_calls_in_timed_region": fedavg_calls,
                        "l2": "working set exceeds L2, no flush needed" if flush_buf is None else "L2 flushed (512 MB write, untimed) before every timed step",
                        "parallelism": "replicas only" if world > 1 else "1 gpu"},
@@ -648,6 +655,7 @@ def main():
     ap.add_argument("--ascending-adamw", action="store_true")
     ap.add_argument("--no-overlap", action="store_true", help="plain launches instead of programmatic dependent launch")
     ap.add_argument("--speculative", action="store_true", help="speculative single pass (guess: clip coefficient 1) with a second set of state buffers")
+    ap.add_argument("--batching", type=int, default=None, choices=[-1, 0, 1], help="all groups in one grid per kernel: -1 automatic (small plans), 0 never, 1 whenever possible")
     ap.add_argument("--l2-keep-mb", type=float, default=None, help="MiB at the end of the reduced gradient stored with L2 evict-last (library default: 64)")
     # slices of a workload, for profiler captures that must stay small (same kernels, fewer bytes)
     ap.add_argument("--n-params", type=int, default=0, help="override P (single flat unit)")

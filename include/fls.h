@@ -281,6 +281,17 @@ int fls_get_spec_stats(const fls_plan* plan, const uint32_t** dev_counts);
  * plans, where every step moves the state to the other buffer set.  Any output may be NULL. */
 int fls_get_state(const fls_plan* plan, uint32_t copy, float** master, float** m, float** v);
 
+/* Small plans are launch-bound when every group gets its own two kernels.  When the plan allows it (G > 1, G*K <= 64,
+ * K = 4 or 8 in a flat or 1/2/4-wide two-level order, the default two-pass route, one state copy per group, and a
+ * reduced-gradient slot per group in the workspace: FLS_AVG_FUSED plans and plans whose G reduced gradients need at
+ * most 32 MiB) fls_sync_step can run all groups in ONE reduce grid and ONE AdamW grid, with the group in the grid's y
+ * dimension; fls_sync_step_fedavg then uses the one reduce grid as well.  mode -1 (default): automatically, only while
+ * the G reduced gradients fit in 32 MiB (beyond that the per-group sequence is faster: its reduced gradient is still in
+ * L2 when AdamW reads it); 0: never; 1: whenever the plan allows it (FLS_ESTATE otherwise).  Results do not change.
+ * fls_plan_get_batching: whether the next fls_sync_step would run that way. */
+int fls_plan_set_batching(fls_plan* plan, int mode);
+int fls_plan_get_batching(const fls_plan* plan, int* active);
+
 /* How many bytes at the end of the reduced gradient the reduce kernel stores with the "evict last" L2 policy (the
  * AdamW kernel walks the reduced gradient backwards, so it reads that part first and finds it in L2); the rest is
  * stored "evict first" like every other stream.  Default 64 MiB.  Scheduling only: results do not change. */

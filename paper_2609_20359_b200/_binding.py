@@ -29,7 +29,7 @@ EXPORTS = [
     "fls_plan_create", "fls_plan_query", "fls_plan_bind", "fls_sync_step", "fls_sync_step_host", "fls_fedavg",
     "fls_sync_step_fedavg", "fls_fedavg_outer",
     "fls_get_norms", "fls_get_reduced_grad", "fls_get_status", "fls_get_step", "fls_set_step", "fls_comm_report",
-    "fls_plan_bind_shadow", "fls_plan_set_speculative", "fls_get_spec_stats", "fls_get_state", "fls_plan_set_l2_keep",
+    "fls_plan_bind_shadow", "fls_plan_set_speculative", "fls_get_spec_stats", "fls_get_state", "fls_plan_set_l2_keep", "fls_plan_set_batching", "fls_plan_get_batching",
     "fls_plan_tune", "fls_plan_set_recompute", "fls_plan_set_single_pass", "fls_plan_set_overlap", "fls_set_profiling", "fls_get_kernel_ms", "fls_get_launch_count", "fls_plan_destroy",
     "fls_last_error", "fls_reduce_norm_noalloc",
 ]
@@ -103,6 +103,8 @@ def _load() -> C.CDLL:
     lib.fls_get_spec_stats.argtypes = [P, C.POINTER(P)]
     lib.fls_get_state.argtypes = [P, C.c_uint32, C.POINTER(P), C.POINTER(P), C.POINTER(P)]
     lib.fls_plan_set_l2_keep.argtypes = [P, C.c_uint64]
+    lib.fls_plan_set_batching.argtypes = [P, C.c_int]
+    lib.fls_plan_get_batching.argtypes = [P, C.POINTER(C.c_int)]
     lib.fls_plan_set_recompute.argtypes = [P, C.c_int]
     lib.fls_plan_set_single_pass.argtypes = [P, C.c_int]
     lib.fls_plan_set_overlap.argtypes = [P, C.c_int]
@@ -286,6 +288,17 @@ def fls_get_state(plan: int, copy: int):
     a, b, c = C.c_void_p(), C.c_void_p(), C.c_void_p()
     _check(lib.fls_get_state(plan, copy, C.byref(a), C.byref(b), C.byref(c)))
     return a.value, b.value, c.value
+
+
+def fls_plan_set_batching(plan: int, mode: int) -> None:
+    """-1 automatic (small plans), 0 never, 1 whenever the plan allows it: all groups in one grid per kernel."""
+    _check(lib.fls_plan_set_batching(plan, mode))
+
+
+def fls_plan_get_batching(plan: int) -> bool:
+    a = C.c_int(0)
+    _check(lib.fls_plan_get_batching(plan, C.byref(a)))
+    return bool(a.value)
 
 
 def fls_plan_set_l2_keep(plan: int, nbytes: int) -> None:

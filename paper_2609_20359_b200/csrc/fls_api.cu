@@ -47,6 +47,8 @@ struct Range {
 
 }  // namespace
 
+constexpr uint64_t kBatchScratchBytes = 32ull << 20;
+
 struct fls_plan {
   fls_plan_desc desc{};
   std::vector<uint64_t> units;
@@ -68,6 +70,8 @@ struct fls_plan {
   std::vector<float*> master2, m2, v2;   // second buffer set of a speculative plan (the one not current)
   std::vector<Range> ranges;             // everything bound, for overlap checks of later additions
   bool speculative = false;
+  bool fused_plan = false;               // fls_sync_step_fedavg may fuse the aggregation into the optimizer kernel
+  int batch_mode = -1;                   // groups in one grid: -1 automatic (small plans), 0 never, 1 whenever possible
   uint64_t l2_keep_bytes = 64ull << 20;  // tail of the reduced gradient stored with L2 evict-last
   char* ws = nullptr;
 
@@ -98,8 +102,20 @@ struct fls_plan {
   double* d_chunk_partials() const { return reinterpret_cast<double*>(ws + lay.ws_chunk_partials_offset); }
   uint32_t* d_chunk_count() const { return reinterpret_cast<uint32_t*>(ws + lay.ws_chunk_count_offset); }
   uint32_t* d_status() const { return reinterpret_cast<uint32_t*>(ws + kWsStatus); }
-  uint32_t* d_ticket() const { return reinterpret_cast<uint32_t*>(ws + kWsStatus) + 1; }
+  uint32_t* d_ticket() const { return reinterpret_cast<uint32_t*>(ws + kWsTickets); }
   uint32_t* d_spec_counts() const { return reinterpret_cast<uint32_t*>(ws + kWsStatus) + 2; }
+  // One grid for all groups (instead of one launch per group) needs a reduced-gradient slot per group, a level structure
+  // the batched kernels are built for, the default two-pass route and one state copy per group.  Automatic: only when all
+  // the reduced gradients together fit in a quarter of the L2 (32 MiB), i.e. when a launch per group would be launch-bound;
+  // larger plans keep the per-group sequence, whose reduced gradient is still in L2 when AdamW reads it.
+  bool can_batch() const {
+    return desc.groups > 1 && lay.scratch_slots >= desc.groups && uint64_t(desc.groups) * K <= FLS_MAX_GRAD_BUFFERS &&
+           reduce_batchable(K, reduce_sg) && plain_reduce() && !single_pass && !recompute && !speculative;
+  }
+  bool batching() const {
+    if (batch_mode == 0 || !can_batch()) return false;
+    return batch_mode > 0 || uint64_t(desc.groups) * lay.n_padded * 4 <= kBatchScratchBytes;
+  }
   // how fls_sync_step currently gets from the gradients to the new state (for the HBM byte count)
   // the routes that form the mean gradient inside the AdamW kernel exist for fp32 partial sums in ascending order
   // and one state copy per group
@@ -199,10 +215,10 @@ int run_group(fls_plan* p, uint32_t g, double lr, uint64_t t_new, cudaStream_t s
   ra.k_is_pow2 = (p->K & (p->K - 1)) == 0 ? 1u : 0u;
   ra.fold_mask = p->fold_mask;
   ra.end_mask = p->end_mask;
-  ra.partials = p->d_partials();
-  ra.chunk_partials = p->d_chunk_partials();
-  ra.chunk_count = p->d_chunk_count();
-  ra.ticket = p->d_ticket();
+  ra.partials = p->d_partials() + size_t(g) * p->lay.n_tiles;
+  ra.chunk_partials = p->d_chunk_partials() + size_t(g) * p->lay.n_chunks;
+  ra.chunk_count = p->d_chunk_count() + size_t(g) * p->lay.n_chunks;
+  ra.ticket = p->d_ticket() + g;
   ra.norm_out = p->d_norms() + g;
   ra.coef_out = p->d_coefs() + g;
   ra.normsq_out = p->d_normsq() + g;
@@ -284,6 +300,64 @@ int run_group(fls_plan* p, uint32_t g, double lr, uint64_t t_new, cudaStream_t s
     e = timed_launch(p, FLS_KERNEL_ADAMW, st, [&] { return launch_adamw(aa, p->grid_for(FLS_KERNEL_ADAMW), st, overlap); });
     if (e != cudaSuccess) return cuda_fail(e, "adamw kernel launch");
   }
+  return FLS_OK;
+}
+
+// All groups in two launches (one reduce grid, one AdamW grid with the groups in the y dimension) instead of two per
+// group; with_adamw = false stops after the reduction (fused aggregation).  Same arithmetic, same results.
+int run_groups_batched(fls_plan* p, double lr, uint64_t t_new, cudaStream_t st, bool with_adamw) {
+  const fls_plan_desc& d = p->desc;
+  const uint32_t G = d.groups;
+  ReduceArgs ra{};
+  for (uint32_t i = 0; i < G * p->K; ++i) ra.grad[i] = p->grads[i];
+  ra.gbar = p->d_gbar(0);
+  ra.gbar_stride = p->lay.scratch_stride / 4;
+  ra.tree_stride = uint32_t(p->lay.n_chunks);
+  p->last_slot = G - 1;
+  p->gbar_valid = true;
+  ra.idx = p->seg_index();
+  ra.K = p->K;
+  ra.k_float = float(p->K);
+  ra.inv_k = 1.0f / float(p->K);
+  ra.k_is_pow2 = 1u;                       // K is 4 or 8 here
+  ra.fold_mask = p->fold_mask;
+  ra.end_mask = p->end_mask;
+  ra.partials = p->d_partials();
+  ra.chunk_partials = p->d_chunk_partials();
+  ra.chunk_count = p->d_chunk_count();
+  ra.ticket = p->d_ticket();
+  ra.norm_out = p->d_norms();
+  ra.coef_out = p->d_coefs();
+  ra.normsq_out = p->d_normsq();
+  ra.status = p->d_status();
+  ra.max_grad_norm = d.max_grad_norm;
+  ra.S = d.shard_dim;
+  ra.R = d.replicate_dim;
+  const uint64_t keep_tiles = std::min<uint64_t>(p->lay.n_tiles, p->l2_keep_bytes / (uint64_t(kTile) * 4));
+  ra.keep_from_tile = uint32_t(p->lay.n_tiles - keep_tiles);
+  ra.store_gbar = 1;
+  const bool f32 = d.grad_dtype == FLS_GRAD_F32;
+  const bool overlap = p->overlap && !p->profiling;
+  cudaError_t e = timed_launch(p, FLS_KERNEL_REDUCE, st, [&] { return launch_reduce_batch(ra, f32, p->reduce_sg, G, st, false); });
+  if (e != cudaSuccess) return cuda_fail(e, "batched reduce kernel launch");
+  if (!with_adamw) return FLS_OK;
+  const AdamScalars sc = adam_scalars(d, lr, t_new);
+  AdamBatchArgs ab{};
+  for (uint32_t g = 0; g < G; ++g) {
+    ab.theta[g] = p->master[g];
+    ab.m[g] = p->m[g];
+    ab.v[g] = p->v[g];
+    ab.pbf16[g] = p->pbf16[g];
+  }
+  ab.gbar = p->d_gbar(0);
+  ab.gbar_stride = ra.gbar_stride;
+  ab.coef = p->d_coefs();
+  ab.idx = ra.idx;
+  ab.descending = p->descending[FLS_KERNEL_ADAMW];
+  ab.decay = sc.decay; ab.beta1 = sc.beta1; ab.omb1 = sc.omb1; ab.beta2 = sc.beta2; ab.omb2 = sc.omb2;
+  ab.step_size = sc.step_size; ab.inv_sqrt_bc2 = sc.inv_sqrt_bc2; ab.eps = sc.eps;
+  e = timed_launch(p, FLS_KERNEL_ADAMW, st, [&] { return launch_adamw_batch(ab, p->grid_for(FLS_KERNEL_ADAMW), G, st, overlap); });
+  if (e != cudaSuccess) return cuda_fail(e, "batched adamw kernel launch");
   return FLS_OK;
 }
 
@@ -384,7 +458,13 @@ int fls_plan_create(const fls_plan_desc* desc, fls_plan** out) {
   p->n_copies = d.groups * p->R_state;
   const bool fused = (d.fedavg_what & FLS_AVG_FUSED) && d.groups <= FLS_MAX_FUSED_GROUPS &&
                      uint64_t(d.groups) * (p->R_state - 1) <= uint64_t(FLS_MAX_FUSED_EXTRA);
-  const std::string msg = build_layout(units, d.shard_dim, d.align_elems, fused ? d.groups : 1, p->ring ? d.replicate_dim : 0, &p->lay);
+  // one reduced-gradient slot per group for the fused aggregation and for small plans (whose groups share a grid)
+  unsigned __int128 padded_bound = 0;
+  for (uint64_t n : units) padded_bound += n + uint64_t(d.shard_dim) * d.align_elems;
+  const bool small = padded_bound * 4 * d.groups <= kBatchScratchBytes;
+  p->fused_plan = fused;
+  const std::string msg = build_layout(units, d.shard_dim, d.align_elems, (fused || small) ? d.groups : 1, p->ring ? d.replicate_dim : 0,
+                                       d.groups, &p->lay);
   if (!msg.empty()) {
     delete p;
     return fail(FLS_EINVAL, "layout: %s", msg.c_str());
@@ -505,9 +585,14 @@ int fls_sync_step(fls_plan* p, double lr, void* cuda_stream, int* fedavg_due) {
   if (!step_preamble(p, &lr)) return fail(FLS_EINVAL, "fls_sync_step: lr must be finite and >= 0");
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const uint64_t t_new = p->step + 1;
-  for (uint32_t g = 0; g < p->desc.groups; ++g) {
-    const int rc = run_group(p, g, lr, t_new, st, g > 0);
+  if (p->batching()) {
+    const int rc = run_groups_batched(p, lr, t_new, st, true);
     if (rc != FLS_OK) return rc;
+  } else {
+    for (uint32_t g = 0; g < p->desc.groups; ++g) {
+      const int rc = run_group(p, g, lr, t_new, st, g > 0);
+      if (rc != FLS_OK) return rc;
+    }
   }
   p->step = t_new;
   if (fedavg_due) *fedavg_due = (t_new % p->desc.sync_period == 0) ? 1 : 0;
@@ -623,7 +708,7 @@ int fls_sync_step_fedavg(fls_plan* p, double lr, const uint64_t* sample_counts, 
   if (!p) return fail(FLS_EINVAL, "fls_sync_step_fedavg: null plan");
   if (!p->bound) return fail(FLS_ESTATE, "fls_sync_step_fedavg: plan has no buffers bound");
   const uint32_t G = p->desc.groups;
-  if (p->lay.scratch_slots < G) {   // not planned for fusion: the two calls in sequence give the same result
+  if (!p->fused_plan) {             // not planned for fusion: the two calls in sequence give the same result
     const int rc = fls_sync_step(p, lr, cuda_stream, nullptr);
     return rc != FLS_OK ? rc : fls_fedavg(p, sample_counts, cuda_stream);
   }
@@ -633,9 +718,14 @@ int fls_sync_step_fedavg(fls_plan* p, double lr, const uint64_t* sample_counts, 
   if (!(total > 0)) return fail(FLS_EINVAL, "fls_sync_step_fedavg: all sample counts are zero");
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const uint64_t t_new = p->step + 1;
-  for (uint32_t g = 0; g < G; ++g) {
-    const int rc = run_group(p, g, lr, t_new, st, g > 0, g, false);
+  if (p->batching()) {
+    const int rc = run_groups_batched(p, lr, t_new, st, false);
     if (rc != FLS_OK) return rc;
+  } else {
+    for (uint32_t g = 0; g < G; ++g) {
+      const int rc = run_group(p, g, lr, t_new, st, g > 0, g, false);
+      if (rc != FLS_OK) return rc;
+    }
   }
   const AdamScalars sc = adam_scalars(p->desc, lr, t_new);
   FusedArgs fa{};
@@ -793,6 +883,21 @@ int fls_get_state(const fls_plan* p, uint32_t copy, float** master, float** m, f
   if (master) *master = p->master[copy];
   if (m) *m = p->m[copy];
   if (v) *v = p->v[copy];
+  return FLS_OK;
+}
+
+int fls_plan_set_batching(fls_plan* p, int mode) {
+  if (!p) return fail(FLS_EINVAL, "fls_plan_set_batching: null plan");
+  if (mode > 0 && !p->can_batch())
+    return fail(FLS_ESTATE, "fls_plan_set_batching: needs G > 1, G*K <= 64, K = 4 or 8 in a flat or 1/2/4-wide two-level order, the default "
+                            "two-pass route, one state copy per group and a reduced-gradient slot per group (FLS_AVG_FUSED, or a small plan)");
+  p->batch_mode = mode < 0 ? -1 : (mode > 0 ? 1 : 0);
+  return FLS_OK;
+}
+
+int fls_plan_get_batching(const fls_plan* p, int* active) {
+  if (!p || !active) return fail(FLS_EINVAL, "fls_plan_get_batching: null argument");
+  *active = p->batching() ? 1 : 0;
   return FLS_OK;
 }
 

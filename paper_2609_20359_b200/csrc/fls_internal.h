@@ -29,18 +29,20 @@ struct Segment {
 };
 
 // Workspace layout (byte offsets); the head is fixed, the segment table and the scratch follow.
-constexpr uint64_t kWsStatus = 0;        // uint32 status, uint32 ticket counter, uint32[2] speculative commits / redos
+constexpr uint64_t kWsStatus = 0;        // uint32 status, uint32 (unused), uint32[2] speculative commits / redos
 constexpr uint64_t kWsNorms = 256;       // float[64]
 constexpr uint64_t kWsCoefs = 512;       // float[64]
 constexpr uint64_t kWsNormSq = 768;      // double[64]
-constexpr uint64_t kWsSegments = 1280;   // Segment[n_segments], then the norm tree (double[n_tiles] CTA partials, chunk
-                                         // sums, chunk arrival counters), then the reduced-gradient scratch
+constexpr uint64_t kWsTickets = 1280;    // uint32[64]: one ticket counter per group
+constexpr uint64_t kWsSegments = 1536;   // Segment[n_segments], then per group the norm tree (double[n_tiles] CTA partials,
+                                         // chunk sums, chunk arrival counters), then the reduced-gradient scratch
 
 struct Layout {
   std::vector<uint64_t> unit_numel, unit_offset, unit_shard_numel, unit_shard_offset;
   std::vector<Segment> segments;
   uint64_t n_params = 0, n_padded = 0, shard_numel = 0, n_tiles = 0;
   uint64_t ws_partials_offset = 0, ws_chunk_partials_offset = 0, ws_chunk_count_offset = 0, ws_chunk_count_bytes = 0;
+  uint64_t n_chunks = 0;                   // chunks of CTA partials per group; every group has its own tree arrays
   uint64_t ws_scratch_offset = 0, workspace_bytes = 0;
   bool vector_path = true;
   uint32_t scratch_slots = 1;              // reduced-gradient buffers in the workspace, each 4*n_padded bytes (256-byte aligned)
@@ -51,8 +53,9 @@ struct Layout {
 // scratch_slots: how many reduced-gradient buffers the workspace holds (1, or G for the fused aggregation).
 // ring_replicas: 0 for the ascending reduction order; R_rep for the ring order, whose segments stay unmerged and
 // carry the owning rank and the all-reduce sub-chunk length.
+// groups: G (every group gets its own norm-tree arrays, so that the groups' kernels may run in one grid).
 std::string build_layout(const std::vector<uint64_t>& unit_numel, uint32_t S, uint32_t Q, uint32_t scratch_slots,
-                         uint32_t ring_replicas, Layout* out);
+                         uint32_t ring_replicas, uint32_t groups, Layout* out);
 
 // Sets the calling thread's message returned by fls_last_error() (defined beside it).
 void set_last_error(const char* msg);

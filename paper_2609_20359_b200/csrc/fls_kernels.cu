@@ -268,12 +268,13 @@ __device__ __forceinline__ void combine_loaded(const ReduceArgs& a, const Raw<N,
   scale_mean<N>(a, outer, mean);
 }
 
+// gk0: index of the group's first buffer in a.grad (0 except in a batched launch).
 template <int N, bool F32, int KT, int SG>
-__device__ __forceinline__ void reduce_elems(const ReduceArgs& a, uint64_t j, float (&mean)[N], uint32_t sc = 0) {
+__device__ __forceinline__ void reduce_elems(const ReduceArgs& a, uint64_t j, float (&mean)[N], uint32_t sc = 0, uint32_t gk0 = 0) {
   if constexpr (KT > 0 && SG >= 0) {
     Raw<N, F32> raw[KT];
 #pragma unroll
-    for (int b = 0; b < KT; ++b) load_raw(raw[b], a.grad[b], j);
+    for (int b = 0; b < KT; ++b) load_raw(raw[b], a.grad[gk0 + b], j);
     combine_loaded<N, F32, KT, SG>(a, raw, mean);
   } else {
     // run-time K: batches of 8 buffers
@@ -287,11 +288,11 @@ __device__ __forceinline__ void reduce_elems(const ReduceArgs& a, uint64_t j, fl
       if (SG < 0 && a.ring) {
 #pragma unroll
         for (int b = 0; b < 8; ++b)
-          if (k0 + b < K) load_raw(raw[b], a.grad[ring_buffer(a, sc, k0 + b)], j);
+          if (k0 + b < K) load_raw(raw[b], a.grad[gk0 + ring_buffer(a, sc, k0 + b)], j);
       } else {
 #pragma unroll
         for (int b = 0; b < 8; ++b)
-          if (k0 + b < K) load_raw(raw[b], a.grad[k0 + b], j);
+          if (k0 + b < K) load_raw(raw[b], a.grad[gk0 + k0 + b], j);
       }
       if constexpr (SG == 0) {
 #pragma unroll
@@ -355,7 +356,7 @@ __device__ __forceinline__ void reduce_elems(const ReduceArgs& a, uint64_t j, fl
 // pos the position of the slice's first element inside it; otherwise both are ignored
 template <bool F32, bool WIRE>
 __device__ __noinline__ float reduce_slice_scalar(const ReduceArgs& a, uint64_t j, uint64_t addr, uint32_t n, const Segment* seg,
-                                                  uint64_t pos) {
+                                                  uint64_t pos, uint32_t gk0, float* gbar) {
   float sq = 0.f;
   uint32_t shard = 0;
   uint64_t sub_len = 1;
@@ -366,8 +367,8 @@ __device__ __noinline__ float reduce_slice_scalar(const ReduceArgs& a, uint64_t 
   for (uint32_t e = 0; e < n; ++e) {
     float g[1];
     const uint32_t sc = a.ring ? (shard | uint32_t((pos + e) / sub_len) << 16) : 0u;
-    reduce_elems<1, F32, 0, WIRE ? -2 : -1>(a, j + e, g, sc);
-    if (a.store_gbar) a.gbar[addr + e] = g[0];
+    reduce_elems<1, F32, 0, WIRE ? -2 : -1>(a, j + e, g, sc, gk0);
+    if (a.store_gbar) gbar[addr + e] = g[0];
     sq = fmaf(g[0], g[0], sq);
   }
   return sq;
@@ -384,8 +385,9 @@ __device__ __noinline__ float reduce_slice_scalar(const ReduceArgs& a, uint64_t 
 // The caller must have zeroed *arrived (shared) behind a __syncthreads() at the start of the kernel.
 constexpr unsigned kNormChunk = kNormChunkCtas;
 
+// y: the group of a batched launch (0 otherwise); it selects the group's own tree arrays, ticket and output slots.
 template <int THREADS>
-__device__ __forceinline__ void finish_norm(const ReduceArgs& a, float sq, unsigned* arrived) {
+__device__ __forceinline__ void finish_norm(const ReduceArgs& a, float sq, unsigned* arrived, uint32_t y = 0) {
   constexpr int W = THREADS / 32;
   __shared__ double sh[W];
   const double x = warp_sum(double(sq));
@@ -401,28 +403,31 @@ __device__ __forceinline__ void finish_norm(const ReduceArgs& a, float sq, unsig
   const double cta = warp_sum(lane < W ? sh[lane] : 0.0);
   const unsigned chunk = blockIdx.x / kNormChunk, n_chunks = (gridDim.x + kNormChunk - 1) / kNormChunk;
   const unsigned chunk_size = min(kNormChunk, gridDim.x - chunk * kNormChunk);
+  double* const partials = a.partials + size_t(y) * gridDim.x;
+  double* const chunk_partials = a.chunk_partials + size_t(y) * a.tree_stride;
+  uint32_t* const chunk_count = a.chunk_count + size_t(y) * a.tree_stride;
   if (lane == 0) {
-    a.partials[blockIdx.x] = cta;
+    partials[blockIdx.x] = cta;
     __threadfence();
-    t = atomicAdd(a.chunk_count + chunk, 1u);
+    t = atomicAdd(chunk_count + chunk, 1u);
   }
   if (__shfl_sync(0xFFFFFFFFu, t, 0) != chunk_size - 1) return;
   __threadfence();
   double c = 0.0;
-  for (unsigned i = lane; i < chunk_size; i += 32) c += __ldcg(a.partials + size_t(chunk) * kNormChunk + i);
+  for (unsigned i = lane; i < chunk_size; i += 32) c += __ldcg(partials + size_t(chunk) * kNormChunk + i);
   c = warp_sum(c);
-  if (lane == 0) a.chunk_count[chunk] = 0u;   // ready for the next launch (stream order)
+  if (lane == 0) chunk_count[chunk] = 0u;     // ready for the next launch (stream order)
   double total = c;
   if (n_chunks > 1) {                    // (a grid of one chunk is complete here: its sum is the total)
     if (lane == 0) {
-      a.chunk_partials[chunk] = c;
+      chunk_partials[chunk] = c;
       __threadfence();
-      t = atomicAdd(a.ticket, 1u);
+      t = atomicAdd(a.ticket + y, 1u);
     }
     if (__shfl_sync(0xFFFFFFFFu, t, 0) != n_chunks - 1) return;
     __threadfence();
     total = 0.0;
-    for (unsigned i = lane; i < n_chunks; i += 32) total += __ldcg(a.chunk_partials + i);
+    for (unsigned i = lane; i < n_chunks; i += 32) total += __ldcg(chunk_partials + i);
     total = warp_sum(total);
   }
   if (lane == 0) {
@@ -432,12 +437,12 @@ __device__ __forceinline__ void finish_norm(const ReduceArgs& a, float sq, unsig
       c1 = a.max_grad_norm / (nrm + 1e-6);
       if (c1 >= 1.0) c1 = 1.0;          // NaN compares false and stays NaN: non-finite norms propagate
     }
-    *a.normsq_out = total;
-    *a.norm_out = float(nrm);
-    *a.coef_out = float(c1);
+    a.normsq_out[y] = total;
+    a.norm_out[y] = float(nrm);
+    a.coef_out[y] = float(c1);
     if (!isfinite(nrm)) atomicOr(a.status, uint32_t(FLS_STATUS_NONFINITE_NORM));
     if (a.spec_counts) atomicAdd(a.spec_counts + (float(c1) == 1.0f ? 0 : 1), 1u);   // speculative step: kept / redone
-    *a.ticket = 0u;                      // ready for the next launch (stream order)
+    a.ticket[y] = 0u;                    // ready for the next launch (stream order)
   }
 }
 
@@ -456,7 +461,7 @@ __device__ __forceinline__ void begin_norm(unsigned* arrived) {
 // With K = 1 or 2 a thread would have only one or two 16-byte loads in flight, so those shapes take U > 1 tiles
 // per thread (512 x 2 CTAs) and issue the loads of all of them before the first add.
 template <bool F32, int KT, int SG>
-__device__ __forceinline__ float reduce_one_tile(const ReduceArgs& a, uint32_t tile, uint32_t lane) {
+__device__ __forceinline__ float reduce_one_tile(const ReduceArgs& a, uint32_t tile, uint32_t lane, uint32_t gk0, float* gbar) {
   float sq = 0.f;
   const Segment* seg = a.idx.segs + find_segment(a.idx, tile);
   const Slice s = slice_of(seg, tile, lane);
@@ -471,31 +476,35 @@ __device__ __forceinline__ float reduce_one_tile(const ReduceArgs& a, uint32_t t
   }
   if (vec) {
     float g[8];
-    reduce_elems<8, F32, KT, SG>(a, s.j, g, sc);
+    reduce_elems<8, F32, KT, SG>(a, s.j, g, sc, gk0);
     F8 o;
 #pragma unroll
     for (int e = 0; e < 8; ++e) { o.v[e] = g[e]; sq = fmaf(g[e], g[e], sq); }
     if (a.store_gbar) {
       dep_wait();                        // the previous group's AdamW kernel may still be reading the scratch
-      if (tile >= a.keep_from_tile) st8_keep(a.gbar + s.a, o); else st8_stream(a.gbar + s.a, o);
+      if (tile >= a.keep_from_tile) st8_keep(gbar + s.a, o); else st8_stream(gbar + s.a, o);
     }
   } else if (s.n) {
     dep_wait();
-    sq = reduce_slice_scalar<F32, SG == -2>(a, s.j, s.a, s.n, seg, s.e);
+    sq = reduce_slice_scalar<F32, SG == -2>(a, s.j, s.a, s.n, seg, s.e, gk0, gbar);
   }
   return sq;
 }
 
-template <bool F32, int KT, int SG, int THREADS, int MINB, int U>
+// BATCH: the grid's y dimension runs over the groups (see ReduceArgs); otherwise one group per launch.
+template <bool F32, int KT, int SG, int THREADS, int MINB, int U, bool BATCH = false>
 __global__ void __launch_bounds__(THREADS, MINB) fls_reduce_kernel(const __grid_constant__ ReduceArgs a) {
   constexpr uint32_t T = THREADS / kThreads;
   __shared__ unsigned arrived;
   begin_norm(&arrived);
+  const uint32_t y = BATCH ? blockIdx.y : 0u;
+  const uint32_t gk0 = BATCH ? y * uint32_t(KT) : 0u;
+  float* const gbar = BATCH ? a.gbar + size_t(y) * a.gbar_stride : a.gbar;
   const uint32_t lane = threadIdx.x % kThreads;
   const uint32_t first = blockIdx.x * (T * U) + threadIdx.x / kThreads;   // this thread's tiles: first + u*T
   float sq = 0.f;
   if constexpr (U == 1) {
-    if (first < a.idx.n_tiles) sq = reduce_one_tile<F32, KT, SG>(a, first, lane);
+    if (first < a.idx.n_tiles) sq = reduce_one_tile<F32, KT, SG>(a, first, lane, gk0, gbar);
   } else {
     static_assert(KT > 0 && SG >= 0, "several tiles per thread only for a static K");
     // fast path: all U tiles lie in one aligned segment and are full, so their addresses are a stride apart
@@ -519,7 +528,7 @@ __global__ void __launch_bounds__(THREADS, MINB) fls_reduce_kernel(const __grid_
 #pragma unroll
       for (int u = 0; u < U; ++u)
 #pragma unroll
-        for (int b = 0; b < KT; ++b) load_raw(raw[u][b], a.grad[b], j0 + u * stride);
+        for (int b = 0; b < KT; ++b) load_raw(raw[u][b], a.grad[gk0 + b], j0 + u * stride);
       if (a.store_gbar) dep_wait();
 #pragma unroll
       for (int u = 0; u < U; ++u) {
@@ -531,25 +540,26 @@ __global__ void __launch_bounds__(THREADS, MINB) fls_reduce_kernel(const __grid_
         for (int e = 0; e < 8; ++e) { o.v[e] = g[e]; s8 = fmaf(g[e], g[e], s8); }
         sq += s8;
         if (a.store_gbar) {
-          if (first + u * T >= a.keep_from_tile) st8_keep(a.gbar + a0 + u * stride, o); else st8_stream(a.gbar + a0 + u * stride, o);
+          if (first + u * T >= a.keep_from_tile) st8_keep(gbar + a0 + u * stride, o); else st8_stream(gbar + a0 + u * stride, o);
         }
       }
     } else {
       for (int u = 0; u < U; ++u) {
         const uint32_t tile = first + u * T;
-        if (tile < a.idx.n_tiles) sq += reduce_one_tile<F32, KT, SG>(a, tile, lane);
+        if (tile < a.idx.n_tiles) sq += reduce_one_tile<F32, KT, SG>(a, tile, lane, gk0, gbar);
       }
     }
   }
   dep_wait();                            // partials, ticket and the norm slots belong to the predecessor until now
   dep_launch();
-  finish_norm<THREADS>(a, sq, &arrived);
+  finish_norm<THREADS>(a, sq, &arrived, y);
 }
 
 // ------------------------------------------------------------------------------------------------
 // K2: clip + AdamW + bf16 copy.
 // ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ void adamw_one(const AdamArgs& a, float c, float gbar, float& th, float& m, float& v) {
+template <class A>
+__device__ __forceinline__ void adamw_one(const A& a, float c, float gbar, float& th, float& m, float& v) {
   const float g = c * gbar;
   th = th * a.decay;                                        // decoupled weight decay: theta (1 - lr wd)
   m = fmaf(a.beta1, m, a.omb1 * g);
@@ -558,16 +568,10 @@ __device__ __forceinline__ void adamw_one(const AdamArgs& a, float c, float gbar
   th = fmaf(-a.step_size, __fdiv_rn(m, denom), th);         // step_size = lr / (1 - beta1^t)
 }
 
-__device__ __noinline__ void adamw_slice_scalar(const AdamArgs& a, float c, uint64_t j, uint64_t addr, uint32_t n) {
-  for (uint32_t e = 0; e < n; ++e) {
-    float th = a.theta[addr + e], m = a.m[addr + e], v = a.v[addr + e];
-    adamw_one(a, c, a.gbar[addr + e], th, m, v);
-    a.theta[addr + e] = th; a.m[addr + e] = m; a.v[addr + e] = v;
-    a.pbf16[j + e] = to_bf16_bits(th);
-  }
-}
-
-__global__ void __launch_bounds__(kThreads, 3) fls_adamw_kernel(const __grid_constant__ AdamArgs a) {
+// Body of the AdamW kernel for one group's state; A is AdamArgs or AdamBatchArgs (layout, direction, scalars).
+template <class A>
+__device__ __forceinline__ void adamw_tiles(const A& a, float* theta, float* m_, float* v_, uint16_t* pbf16, const float* gbar,
+                                            const float* coef) {
   const uint32_t n_tiles = a.idx.n_tiles;
   if (blockIdx.x >= n_tiles) { dep_wait(); dep_launch(); return; }
   float c = 0.f;
@@ -579,23 +583,38 @@ __global__ void __launch_bounds__(kThreads, 3) fls_adamw_kernel(const __grid_con
     const Slice s = slice_of(w.seek(tile), tile, threadIdx.x);
     if (s.vec) {
       // theta, m and v of this group are not touched by the reduce kernel: fetch them before waiting for it
-      F8 th = ld8_stream(a.theta + s.a);
-      F8 m = ld8_stream(a.m + s.a);
-      F8 v = ld8_stream(a.v + s.a);
-      if (!waited) { dep_wait(); dep_launch(); c = __ldcg(a.coef); waited = true; }
-      const F8 g = ld8_keep(a.gbar + s.a);
+      F8 th = ld8_stream(theta + s.a);
+      F8 m = ld8_stream(m_ + s.a);
+      F8 v = ld8_stream(v_ + s.a);
+      if (!waited) { dep_wait(); dep_launch(); c = __ldcg(coef); waited = true; }
+      const F8 g = ld8_keep(gbar + s.a);
 #pragma unroll
       for (int e = 0; e < 8; ++e) adamw_one(a, c, g.v[e], th.v[e], m.v[e], v.v[e]);
-      st8_stream(a.theta + s.a, th);
-      st8_stream(a.m + s.a, m);
-      st8_stream(a.v + s.a, v);
-      st_b128_stream(a.pbf16 + s.j, pack_bf16x8(th));
+      st8_stream(theta + s.a, th);
+      st8_stream(m_ + s.a, m);
+      st8_stream(v_ + s.a, v);
+      st_b128_stream(pbf16 + s.j, pack_bf16x8(th));
     } else if (s.n) {
-      if (!waited) { dep_wait(); dep_launch(); c = __ldcg(a.coef); waited = true; }
-      adamw_slice_scalar(a, c, s.j, s.a, s.n);
+      if (!waited) { dep_wait(); dep_launch(); c = __ldcg(coef); waited = true; }
+      for (uint32_t e = 0; e < s.n; ++e) {
+        float th = theta[s.a + e], m = m_[s.a + e], v = v_[s.a + e];
+        adamw_one(a, c, gbar[s.a + e], th, m, v);
+        theta[s.a + e] = th; m_[s.a + e] = m; v_[s.a + e] = v;
+        pbf16[s.j + e] = to_bf16_bits(th);
+      }
     }
   }
   if (!waited) { dep_wait(); dep_launch(); }
+}
+
+__global__ void __launch_bounds__(kThreads, 3) fls_adamw_kernel(const __grid_constant__ AdamArgs a) {
+  adamw_tiles(a, a.theta, a.m, a.v, a.pbf16, a.gbar, a.coef);
+}
+
+// The same for all groups in one grid (small plans, where one launch per group would be launch-bound).
+__global__ void __launch_bounds__(kThreads, 3) fls_adamw_batch_kernel(const __grid_constant__ AdamBatchArgs a) {
+  const uint32_t y = blockIdx.y;
+  adamw_tiles(a, a.theta[y], a.m[y], a.v[y], a.pbf16[y], a.gbar + size_t(y) * a.gbar_stride, a.coef + y);
 }
 
 // AdamW with the mean gradient formed in place (recompute plan).  With few gradient bytes per element
@@ -994,6 +1013,63 @@ void launch_reduce_t(const ReduceArgs& a, int sg, unsigned grid, cudaStream_t st
 unsigned reduce_grid(const ReduceArgs& a, int sg, bool f32) {
   const unsigned tiles_per_cta = reduce_tiles_per_cta(a, sg, f32);
   return (a.idx.n_tiles + tiles_per_cta - 1) / tiles_per_cta;
+}
+
+namespace {
+template <typename Args>
+void launch_k2(void (*kernel)(Args), const Args& a, unsigned grid_x, unsigned grid_y, unsigned threads, cudaStream_t st, bool overlap) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid_x, grid_y);
+  cfg.blockDim = dim3(threads);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = overlap ? 1 : 0;
+  cudaLaunchKernelEx(&cfg, kernel, a);
+}
+
+template <bool F32, int KT, int SG>
+void launch_reduce_batch_shape(const ReduceArgs& a, unsigned grid, unsigned groups, cudaStream_t st, bool ov) {
+  if constexpr (SG == 0)
+    launch_k2(fls_reduce_kernel<F32, KT, SG, kFlatThreads, kFlatMinB, 1, true>, a, grid, groups, kFlatThreads, st, ov);
+  else
+    launch_k2(fls_reduce_kernel<F32, KT, SG, kLevelThreads, kLevelMinB, 1, true>, a, grid, groups, kLevelThreads, st, ov);
+}
+
+template <bool F32>
+void launch_reduce_batch_t(const ReduceArgs& a, int sg, unsigned grid, unsigned groups, cudaStream_t st, bool ov) {
+  if (a.K == 4) {
+    if (sg == 0) launch_reduce_batch_shape<F32, 4, 0>(a, grid, groups, st, ov);
+    else if (sg == 1) launch_reduce_batch_shape<F32, 4, 1>(a, grid, groups, st, ov);
+    else launch_reduce_batch_shape<F32, 4, 2>(a, grid, groups, st, ov);
+  } else {
+    if (sg == 0) launch_reduce_batch_shape<F32, 8, 0>(a, grid, groups, st, ov);
+    else if (sg == 1) launch_reduce_batch_shape<F32, 8, 1>(a, grid, groups, st, ov);
+    else if (sg == 2) launch_reduce_batch_shape<F32, 8, 2>(a, grid, groups, st, ov);
+    else launch_reduce_batch_shape<F32, 8, 4>(a, grid, groups, st, ov);
+  }
+}
+}  // namespace
+
+bool reduce_batchable(uint32_t K, int sg) {
+  return (K == 4 && (sg == 0 || sg == 1 || sg == 2)) || (K == 8 && (sg == 0 || sg == 1 || sg == 2 || sg == 4));
+}
+
+cudaError_t launch_reduce_batch(const ReduceArgs& a, bool f32, int sg, unsigned groups, cudaStream_t st, bool overlap) {
+  const unsigned grid = reduce_grid(a, sg, f32);
+  if (f32)
+    launch_reduce_batch_t<true>(a, sg, grid, groups, st, overlap);
+  else
+    launch_reduce_batch_t<false>(a, sg, grid, groups, st, overlap);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_adamw_batch(const AdamBatchArgs& a, unsigned grid, unsigned groups, cudaStream_t st, bool overlap) {
+  launch_k2(fls_adamw_batch_kernel, a, grid, groups, kThreads, st, overlap);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_reduce(const ReduceArgs& a, bool f32, int sg, cudaStream_t st, bool overlap) {

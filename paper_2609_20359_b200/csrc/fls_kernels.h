@@ -20,8 +20,14 @@ struct SegIndex {
 };
 
 struct ReduceArgs {
-  const void* grad[FLS_MAX_GRAD_BUFFERS];  // device, K buffers of this group, index rho*S + sigma
+  const void* grad[FLS_MAX_GRAD_BUFFERS];  // device, K buffers of this group, index rho*S + sigma (batched launch: the
+                                           // buffers of all groups, index g*K + rho*S + sigma)
   float* gbar;                             // device, reduced gradient (shard order)
+  // Batched launch (gridDim.y = groups, K in {4, 8}): group y = blockIdx.y uses grad[y*K ..], gbar + y*gbar_stride,
+  // entries y*gridDim.x.. of partials, y*tree_stride.. of the chunk arrays, and entry y of ticket, norm_out, coef_out,
+  // normsq_out.  A plain launch is the case y = 0.
+  uint64_t gbar_stride;                    // elements
+  uint32_t tree_stride;                    // chunks per group
   SegIndex idx;
   uint32_t K;
   float k_float, inv_k;                    // K and 1/K as float: the mean is scaled by 1/K once
@@ -55,6 +61,20 @@ struct AdamArgs {
   SegIndex idx;
   int descending;
   const float* coef;                       // device, written by the reduce kernel of the same group
+  float decay, beta1, omb1, beta2, omb2, step_size, inv_sqrt_bc2, eps;
+};
+
+// AdamW of all groups in one grid (gridDim.y = groups): group y = blockIdx.y.
+struct AdamBatchArgs {
+  float* theta[FLS_MAX_GROUPS];
+  float* m[FLS_MAX_GROUPS];
+  float* v[FLS_MAX_GROUPS];
+  uint16_t* pbf16[FLS_MAX_GROUPS];
+  const float* gbar;                       // group 0's reduced gradient
+  uint64_t gbar_stride;                    // elements between the groups' reduced gradients
+  const float* coef;                       // group 0's clip coefficient; group y's is coef[y]
+  SegIndex idx;
+  int descending;
   float decay, beta1, omb1, beta2, omb2, step_size, inv_sqrt_bc2, eps;
 };
 
@@ -115,6 +135,10 @@ unsigned reduce_grid(const ReduceArgs& a, int sg, bool f32);
 // overlap: launch with programmatic stream serialization, so that the kernel's first CTAs may start during
 // the tail of the kernel launched just before it on the same stream (which must be one of these three).
 cudaError_t launch_reduce(const ReduceArgs& a, bool f32, int sg, cudaStream_t st, bool overlap);
+// All groups in one grid; only for K in {4, 8} with a static level structure (reduce_batchable).
+bool reduce_batchable(uint32_t K, int sg);
+cudaError_t launch_reduce_batch(const ReduceArgs& a, bool f32, int sg, unsigned groups, cudaStream_t st, bool overlap);
+cudaError_t launch_adamw_batch(const AdamBatchArgs& a, unsigned grid, unsigned groups, cudaStream_t st, bool overlap);
 cudaError_t launch_step_noclip(const ReduceAdamArgs& a, bool f32, int sg, cudaStream_t st, bool overlap);
 cudaError_t launch_reduce_adamw(const ReduceAdamArgs& a, bool f32, int sg, unsigned grid, cudaStream_t st, bool overlap);
 cudaError_t launch_adamw(const AdamArgs& a, unsigned grid, cudaStream_t st, bool overlap);

@@ -10,7 +10,7 @@
 namespace fls {
 
 std::string build_layout(const std::vector<uint64_t>& unit_numel, uint32_t S, uint32_t Q, uint32_t scratch_slots,
-                         uint32_t ring_replicas, Layout* out) {
+                         uint32_t ring_replicas, uint32_t groups, Layout* out) {
   if (unit_numel.empty()) return "empty unit table";
   if (S == 0 || Q == 0) return "shard_dim and align_elems must be >= 1";
   Layout& L = *out;
@@ -74,10 +74,13 @@ std::string build_layout(const std::vector<uint64_t>& unit_numel, uint32_t S, ui
   if (L.n_tiles >= (1ull << 32)) return "plan too large";
   L.ws_partials_offset = (kWsSegments + seg_bytes + 255) / 256 * 256;
   // norm tree: at most one partial per tile, then one sum and one arrival counter per chunk of kNormChunkCtas partials
+  // (per group: group g's arrays start g * n_tiles, g * n_chunks entries in)
   const uint64_t n_chunks = (L.n_tiles + kNormChunkCtas - 1) / kNormChunkCtas;
-  L.ws_chunk_partials_offset = (L.ws_partials_offset + 8 * L.n_tiles + 255) / 256 * 256;
-  L.ws_chunk_count_offset = (L.ws_chunk_partials_offset + 8 * n_chunks + 255) / 256 * 256;
-  L.ws_chunk_count_bytes = 4 * n_chunks;
+  const uint64_t G = groups ? groups : 1;
+  L.n_chunks = n_chunks;
+  L.ws_chunk_partials_offset = (L.ws_partials_offset + 8 * L.n_tiles * G + 255) / 256 * 256;
+  L.ws_chunk_count_offset = (L.ws_chunk_partials_offset + 8 * n_chunks * G + 255) / 256 * 256;
+  L.ws_chunk_count_bytes = 4 * n_chunks * G;
   L.ws_scratch_offset = (L.ws_chunk_count_offset + L.ws_chunk_count_bytes + 255) / 256 * 256;
   L.scratch_slots = scratch_slots ? scratch_slots : 1;
   L.scratch_stride = (4ull * L.n_padded + 255) / 256 * 256;

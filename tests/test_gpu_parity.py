@@ -112,6 +112,56 @@ def test_tuned_launch_shapes_give_identical_results(fls, ctas, descending, overl
     assert all(torch.equal(x, y) for x, y in zip(run(False), run(True)))
 
 
+@pytest.mark.parametrize("units,G,S,R_rep,Q,dtype,fused", [
+    ([40000, 30011, 5000], 3, 4, 1, 8, "bf16", False),     # K = 4 flat
+    ([40000, 30011, 5000], 4, 8, 1, 8, "bf16", True),      # K = 8 flat, fused aggregation on the one reduce grid
+    ([40000, 30011], 2, 4, 2, 8, "bf16", True),            # two-level 4 x 2
+    ([70001], 8, 2, 2, 1, "f32", False),                   # fp32 gradients, unaligned shards, G*K = 32
+    ([1000003], 2, 4, 1, 1, "bf16", True),                 # the tiny workload's shape
+    ([17], 2, 2, 2, 1, "bf16", False),
+])
+def test_groups_in_one_grid_give_identical_results(fls, units, G, S, R_rep, Q, dtype, fused):
+    """Small plans run all groups in one reduce grid and one AdamW grid (the group is the grid's y coordinate).
+    Against the oracle, and bit for bit against one launch per group; the launch count shows which way it ran."""
+    outs, launches = [], []
+    counts = [sy.sample_count(29, g) for g in range(G)]
+    for mode in (-1, 0):
+        c = Case(units, G, S, R_rep, H=2, Q=Q, grad_dtype=dtype, opt_state=True, hp=orc.Hyper(max_grad_norm=0.05), fused=fused,
+                 per_buffer_scale=True)
+        fls.fls_plan_set_batching(c.sess.plan, mode)
+        assert fls.fls_plan_get_batching(c.sess.plan) == (mode == -1)      # these plans are small: automatic means on
+        for _ in range(4):
+            c.step(counts)
+            c.compare()
+        outs.append([x.clone() for x in c.sess.master + c.sess.m + c.sess.v + c.sess.param_bf16] + [c.sess.norms().clone(), c.sess.coefs().clone()])
+        launches.append(fls.fls_get_launch_count(c.sess.plan))
+        assert c.sess.status() == 0
+        c.close()
+    assert all(torch.equal(x, y) for x, y in zip(*outs))
+    n_avg = 3                                                             # opt_state: FedAvg launches per call (parameters, m, v)
+    if fused and G <= 16:
+        assert launches == [2 * 2 + 2 * 2, 2 * 2 * G + 2 * (G + 1)]       # plain steps: 2 | 2G; aggregation steps: 2 | G + 1
+    else:
+        assert launches == [4 * 2 + 2 * n_avg, 4 * 2 * G + 2 * n_avg]
+
+
+def test_batching_is_automatic_only_for_small_plans(fls):
+    from paper_2609_20359_b200.session import Session
+    big = Session(6_000_000, None, groups=2, shard_dim=4, fused=True)      # 2 x 24 MB of reduced gradients: above 32 MiB
+    assert not fls.fls_plan_get_batching(big.plan)
+    fls.fls_plan_set_batching(big.plan, 1)                                  # the fused plan has a slot per group: may be forced
+    assert fls.fls_plan_get_batching(big.plan)
+    big.close()
+    unfused = Session(6_000_000, None, groups=2, shard_dim=4)
+    with pytest.raises(fls.FlsError) as e:
+        fls.fls_plan_set_batching(unfused.plan, 1)                          # one slot only
+    assert e.value.code == fls.FLS_ESTATE
+    unfused.close()
+    odd = Session(4096, None, groups=2, shard_dim=3)                        # K = 3: no batched kernel
+    assert not fls.fls_plan_get_batching(odd.plan)
+    odd.close()
+
+
 @pytest.mark.parametrize("units,G,S,R_rep,Q,dtype", [([40000, 30011], 2, 1, 1, 8, "bf16"), ([40000, 30011], 2, 2, 1, 8, "bf16"),
                                                      ([40000, 30011], 2, 1, 2, 8, "bf16"), ([70001], 2, 3, 1, 1, "bf16"),
                                                      ([70001], 2, 1, 3, 8, "bf16"), ([40000, 30011], 2, 1, 1, 8, "f32")])
@@ -685,7 +735,7 @@ def _random_cases(n, seed=20260920):
                         dtype=dtype, opt_state=bool(rng.integers(0, 2)), fused=bool(rng.integers(0, 2)), wire=wire, ring=ring,
                         per_replica=per_replica, spec=spec, H=int(rng.choice([1, 2, 3])), clip=clip,
                         ctas=int(rng.choice([0, 0, 1, 5])), desc=int(rng.integers(0, 2)), overlap=bool(rng.integers(0, 2)),
-                        keep_mb=float(rng.choice([0.0, 0.05, 64.0])), idx=i))
+                        keep_mb=float(rng.choice([0.0, 0.05, 64.0])), batch=int(rng.choice([-1, 0, 1])), idx=i))
     return out
 
 
@@ -701,6 +751,10 @@ def test_random_combinations(fls, p):
         fls.fls_plan_tune(c.sess.plan, kern, p["ctas"], p["desc"])
     fls.fls_plan_set_overlap(c.sess.plan, p["overlap"])
     fls.fls_plan_set_l2_keep(c.sess.plan, int(p["keep_mb"] * 2 ** 20))
+    try:
+        fls.fls_plan_set_batching(c.sess.plan, p["batch"])
+    except fls.FlsError as e:                               # forcing it on a plan that cannot share a grid
+        assert p["batch"] == 1 and e.code == fls.FLS_ESTATE
     counts = [sy.sample_count(p["idx"], g) for g in range(p["G"])]
     for _ in range(3):
         c.step(counts)
