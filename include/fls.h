@@ -284,9 +284,9 @@ int fls_get_state(const fls_plan* plan, uint32_t copy, float** master, float** m
 /* Small plans are launch-bound when every group gets its own two kernels.  When the plan allows it (G > 1, G*K <= 64,
  * K = 4 or 8 in a flat or 1/2/4-wide two-level order, the default two-pass route, one state copy per group, and a
  * reduced-gradient slot per group in the workspace: FLS_AVG_FUSED plans and plans whose G reduced gradients need at
- * most 32 MiB) fls_sync_step can run all groups in ONE reduce grid and ONE AdamW grid, with the group in the grid's y
+ * most 24 MiB) fls_sync_step can run all groups in ONE reduce grid and ONE AdamW grid, with the group in the grid's y
  * dimension; fls_sync_step_fedavg then uses the one reduce grid as well.  mode -1 (default): automatically, only while
- * the G reduced gradients fit in 32 MiB (beyond that the per-group sequence is faster: its reduced gradient is still in
+ * the G reduced gradients fit in 24 MiB (beyond that the per-group sequence is faster: its reduced gradient is still in
  * L2 when AdamW reads it); 0: never; 1: whenever the plan allows it (FLS_ESTATE otherwise).  Results do not change.
  * fls_plan_get_batching: whether the next fls_sync_step would run that way. */
 int fls_plan_set_batching(fls_plan* plan, int mode);

@@ -47,7 +47,7 @@ struct Range {
 
 }  // namespace
 
-constexpr uint64_t kBatchScratchBytes = 32ull << 20;
+constexpr uint64_t kBatchScratchBytes = 24ull << 20;
 
 struct fls_plan {
   fls_plan_desc desc{};
@@ -106,7 +106,7 @@ struct fls_plan {
   uint32_t* d_spec_counts() const { return reinterpret_cast<uint32_t*>(ws + kWsStatus) + 2; }
   // One grid for all groups (instead of one launch per group) needs a reduced-gradient slot per group, a level structure
   // the batched kernels are built for, the default two-pass route and one state copy per group.  Automatic: only when all
-  // the reduced gradients together fit in a quarter of the L2 (32 MiB), i.e. when a launch per group would be launch-bound;
+  // the reduced gradients together take at most 24 MiB (a fifth of the L2), i.e. when a launch per group would be launch-bound;
   // larger plans keep the per-group sequence, whose reduced gradient is still in L2 when AdamW reads it.
   bool can_batch() const {
     return desc.groups > 1 && lay.scratch_slots >= desc.groups && uint64_t(desc.groups) * K <= FLS_MAX_GRAD_BUFFERS &&

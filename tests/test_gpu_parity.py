@@ -147,7 +147,7 @@ def test_groups_in_one_grid_give_identical_results(fls, units, G, S, R_rep, Q, d
 
 def test_batching_is_automatic_only_for_small_plans(fls):
     from paper_2609_20359_b200.session import Session
-    big = Session(6_000_000, None, groups=2, shard_dim=4, fused=True)      # 2 x 24 MB of reduced gradients: above 32 MiB
+    big = Session(6_000_000, None, groups=2, shard_dim=4, fused=True)      # 2 x 24 MB of reduced gradients: above 24 MiB
     assert not fls.fls_plan_get_batching(big.plan)
     fls.fls_plan_set_batching(big.plan, 1)                                  # the fused plan has a slot per group: may be forced
     assert fls.fls_plan_get_batching(big.plan)
@@ -517,10 +517,12 @@ def test_speculative_mixed_hits_and_misses_and_errors(fls):
     noclip.close()
 
 
-@pytest.mark.parametrize("G,nesterov,opt_state,units,Q", [(4, True, False, [30000, 517], 8), (3, False, True, [70001], 1), (9, True, False, [999], 8)])
-def test_fedavg_outer_optimizer(fls, G, nesterov, opt_state, units, Q):
-    """Aggregation through an outer SGD step with momentum on a global copy, three rounds, against the oracle."""
-    c = Case(units, G, 2, 1, H=1, Q=Q, opt_state=opt_state, hp=orc.Hyper(max_grad_norm=0.01))
+@pytest.mark.parametrize("G,nesterov,opt_state,units,Q,R_rep", [(4, True, False, [30000, 517], 8, 1), (3, False, True, [70001], 1, 1),
+                                                                 (9, True, False, [999], 8, 1), (3, True, True, [30000, 517], 8, 2)])
+def test_fedavg_outer_optimizer(fls, G, nesterov, opt_state, units, Q, R_rep):
+    """Aggregation through an outer SGD step with momentum on a global copy, three rounds, against the oracle (the last
+    case with one state copy per replica: the new global parameters reach every copy)."""
+    c = Case(units, G, 2, R_rep, H=1, Q=Q, opt_state=opt_state, hp=orc.Hyper(max_grad_norm=0.01), state_per_replica=R_rep > 1)
     counts = [sy.sample_count(31, g) for g in range(G)]
     xg = c.states[0].theta.copy()
     buf = np.zeros_like(xg)
@@ -534,13 +536,18 @@ def test_fedavg_outer_optimizer(fls, G, nesterov, opt_state, units, Q):
             mbar = orc.fedavg_array([st.m for st in c.states], w); vbar = orc.fedavg_array([st.v for st in c.states], w)
             for st in c.states:
                 st.m = mbar.copy(); st.v = vbar.copy()
+        for reps in c.copies:   # the broadcast inside every group
+            for st in reps[1:]:
+                st.theta = reps[0].theta.copy(); st.param_bf16 = reps[0].param_bf16.copy()
+                if opt_state:
+                    st.m = reps[0].m.copy(); st.v = reps[0].v.copy()
         fls.fls_fedavg_outer(c.sess.plan, counts, 0.7, 0.9, nesterov, d_xg, d_buf)
         c.compare(check_norms=False)
         assert_state_close(d_xg.cpu().numpy(), orc.pack_sharded(c.L, xg), "x_global")
         # the buffer accumulates x_global - xbar, a difference of nearly equal fp32 numbers: its error is a few
         # ulps of the parameters' magnitude (0.02 -> 2e-9), whatever the size of the difference itself
         assert np.allclose(d_buf.cpu().numpy(), orc.pack_sharded(c.L, buf), rtol=1e-5, atol=3e-8)
-        assert torch.equal(c.sess.master[G - 1], d_xg)
+        assert all(torch.equal(x, d_xg) for x in c.sess.master)
     with pytest.raises(fls.FlsError) as e:
         fls.fls_fedavg_outer(c.sess.plan, counts, float("nan"), 0.9, True, d_xg, d_buf)
     assert e.value.code == fls.FLS_EINVAL
