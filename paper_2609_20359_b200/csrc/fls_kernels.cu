@@ -454,8 +454,9 @@ __device__ __forceinline__ void begin_norm(unsigned* arrived) {
 
 // One pass, no loop: a CTA of THREADS threads owns U * THREADS/256 consecutive tiles (each group of 256
 // threads takes every (THREADS/256)-th of them, U in all) and the grid covers the whole buffer.  MINB resident
-// CTAs per SM fix the register budget: 256 x 8 (32 registers) for the flat order with K = 4 or 8, 256 x 6 (40
-// registers) for the two-level orders, which carry a second set of accumulators, 256 x 2 for a run-time K.
+// CTAs per SM fix the register budget: 256 x 8 (32 registers) for the flat order with K = 4 or 8, 256 x 5 (48
+// registers, what the kernel needs without spilling) for the two-level orders, which carry a second set of
+// accumulators; 256 x 2 for a run-time K.
 // Small CTAs turn over independently (no warp waits for the slowest of 32); they became the fastest shape once
 // the norm epilogue lost its block-wide barriers.
 // With K = 1 or 2 a thread would have only one or two 16-byte loads in flight, so those shapes take U > 1 tiles
@@ -937,7 +938,7 @@ __global__ void __launch_bounds__(kThreads, 3) fls_adamw_fedavg_kernel(const __g
 #endif
 #ifndef FLS_LEVEL_THREADS
 #define FLS_LEVEL_THREADS 256
-#define FLS_LEVEL_MINB 6
+#define FLS_LEVEL_MINB 5
 #endif
 constexpr int kFlatThreads = FLS_FLAT_THREADS, kFlatMinB = FLS_FLAT_MINB;       // SG == 0 with a static K
 constexpr int kLevelThreads = FLS_LEVEL_THREADS, kLevelMinB = FLS_LEVEL_MINB;   // two-level orders with a static K
