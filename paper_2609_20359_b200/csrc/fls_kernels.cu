@@ -608,12 +608,18 @@ __device__ __forceinline__ void adamw_tiles(const A& a, float* theta, float* m_,
   if (!waited) { dep_wait(); dep_launch(); }
 }
 
-__global__ void __launch_bounds__(kThreads, 3) fls_adamw_kernel(const __grid_constant__ AdamArgs a) {
+#ifndef FLS_ADAMW_MINB
+#define FLS_ADAMW_MINB 3
+#endif
+#ifndef FLS_FUSED_MINB
+#define FLS_FUSED_MINB 3
+#endif
+__global__ void __launch_bounds__(kThreads, FLS_ADAMW_MINB) fls_adamw_kernel(const __grid_constant__ AdamArgs a) {
   adamw_tiles(a, a.theta, a.m, a.v, a.pbf16, a.gbar, a.coef);
 }
 
 // The same for all groups in one grid (small plans, where one launch per group would be launch-bound).
-__global__ void __launch_bounds__(kThreads, 3) fls_adamw_batch_kernel(const __grid_constant__ AdamBatchArgs a) {
+__global__ void __launch_bounds__(kThreads, FLS_ADAMW_MINB) fls_adamw_batch_kernel(const __grid_constant__ AdamBatchArgs a) {
   const uint32_t y = blockIdx.y;
   adamw_tiles(a, a.theta[y], a.m[y], a.v[y], a.pbf16[y], a.gbar + size_t(y) * a.gbar_stride, a.coef + y);
 }
@@ -873,7 +879,7 @@ __device__ __noinline__ void fused_slice_scalar(const FusedArgs& a, uint64_t j, 
 }
 
 template <bool OPT>
-__global__ void __launch_bounds__(kThreads, 3) fls_adamw_fedavg_kernel(const __grid_constant__ FusedArgs a) {
+__global__ void __launch_bounds__(kThreads, FLS_FUSED_MINB) fls_adamw_fedavg_kernel(const __grid_constant__ FusedArgs a) {
   const uint32_t n_tiles = a.idx.n_tiles;
   if (blockIdx.x >= n_tiles) { dep_wait(); dep_launch(); return; }
   bool waited = false;
