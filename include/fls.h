@@ -125,7 +125,7 @@ typedef struct {
                                index g*R_rep + rho): fp32 parameters, shard order, in/out                   */
   float* const* m;          /* same: first moment                                                        */
   float* const* v;          /* same: second moment                                                       */
-  void* const* param_bf16;  /* host array of G device pointers: bf16 copy, unsharded order, output       */
+  void* const* param_bf16;  /* host array of n_state_copies device pointers: bf16 copy, unsharded order, output */
   void* workspace;          /* device, >= workspace_bytes; holds the reduced gradient, the norm partials,
                                per-group norm / clip coefficient, the status word and the segment table  */
   uint64_t workspace_bytes;
@@ -168,10 +168,12 @@ int fls_plan_bind(fls_plan* plan, const fls_buffers* buffers);
 /* One local training step of all G groups (the groups train without waiting for one another), enqueued
  * on `cuda_stream` (a cudaStream_t; NULL = default stream).  Per group: mean of the K gradient buffers
  * in fp32, ascending buffer order inside a sharding group, then ascending replica order (reduce-scatter
- * over S, then all-reduce over R: Background FSDP/HSDP, Eq. 2), one multiply by 1/K; L2 norm of the mean
+ * over S, then all-reduce over R: Background FSDP/HSDP, Eq. 2; reduce_wire and reduce_order change the
+ * precision of the partial sums and the order), one multiply by 1/K; L2 norm of the mean
  * gradient over the whole group; c = min(1, max_grad_norm/(norm + 1e-6)); AdamW with decoupled weight
- * decay and bias correction on master/m/v in place; bf16 copy of the new parameters (round to nearest
- * even).  `lr` overrides the plan's learning rate for this step; pass NaN to use the plan's.  The step
+ * decay and bias correction on master/m/v in place (on every state copy of the group; speculative plans
+ * write the other buffer set, see fls_plan_set_speculative); bf16 copy of the new parameters (round to
+ * nearest even).  `lr` overrides the plan's learning rate for this step; pass NaN to use the plan's.  The step
  * counter t is incremented; *fedavg_due (host, may be NULL) is set to (t % H == 0).
  * Errors: FLS_ESTATE if not bound, FLS_ECUDA on a launch failure (state is then undefined). */
 int fls_sync_step(fls_plan* plan, double lr, void* cuda_stream, int* fedavg_due);
@@ -187,7 +189,9 @@ int fls_sync_step_host(fls_plan* plan, const void* const* host_grads, double lr,
 /* FedAvg: every group's parameters become sum_g w_g x_g, w_g = n_g / sum n (the weighted mean of the
  * locally trained models of Background "Federated Learning", taken shard by shard across the federation
  * groups, Section FL+FSDP).  fp32 accumulation in ascending group order; all G master copies and
- * all G bf16 copies are rewritten; m and v too if the plan has FLS_AVG_OPT_STATE.  sample_counts: host,
+ * all G bf16 copies are rewritten; m and v too if the plan has FLS_AVG_OPT_STATE.  With
+ * FLS_STATE_PER_REPLICA replica 0 of every group is read and all G*R_rep copies are rewritten (the
+ * broadcast inside each group, Section FL+HSDP).  sample_counts: host,
  * G entries, NULL = equal weights.  The step counter is unchanged.
  * Errors: FLS_EINVAL if all counts are zero, FLS_ESTATE, FLS_ECUDA. */
 int fls_fedavg(fls_plan* plan, const uint64_t* sample_counts, void* cuda_stream);
@@ -211,8 +215,8 @@ int fls_fedavg_outer(fls_plan* plan, const uint64_t* sample_counts, double outer
  * its optimizer update).  With FLS_AVG_FUSED in the plan and G <= FLS_MAX_FUSED_GROUPS the aggregation is fused
  * into the optimizer kernel: after the G reductions one kernel applies AdamW to every group's element,
  * averages the G results in registers and writes the average to all G copies, which saves FedAvg's own
- * read and write of the parameters (10*G bytes per parameter).  Otherwise it runs the two calls one after the
- * other.  sample_counts: host, G entries, NULL = equal weights.  Errors: as fls_sync_step and fls_fedavg. */
+ * read and write of the parameters (10*G bytes per parameter).  Otherwise (and with more than 32 extra replica
+ * copies) it runs the two calls one after the other.  sample_counts: host, G entries, NULL = equal weights.  Errors: as fls_sync_step and fls_fedavg. */
 int fls_sync_step_fedavg(fls_plan* plan, double lr, const uint64_t* sample_counts, void* cuda_stream);
 
 /* Device pointers (inside the workspace) to G floats each: the gradient norm and the clip coefficient of
