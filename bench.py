@@ -38,7 +38,7 @@ OTHER_WORKLOADS = ("llama31_8b_block_fl_fsdp", "gpt2_small_fl_fsdp")
 # slices of the workloads (one kernel per capture, a few GB on the device); the traffic of these streams grows
 # in proportion to the element count, so a launch over N elements moves N times the figure.  Keyed by kernel
 # and, for the kernels that read the gradients, by the gradient bytes per element K*e_g.
-NCU_TRAFFIC_BYTES_PER_ELEM = {("reduce", 16): 19.59, ("adamw", None): 28.85, ("adamw_fedavg", None): 29.39, ("fedavg", None): 9.54,
+NCU_TRAFFIC_BYTES_PER_ELEM = {("reduce", 16): 19.46, ("adamw", None): 28.85, ("adamw_fedavg", None): 29.39, ("fedavg", None): 9.54,
                               ("step_noclip", 16): 40.66}
 # The CPU oracle is timed on the first ORACLE_SAMPLE parameters of every buffer: once on one thread, once with
 # the sample cut into chunks that a pool of all host cores works through.
