@@ -378,7 +378,12 @@ def measure_workload(args, cfg, fls, Session, rank, world, local, with_e2e, samp
     if with_e2e and h2d > args.e2e_max_gb * 2 ** 30:
         e2e = {"value": None, "unit": UNIT, "skipped": f"pinned host buffers above --e2e-max-gb {args.e2e_max_gb}"}
     elif with_e2e:
-        host = [[torch.empty(sess.n_padded, dtype=sess.grad_torch_dtype, pin_memory=True) for _ in range(sess.K)] for _ in range(G)]
+        try:
+            host = [[torch.empty(sess.n_padded, dtype=sess.grad_torch_dtype, pin_memory=True) for _ in range(sess.K)] for _ in range(G)]
+        except RuntimeError as err:                  # the host cannot pin that much memory: say so instead of failing the run
+            host = None
+            e2e = {"value": None, "unit": UNIT, "skipped": f"pinned host buffers of {h2d} bytes could not be allocated: {str(err)[:120]}"}
+    if with_e2e and e2e is None:
         for g in range(G):
             for k in range(sess.K):
                 host[g][k].copy_(sess.grads[g][k])
@@ -497,7 +502,14 @@ def run_ours(args, cfg):
         for name in OTHER_WORKLOADS:
             if name == cfg["name"]:
                 continue
-            r = measure_workload(args, sy.config_by_name(name), fls, Session, rank, world, local, False, sampler)
+            try:
+                r = measure_workload(args, sy.config_by_name(name), fls, Session, rank, world, local, False, sampler)
+            except (RuntimeError, MemoryError) as err:     # e.g. not enough free HBM: the main line must still be printed
+                if world > 1:
+                    raise                                   # the ranks' barriers would no longer match
+                others[name] = {"error": str(err)[:200]}
+                torch.cuda.empty_cache()
+                continue
             if r is not None:
                 others[name] = {k: r[k] for k in ("value", "ms_per_step", "hbm_gbs", "hbm_frac_of_measured_peak", "hbm_frac_of_8tbs",
                                                   "roofline", "kernels", "gpu_launches", "config")}
