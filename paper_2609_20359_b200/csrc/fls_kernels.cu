@@ -839,21 +839,12 @@ __global__ void __launch_bounds__(kThreads, MINB) fls_fedavg_kernel(const __grid
 // results are bit-identical to the two-kernel sequence; what is saved is FedAvg's own pass over the
 // parameters.  m and v stay per group unless the plan averages the optimizer state.
 // ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ void adamw_one_f(const FusedArgs& a, float c, float gbar, float& th, float& m, float& v) {
-  const float g = c * gbar;
-  th = th * a.decay;
-  m = fmaf(a.beta1, m, a.omb1 * g);
-  v = fmaf(a.beta2, v, a.omb2 * (g * g));
-  const float denom = fmaf(sqrtf(v), a.inv_sqrt_bc2, a.eps);
-  th = fmaf(-a.step_size, __fdiv_rn(m, denom), th);
-}
-
 __device__ __noinline__ void fused_slice_scalar(const FusedArgs& a, uint64_t j, uint64_t addr, uint32_t n) {
   for (uint32_t e = 0; e < n; ++e) {
     float ath = 0.f, am = 0.f, av = 0.f;
     for (uint32_t g = 0; g < a.G; ++g) {
       float th = a.theta[g][addr + e], m = a.m[g][addr + e], v = a.v[g][addr + e];
-      adamw_one_f(a, __ldcg(a.coefs + g), a.gbar[g][addr + e], th, m, v);
+      adamw_one(a, __ldcg(a.coefs + g), a.gbar[g][addr + e], th, m, v);
       ath = fmaf(a.w[g], th, ath);
       if (a.avg_opt_state) { am = fmaf(a.w[g], m, am); av = fmaf(a.w[g], v, av); }
       else {
@@ -903,7 +894,7 @@ __global__ void __launch_bounds__(kThreads, FLS_FUSED_MINB) fls_adamw_fedavg_ker
         const float c = __ldcg(a.coefs + g), wg = a.w[g];
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-          adamw_one_f(a, c, gb.v[e], th.v[e], m.v[e], v.v[e]);
+          adamw_one(a, c, gb.v[e], th.v[e], m.v[e], v.v[e]);
           ath.v[e] = fmaf(wg, th.v[e], ath.v[e]);
           if (OPT) { am.v[e] = fmaf(wg, m.v[e], am.v[e]); av.v[e] = fmaf(wg, v.v[e], av.v[e]); }
         }
