@@ -460,7 +460,7 @@ __device__ __forceinline__ void begin_norm(unsigned* arrived) {
 // Small CTAs turn over independently (no warp waits for the slowest of 32); they became the fastest shape once
 // the norm epilogue lost its block-wide barriers.
 // With K = 1 or 2 a thread would have only one or two 16-byte loads in flight, so those shapes take U > 1 tiles
-// per thread (512 x 2 CTAs) and issue the loads of all of them before the first add.
+// per thread (256 x 4 CTAs, 64 registers) and issue the loads of all of them before the first add.
 template <bool F32, int KT, int SG>
 __device__ __forceinline__ float reduce_one_tile(const ReduceArgs& a, uint32_t tile, uint32_t lane, uint32_t gk0, float* gbar) {
   float sq = 0.f;
@@ -940,7 +940,11 @@ __global__ void __launch_bounds__(kThreads, FLS_FUSED_MINB) fls_adamw_fedavg_ker
 constexpr int kFlatThreads = FLS_FLAT_THREADS, kFlatMinB = FLS_FLAT_MINB;       // SG == 0 with a static K
 constexpr int kLevelThreads = FLS_LEVEL_THREADS, kLevelMinB = FLS_LEVEL_MINB;   // two-level orders with a static K
 constexpr int kAnyThreads = 256, kAnyMinB = 2;         // run-time K: batches of 8 loads need the registers
-constexpr int kFewThreads = 512, kFewMinB = 2;         // K = 1 or 2: several tiles per thread (see tiles_per_thread)
+#ifndef FLS_FEW_THREADS
+#define FLS_FEW_THREADS 256
+#define FLS_FEW_MINB 4
+#endif
+constexpr int kFewThreads = FLS_FEW_THREADS, kFewMinB = FLS_FEW_MINB;   // K = 1 or 2: several tiles per thread (see tiles_per_thread)
 
 // tiles per thread so that 8 (bf16) or 4 (fp32, 32-byte) loads are in flight per thread; 1 for K >= 4
 template <bool F32, int KT> constexpr int tiles_per_thread() { return (KT == 1 || KT == 2) ? (F32 ? 4 : 8) / KT : 1; }
