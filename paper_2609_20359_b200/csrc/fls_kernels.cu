@@ -768,9 +768,13 @@ __device__ __noinline__ void fedavg_slice_scalar(const FedavgArgs& a, uint64_t j
   }
 }
 
+#ifndef FLS_FEDAVG_BATCH
+#define FLS_FEDAVG_BATCH 8               // copies loaded before the first use (G = 8 and run-time G)
+#define FLS_FEDAVG_BATCH_MINB 2
+#endif
 template <int GT, int MINB>
 __global__ void __launch_bounds__(kThreads, MINB) fls_fedavg_kernel(const __grid_constant__ FedavgArgs a) {
-  constexpr int B = GT ? GT : 8;
+  constexpr int B = (GT == 0 || GT > FLS_FEDAVG_BATCH) ? FLS_FEDAVG_BATCH : GT;
   const uint32_t G = GT ? uint32_t(GT) : a.G;
   const uint32_t n_tiles = a.idx.n_tiles;
   dep_wait();                            // the copies being averaged were just written by the predecessor
@@ -790,11 +794,11 @@ __global__ void __launch_bounds__(kThreads, MINB) fls_fedavg_kernel(const __grid
         F8 raw[B];
 #pragma unroll
         for (int b = 0; b < B; ++b)
-          if (GT || g0 + b < G) raw[b] = ld8_stream(a.x[GT ? b : g0 + b] + s.a);
+          if (GT || g0 + b < G) raw[b] = ld8_stream(a.x[g0 + b] + s.a);
 #pragma unroll
         for (int b = 0; b < B; ++b) {
           if (GT || g0 + b < G) {
-            const float wg = a.w[GT ? b : g0 + b];
+            const float wg = a.w[g0 + b];
 #pragma unroll
             for (int e = 0; e < 8; ++e) acc.v[e] = fmaf(wg, raw[b].v[e], acc.v[e]);   // acc starts at 0: first term w_0 x_0
           }
@@ -1155,8 +1159,8 @@ cudaError_t launch_fedavg(const FedavgArgs& a, unsigned grid, cudaStream_t st, b
     case 1: launch_k(fls_fedavg_kernel<1, 6>, a, grid, kThreads, st, overlap); break;
     case 2: launch_k(fls_fedavg_kernel<2, 5>, a, grid, kThreads, st, overlap); break;
     case 4: launch_k(fls_fedavg_kernel<4, 4>, a, grid, kThreads, st, overlap); break;
-    case 8: launch_k(fls_fedavg_kernel<8, 2>, a, grid, kThreads, st, overlap); break;
-    default: launch_k(fls_fedavg_kernel<0, 2>, a, grid, kThreads, st, overlap); break;
+    case 8: launch_k(fls_fedavg_kernel<8, FLS_FEDAVG_BATCH_MINB>, a, grid, kThreads, st, overlap); break;
+    default: launch_k(fls_fedavg_kernel<0, FLS_FEDAVG_BATCH_MINB>, a, grid, kThreads, st, overlap); break;
   }
   return cudaGetLastError();
 }
