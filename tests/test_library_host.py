@@ -31,6 +31,33 @@ def test_library_exports_every_declared_symbol(fls):
         assert hasattr(lib, name), name
 
 
+def test_header_is_plain_c(tmp_path):
+    """include/fls.h is the boundary: it must compile as C99 on its own, and a C program must link against the library."""
+    import shutil
+    import subprocess
+    if shutil.which("gcc") is None:
+        pytest.skip("no C compiler")
+    src = tmp_path / "use_fls.c"
+    src.write_text('#include "fls.h"\n#include <stdio.h>\n'
+                   'int main(void) {\n'
+                   '  fls_plan_desc d = {0}; fls_plan* p = 0; fls_layout lay; fls_comm_costs c;\n'
+                   '  d.n_params = 1000; d.groups = 2; d.shard_dim = 4; d.replicate_dim = 1; d.sync_period = 2; d.align_elems = 8;\n'
+                   '  d.fedavg_what = FLS_AVG_PARAMS; d.lr = 3e-4; d.beta1 = 0.9; d.beta2 = 0.95; d.eps = 1e-8; d.weight_decay = 0.1; d.max_grad_norm = 1.0;\n'
+                   '  if (fls_plan_create(&d, &p) != FLS_OK) { printf("%s\\n", fls_last_error()); return 1; }\n'
+                   '  if (fls_plan_query(p, &lay) != FLS_OK || fls_comm_report(p, 0, &c) != FLS_OK) return 2;\n'
+                   '  printf("%llu %llu %.0f\\n", (unsigned long long)lay.n_padded, (unsigned long long)lay.shard_numel, c.hbm_bytes_sync_step);\n'
+                   '  return fls_plan_destroy(p);\n}\n')
+    inc = os.path.join(ROOT, "include")
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-I", inc, "-fsyntax-only", str(src)], check=True)
+    from paper_2609_20359_b200 import build
+    lib = build.build()
+    exe = tmp_path / "use_fls"
+    subprocess.run(["gcc", "-std=c99", "-I", inc, str(src), "-o", str(exe), lib, "-Wl,-rpath," + os.path.dirname(lib)], check=True)
+    out = subprocess.run([str(exe)], capture_output=True, text=True)
+    assert out.returncode == 0, out.stdout + out.stderr
+    assert out.stdout.split() == ["1024", "256", str(2 * 1024 * (4 * 2 + 34))]     # G * N_pad * (K*e_g + 34), K = 4 bf16
+
+
 def test_struct_sizes_match_header_layout(fls):
     # natural alignment of the C structs in include/fls.h
     assert ctypes.sizeof(fls.fls_plan_desc) == 8 + 8 + 8 + 10 * 4 + 6 * 8
