@@ -50,6 +50,7 @@ class Session:
         self.param_bf16 = [self._alloc(N, torch.bfloat16) for _ in range(self.n_copies)]
         self.workspace = self._alloc(self.layout["workspace_bytes"], torch.uint8, zero=False)
         self.speculative = speculative
+        self._cur = self._state            # where the state is now (speculative plans move it with every step)
         self._shadow = None
         if speculative:
             # the second buffer set that speculative steps write to; which set is current changes with every step
@@ -83,32 +84,37 @@ class Session:
         if grads is not None:
             self.grads = grads
         flat = [t for row in self.grads for t in row]
-        st = self._state
+        st = self._cur                     # the buffers that hold the state now are the ones to bind
         fls.fls_plan_bind(self.plan, flat, st["master"], st["m"], st["v"], self.param_bf16, self.workspace)
         if self._shadow is not None:
-            sh = self._shadow
-            fls.fls_plan_bind_shadow(self.plan, sh["master"], sh["m"], sh["v"])
+            both = {k: self._state[k] + self._shadow[k] for k in ("master", "m", "v")}
+            held = {k: {t.data_ptr() for t in st[k]} for k in both}
+            other = {k: [t for t in both[k] if t.data_ptr() not in held[k]] for k in both}
+            fls.fls_plan_bind_shadow(self.plan, other["master"], other["m"], other["v"])
             fls.fls_plan_set_speculative(self.plan, True)
 
-    def _current(self, which: str):
-        """The tensors that hold `which` ("master", "m", "v") of every state copy right now."""
+    def _refresh(self) -> None:
+        """After a step of a speculative plan: ask the library which buffer set holds the state now."""
         if self._shadow is None:
-            return self._state[which]
-        by_ptr = {t.data_ptr(): t for t in self._state[which] + self._shadow[which]}
-        i = ("master", "m", "v").index(which)
-        return [by_ptr[fls.fls_get_state(self.plan, c)[i]] for c in range(self.n_copies)]
+            return
+        ptrs = [fls.fls_get_state(self.plan, c) for c in range(self.n_copies)]
+        cur = {}
+        for i, k in enumerate(("master", "m", "v")):
+            by_ptr = {t.data_ptr(): t for t in self._state[k] + self._shadow[k]}
+            cur[k] = [by_ptr[p[i]] for p in ptrs]
+        self._cur = cur
 
     @property
     def master(self):
-        return self._current("master")
+        return self._cur["master"]
 
     @property
     def m(self):
-        return self._current("m")
+        return self._cur["m"]
 
     @property
     def v(self):
-        return self._current("v")
+        return self._cur["v"]
 
     def spec_stats(self):
         """(group-steps whose guess held, group-steps redone) of a speculative plan so far."""
@@ -117,14 +123,19 @@ class Session:
 
     # ------------------------------------------------------------------ calls
     def step(self, lr: float = math.nan, stream=None) -> bool:
-        return fls.fls_sync_step(self.plan, lr, stream)
+        due = fls.fls_sync_step(self.plan, lr, stream)
+        self._refresh()
+        return due
 
     def step_host(self, host_grads, lr: float = math.nan, stream=None, host_norms=None) -> bool:
         flat = [t for row in host_grads for t in row]
-        return fls.fls_sync_step_host(self.plan, flat, lr, stream, host_norms)
+        due = fls.fls_sync_step_host(self.plan, flat, lr, stream, host_norms)
+        self._refresh()
+        return due
 
     def step_fedavg(self, sample_counts=None, lr: float = math.nan, stream=None) -> None:
         fls.fls_sync_step_fedavg(self.plan, lr, sample_counts, stream)
+        self._refresh()
 
     def fedavg(self, sample_counts=None, stream=None) -> None:
         fls.fls_fedavg(self.plan, sample_counts, stream)

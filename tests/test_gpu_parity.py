@@ -592,18 +592,19 @@ def test_h1_equal_weights_equals_fsdp_over_all_replicas(fls):
     fl.close(); big.close()
 
 
-def test_determinism_and_resume(fls):
+@pytest.mark.parametrize("speculative", [False, True])
+def test_determinism_and_resume(fls, speculative):
     def run(split):
-        c = Case([50000, 1234], 2, 4, 1, H=2, Q=8, opt_state=True, hp=orc.Hyper(max_grad_norm=0.02))
-        for t in range(4):
-            if split and t == 2:       # checkpoint: a new plan over the same tensors, step counter restored
+        c = Case([50000, 1234], 2, 4, 1, H=2, Q=8, opt_state=True, hp=orc.Hyper(max_grad_norm=0.02), speculative=speculative)
+        for t in range(4 if not speculative else 5):
+            if split and t == (2 if not speculative else 3):       # checkpoint: a new plan over the same tensors, step counter restored
                 from paper_2609_20359_b200 import _binding as b
                 old = c.sess.plan
                 c.sess.plan = b.fls_plan_create(c.P, c.units, 2, 4, 1, 2, b.FLS_GRAD_BF16, 8, 3, c.hp.lr, c.hp.beta1, c.hp.beta2,
                                                 c.hp.eps, c.hp.weight_decay, c.hp.max_grad_norm)
                 b.fls_plan_destroy(old)
-                c.sess.bind()
-                b.fls_set_step(c.sess.plan, 2)
+                c.sess.bind()          # binds the buffers that hold the state now (after an odd number of speculative steps: the second set)
+                b.fls_set_step(c.sess.plan, 2 if not speculative else 3)
             c.step()
         out = [x.clone() for x in c.sess.master + c.sess.m + c.sess.v + c.sess.param_bf16]
         c.close()
@@ -674,9 +675,10 @@ def test_non_default_stream(fls):
     c.close()
 
 
-def test_step_from_host_buffers_matches_device_step(fls):
-    a = Case([50000, 777], 2, 2, 2, H=2, Q=8, hp=orc.Hyper(max_grad_norm=0.02))
-    b = Case([50000, 777], 2, 2, 2, H=2, Q=8, hp=orc.Hyper(max_grad_norm=0.02))
+@pytest.mark.parametrize("kw", [{}, {"speculative": True}, {"state_per_replica": True}], ids=["plain", "speculative", "replica_copies"])
+def test_step_from_host_buffers_matches_device_step(fls, kw):
+    a = Case([50000, 777], 2, 2, 2, H=2, Q=8, hp=orc.Hyper(max_grad_norm=0.02), **kw)
+    b = Case([50000, 777], 2, 2, 2, H=2, Q=8, hp=orc.Hyper(max_grad_norm=0.02), **kw)
     for t in range(1, 3):
         a.step()
         host = [[torch.from_numpy(orc.pack_unsharded(b.L, bf16_bits(b.grad_logical(t, g, k)).view(np.int16))).view(torch.bfloat16).pin_memory()
