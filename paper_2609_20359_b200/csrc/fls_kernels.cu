@@ -381,7 +381,8 @@ __device__ __noinline__ float reduce_slice_scalar(const ReduceArgs& a, uint64_t 
 //   counter) adds the warp sums in index order -> chunk of kNormChunk consecutive CTAs: the last CTA of the chunk
 //   to arrive (one global counter per chunk) adds the chunk's CTA partials in index order -> grid: the last chunk
 //   to arrive (the ticket) adds the chunk sums in index order, writes the group's norm and clip coefficient and
-//   re-arms the ticket; every chunk counter is re-armed by the warp that closes the chunk.
+//   re-arms the ticket; every chunk counter is re-armed by the warp that closes the chunk.  A grid of at most
+//   4 * kNormChunk CTAs forms a single chunk, whose closing warp finishes the job (one level less for small plans).
 // The caller must have zeroed *arrived (shared) behind a __syncthreads() at the start of the kernel.
 constexpr unsigned kNormChunk = kNormChunkCtas;
 
@@ -401,8 +402,10 @@ __device__ __forceinline__ void finish_norm(const ReduceArgs& a, float sq, unsig
   if (__shfl_sync(0xFFFFFFFFu, t, 0) != W - 1) return;
   __threadfence_block();
   const double cta = warp_sum(lane < W ? sh[lane] : 0.0);
-  const unsigned chunk = blockIdx.x / kNormChunk, n_chunks = (gridDim.x + kNormChunk - 1) / kNormChunk;
-  const unsigned chunk_size = min(kNormChunk, gridDim.x - chunk * kNormChunk);
+  // chunks of kNormChunk CTAs; a grid of up to 4 * kNormChunk CTAs is one chunk (one level less for small plans)
+  const unsigned per_chunk = gridDim.x <= 4 * kNormChunk ? gridDim.x : kNormChunk;
+  const unsigned chunk = blockIdx.x / per_chunk, n_chunks = (gridDim.x + per_chunk - 1) / per_chunk;
+  const unsigned chunk_size = min(per_chunk, gridDim.x - chunk * per_chunk);
   double* const partials = a.partials + size_t(y) * gridDim.x;
   double* const chunk_partials = a.chunk_partials + size_t(y) * a.tree_stride;
   uint32_t* const chunk_count = a.chunk_count + size_t(y) * a.tree_stride;
@@ -414,7 +417,7 @@ __device__ __forceinline__ void finish_norm(const ReduceArgs& a, float sq, unsig
   if (__shfl_sync(0xFFFFFFFFu, t, 0) != chunk_size - 1) return;
   __threadfence();
   double c = 0.0;
-  for (unsigned i = lane; i < chunk_size; i += 32) c += __ldcg(partials + size_t(chunk) * kNormChunk + i);
+  for (unsigned i = lane; i < chunk_size; i += 32) c += __ldcg(partials + size_t(chunk) * per_chunk + i);
   c = warp_sum(c);
   if (lane == 0) chunk_count[chunk] = 0u;     // ready for the next launch (stream order)
   double total = c;
