@@ -1,20 +1,28 @@
-// sm_100a kernels of libfls.  All three are HBM streams over 2048-element tiles; a group of 256
+// sm_100a kernels of libfls.  All of them are HBM streams over 2048-element tiles; a group of 256
 // threads owns a tile, a thread owns 8 consecutive elements of it and moves them with 128-bit (bf16)
 // and 256-bit (fp32) global accesses.  By default the grid covers the whole buffer in one pass (no
 // grid-stride loop): the hardware scheduler hands out CTAs in order, so the tiles in flight form a
 // compact window that moves through memory and the SMs stay balanced, which measured 5-15 % faster
-// than persistent grid-stride CTAs.  The kernels are kept small in registers (32-72) so that 768-2048
+// than persistent grid-stride CTAs.  The kernels are kept small in registers (32-80) so that 768-2048
 // threads are resident per SM; that, not unrolling, is what keeps enough loads in flight.
 // No shared-memory staging and no tensor cores: nothing here is a contraction, and each byte is touched
 // once.
 //
-//   fls_reduce_kernel  : K gradient buffers -> mean gradient (fp32, shard order) + squared-norm partials,
-//                        added up over a fixed tree (warp, CTA, chunk of CTAs, grid) by whoever arrives last
-//                        at each level; the last of all writes the group's norm and clip coefficient (no
-//                        floating-point atomics, no block-wide barrier: the result does not depend on the
-//                        order of arrival).
-//   fls_adamw_kernel   : clip + AdamW on master/m/v in place + bf16 copy in unsharded order.
-//   fls_fedavg_kernel  : weighted average of G copies written back to all G (+ bf16 copies).
+//   fls_reduce_kernel       : K gradient buffers -> mean gradient (fp32, shard order) + squared-norm partials,
+//                             added up over a fixed tree (warp, CTA, chunk of CTAs, grid) by whoever arrives
+//                             last at each level; the last of all writes the group's norm and clip coefficient
+//                             (no floating-point atomics, no block-wide barrier: the result does not depend on
+//                             the order of arrival).  Also the norm-only pass of the recompute route, and, with
+//                             the group in blockIdx.y, the reduction of all groups of a small plan at once.
+//   fls_adamw_kernel        : clip + AdamW on master/m/v in place + bf16 copy in unsharded order
+//                             (fls_adamw_batch_kernel: all groups of a small plan in one grid).
+//   fls_reduce_adamw_kernel : AdamW that forms the mean gradient itself (recompute route; redo kernel of a
+//                             speculative step).
+//   fls_step_noclip_kernel  : reduce + norm + AdamW in one pass (plans without clipping; first kernel of a
+//                             speculative step).
+//   fls_fedavg_kernel       : weighted average of G copies written back to all copies (+ bf16 copies), optionally
+//                             through an outer SGD step on a global copy.
+//   fls_adamw_fedavg_kernel : AdamW of every group and FedAvg of the results in one pass (aggregation steps).
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
