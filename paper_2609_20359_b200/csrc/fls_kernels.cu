@@ -32,8 +32,8 @@ namespace fls {
 namespace {
 
 // ------------------------------------------------------------------------------------------------
-// Global-memory accessors.  "stream": data touched once (evict-first, no L1 allocation).
-// "keep": the reduced gradient, written by one kernel and read back by the next.
+// Global-memory accessors.  "stream": data touched once, or for the last time (evict-first, no L1 allocation).
+// "keep": stores of the part of the reduced gradient that the next kernel reads first.
 // ------------------------------------------------------------------------------------------------
 struct alignas(32) F8 { float v[8]; };
 
@@ -43,14 +43,6 @@ struct alignas(32) F8 { float v[8]; };
 __device__ __forceinline__ F8 ld8_stream(const float* p) {
   uint32_t u[8];
   asm volatile("ld.global.L1::no_allocate.L2::evict_first.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];" : FLS_O8(u) : "l"(p));
-  F8 r;
-#pragma unroll
-  for (int e = 0; e < 8; ++e) r.v[e] = __uint_as_float(u[e]);
-  return r;
-}
-__device__ __forceinline__ F8 ld8_keep(const float* p) {
-  uint32_t u[8];
-  asm volatile("ld.global.L1::no_allocate.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];" : FLS_O8(u) : "l"(p));
   F8 r;
 #pragma unroll
   for (int e = 0; e < 8; ++e) r.v[e] = __uint_as_float(u[e]);
@@ -599,7 +591,7 @@ __device__ __forceinline__ void adamw_tiles(const A& a, float* theta, float* m_,
       F8 m = ld8_stream(m_ + s.a);
       F8 v = ld8_stream(v_ + s.a);
       if (!waited) { dep_wait(); dep_launch(); c = __ldcg(coef); waited = true; }
-      const F8 g = ld8_keep(gbar + s.a);
+      const F8 g = ld8_stream(gbar + s.a);      // last use: evict-first also releases the lines K1 stored "evict last"
 #pragma unroll
       for (int e = 0; e < 8; ++e) adamw_one(a, c, g.v[e], th.v[e], m.v[e], v.v[e]);
       st8_stream(theta + s.a, th);
@@ -905,7 +897,7 @@ __global__ void __launch_bounds__(kThreads, FLS_FUSED_MINB) fls_adamw_fedavg_ker
         F8 m = ld8_stream(a.m[g] + s.a);
         F8 v = ld8_stream(a.v[g] + s.a);
         if (!waited) { dep_wait(); dep_launch(); waited = true; }
-        const F8 gb = ld8_keep(a.gbar[g] + s.a);
+        const F8 gb = ld8_stream(a.gbar[g] + s.a);
         const float c = __ldcg(a.coefs + g), wg = a.w[g];
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
