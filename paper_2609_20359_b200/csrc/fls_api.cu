@@ -196,6 +196,34 @@ void set_adam_scalars(AdamArgs* aa, const AdamScalars& sc) {
   aa->step_size = sc.step_size; aa->inv_sqrt_bc2 = sc.inv_sqrt_bc2; aa->eps = sc.eps;
 }
 
+// The part of the reduce kernel's arguments that does not depend on the group.
+ReduceArgs common_reduce_args(const fls_plan* p) {
+  const fls_plan_desc& d = p->desc;
+  ReduceArgs ra{};
+  ra.idx = p->seg_index();
+  ra.K = p->K;
+  ra.k_float = float(p->K);
+  ra.inv_k = 1.0f / float(p->K);
+  ra.k_is_pow2 = (p->K & (p->K - 1)) == 0 ? 1u : 0u;
+  ra.fold_mask = p->fold_mask;
+  ra.end_mask = p->end_mask;
+  ra.status = p->d_status();
+  ra.max_grad_norm = d.max_grad_norm;
+  ra.ring = p->ring ? 1u : 0u;
+  ra.S = d.shard_dim;
+  ra.R = d.replicate_dim;
+  ra.spec_counts = nullptr;
+  ra.gbar_stride = p->lay.scratch_stride / 4;
+  ra.tree_stride = uint32_t(p->lay.n_chunks);
+  return ra;
+}
+
+// Tiles from which on the reduced gradient is stored "evict last": the AdamW kernel walks it from its end.
+uint32_t keep_from_tile(const fls_plan* p, bool reader_descends) {
+  const uint64_t keep_tiles = std::min<uint64_t>(p->lay.n_tiles, p->l2_keep_bytes / (uint64_t(kTile) * 4));
+  return reader_descends ? uint32_t(p->lay.n_tiles - keep_tiles) : uint32_t(p->lay.n_tiles);
+}
+
 // One group's reduce (+ AdamW) launches.  chain: the previous operation on `st` is a kernel of this same call,
 // so this group's first kernel may overlap its tail.  slot: which reduced-gradient buffer of the workspace
 // receives the mean gradient; with_adamw = false stops after the reduction (the fused aggregation applies AdamW
@@ -204,17 +232,10 @@ int run_group(fls_plan* p, uint32_t g, double lr, uint64_t t_new, cudaStream_t s
               bool with_adamw = true) {
   const fls_plan_desc& d = p->desc;
   const uint32_t c0 = g * p->R_state;      // the group's first state copy
-  ReduceArgs ra{};
+  ReduceArgs ra = common_reduce_args(p);
   for (uint32_t k = 0; k < p->K; ++k) ra.grad[k] = p->grads[size_t(g) * p->K + k];
   ra.gbar = p->d_gbar(slot);
   p->last_slot = slot;
-  ra.idx = p->seg_index();
-  ra.K = p->K;
-  ra.k_float = float(p->K);
-  ra.inv_k = 1.0f / float(p->K);
-  ra.k_is_pow2 = (p->K & (p->K - 1)) == 0 ? 1u : 0u;
-  ra.fold_mask = p->fold_mask;
-  ra.end_mask = p->end_mask;
   ra.partials = p->d_partials() + size_t(g) * p->lay.n_tiles;
   ra.chunk_partials = p->d_chunk_partials() + size_t(g) * p->lay.n_chunks;
   ra.chunk_count = p->d_chunk_count() + size_t(g) * p->lay.n_chunks;
@@ -222,15 +243,9 @@ int run_group(fls_plan* p, uint32_t g, double lr, uint64_t t_new, cudaStream_t s
   ra.norm_out = p->d_norms() + g;
   ra.coef_out = p->d_coefs() + g;
   ra.normsq_out = p->d_normsq() + g;
-  ra.status = p->d_status();
-  ra.max_grad_norm = d.max_grad_norm;
-  ra.ring = p->ring ? 1u : 0u;
-  ra.S = d.shard_dim;
-  ra.R = d.replicate_dim;
-  ra.spec_counts = nullptr;
-  // the AdamW kernel walks the reduced gradient from its end: keep that end in L2, stream the rest
-  const uint64_t keep_tiles = std::min<uint64_t>(p->lay.n_tiles, p->l2_keep_bytes / (uint64_t(kTile) * 4));
-  ra.keep_from_tile = with_adamw && p->descending[FLS_KERNEL_ADAMW] ? uint32_t(p->lay.n_tiles - keep_tiles) : uint32_t(p->lay.n_tiles);
+  // keep the end of the reduced gradient in L2 for the AdamW kernel, stream the rest; before a fused aggregation nothing
+  // is kept (that kernel reads G reduced gradients: keeping their ends measured slower)
+  ra.keep_from_tile = keep_from_tile(p, with_adamw && p->descending[FLS_KERNEL_ADAMW]);
   const bool speculate = p->speculative && with_adamw;
   const bool single = (p->single_pass || speculate) && with_adamw;
   const bool recompute = p->recompute && with_adamw && !single;   // the fused aggregation needs the stored gradients
@@ -308,20 +323,11 @@ int run_group(fls_plan* p, uint32_t g, double lr, uint64_t t_new, cudaStream_t s
 int run_groups_batched(fls_plan* p, double lr, uint64_t t_new, cudaStream_t st, bool with_adamw) {
   const fls_plan_desc& d = p->desc;
   const uint32_t G = d.groups;
-  ReduceArgs ra{};
+  ReduceArgs ra = common_reduce_args(p);
   for (uint32_t i = 0; i < G * p->K; ++i) ra.grad[i] = p->grads[i];
   ra.gbar = p->d_gbar(0);
-  ra.gbar_stride = p->lay.scratch_stride / 4;
-  ra.tree_stride = uint32_t(p->lay.n_chunks);
   p->last_slot = G - 1;
   p->gbar_valid = true;
-  ra.idx = p->seg_index();
-  ra.K = p->K;
-  ra.k_float = float(p->K);
-  ra.inv_k = 1.0f / float(p->K);
-  ra.k_is_pow2 = 1u;                       // K is 4 or 8 here
-  ra.fold_mask = p->fold_mask;
-  ra.end_mask = p->end_mask;
   ra.partials = p->d_partials();
   ra.chunk_partials = p->d_chunk_partials();
   ra.chunk_count = p->d_chunk_count();
@@ -329,12 +335,7 @@ int run_groups_batched(fls_plan* p, double lr, uint64_t t_new, cudaStream_t st, 
   ra.norm_out = p->d_norms();
   ra.coef_out = p->d_coefs();
   ra.normsq_out = p->d_normsq();
-  ra.status = p->d_status();
-  ra.max_grad_norm = d.max_grad_norm;
-  ra.S = d.shard_dim;
-  ra.R = d.replicate_dim;
-  const uint64_t keep_tiles = std::min<uint64_t>(p->lay.n_tiles, p->l2_keep_bytes / (uint64_t(kTile) * 4));
-  ra.keep_from_tile = uint32_t(p->lay.n_tiles - keep_tiles);
+  ra.keep_from_tile = keep_from_tile(p, true);      // small plans: everything fits in L2 anyway
   ra.store_gbar = 1;
   const bool f32 = d.grad_dtype == FLS_GRAD_F32;
   const bool overlap = p->overlap && !p->profiling;
