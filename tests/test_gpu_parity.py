@@ -412,6 +412,7 @@ def test_fused_step_fedavg_matches_oracle_and_unfused(fls, units, G, S, R_rep, Q
     ([30000, 517], 16, 2, 3, 8, "bf16", False, True),    # 32 extra copies: the most the fused kernel serves
     ([30000, 517], 16, 2, 4, 8, "bf16", True, True),     # 48 extra copies: the fused call falls back to step + FedAvg
     ([17], 2, 2, 2, 1, "bf16", True, True),
+    ([999, 40], 32, 1, 2, 8, "bf16", True, False),       # 64 state copies: the most a plan may hold
 ])
 def test_state_copy_per_replica(fls, units, G, S, R_rep, Q, dtype, opt_state, fused):
     """FLS_STATE_PER_REPLICA: G*R_rep state copies.  Every replica of a group applies the group's mean gradient to
