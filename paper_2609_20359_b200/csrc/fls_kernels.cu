@@ -217,15 +217,26 @@ __device__ __forceinline__ uint32_t ring_buffer(const ReduceArgs& a, uint32_t sc
   return rho * a.S + sigma;
 }
 
+// Accumulator of the sums.  bf16 gradients are added in fp32: their 8-bit significands leave 16 spare bits, so
+// the running sums are exact unless the addends span more than 16 binades.  fp32 gradients are added in double and
+// rounded to fp32 once, after the scaling: an fp32 running sum of fp32 addends rounds at every step, by up to
+// 2^-24 of the LARGEST addend, and where the addends cancel that error is large relative to the mean -- AdamW
+// divides by sqrt(v)+eps, so a mean of 1e-9 that is off by 1e-10 moves theta by more than the parity tolerance.
+template <bool F32> struct AccOf { using type = float; };
+template <> struct AccOf<true> { using type = double; };
+
 // one scaling by 1/K after the last level: a multiply when 1/K is exact, else an IEEE division
-template <int N>
-__device__ __forceinline__ void scale_mean(const ReduceArgs& a, const float (&outer)[N], float (&mean)[N]) {
+template <int N, typename A>
+__device__ __forceinline__ void scale_mean(const ReduceArgs& a, const A (&outer)[N], float (&mean)[N]) {
   if (a.k_is_pow2) {
 #pragma unroll
-    for (int e = 0; e < N; ++e) mean[e] = outer[e] * a.inv_k;
+    for (int e = 0; e < N; ++e) mean[e] = float(outer[e] * A(a.inv_k));
   } else {
 #pragma unroll
-    for (int e = 0; e < N; ++e) mean[e] = __fdiv_rn(outer[e], a.k_float);
+    for (int e = 0; e < N; ++e) {
+      if constexpr (sizeof(A) == 8) mean[e] = float(__ddiv_rn(outer[e], double(a.k_float)));
+      else mean[e] = __fdiv_rn(outer[e], a.k_float);
+    }
   }
 }
 
@@ -233,13 +244,14 @@ __device__ __forceinline__ void scale_mean(const ReduceArgs& a, const float (&ou
 template <int N, bool F32, int KT, int SG>
 __device__ __forceinline__ void combine_loaded(const ReduceArgs& a, const Raw<N, F32> (&raw)[KT], float (&mean)[N]) {
   static_assert(KT > 0 && SG >= 0, "static shapes only");
-  float outer[N];
+  using A = typename AccOf<F32>::type;
+  A outer[N];
 #pragma unroll
-  for (int e = 0; e < N; ++e) outer[e] = 0.f;
+  for (int e = 0; e < N; ++e) outer[e] = A(0);
   if constexpr (SG == 0) {
-    float inner[N];
+    A inner[N];
 #pragma unroll
-    for (int e = 0; e < N; ++e) inner[e] = 0.f;
+    for (int e = 0; e < N; ++e) inner[e] = A(0);
 #pragma unroll
     for (int b = 0; b < KT; ++b) {
       float x[N];
@@ -252,8 +264,13 @@ __device__ __forceinline__ void combine_loaded(const ReduceArgs& a, const Raw<N,
   } else {
 #pragma unroll
     for (int g0 = 0; g0 < KT; g0 += SG) {
-      float s[N];
-      unpack(raw[g0], s);
+      A s[N];
+      {
+        float x[N];
+        unpack(raw[g0], x);
+#pragma unroll
+        for (int e = 0; e < N; ++e) s[e] = x[e];
+      }
 #pragma unroll
       for (int i = 1; i < SG; ++i) {
         float x[N];
@@ -265,7 +282,7 @@ __device__ __forceinline__ void combine_loaded(const ReduceArgs& a, const Raw<N,
       for (int e = 0; e < N; ++e) outer[e] += s[e];
     }
   }
-  scale_mean<N>(a, outer, mean);
+  scale_mean<N, A>(a, outer, mean);
 }
 
 // gk0: index of the group's first buffer in a.grad (0 except in a batched launch).
@@ -278,10 +295,11 @@ __device__ __forceinline__ void reduce_elems(const ReduceArgs& a, uint64_t j, fl
     combine_loaded<N, F32, KT, SG>(a, raw, mean);
   } else {
     // run-time K: batches of 8 buffers
+    using A = typename AccOf<F32>::type;
     const uint32_t K = a.K;
-    float inner[N], outer[N];
+    A inner[N], outer[N];
 #pragma unroll
-    for (int e = 0; e < N; ++e) inner[e] = outer[e] = 0.f;
+    for (int e = 0; e < N; ++e) inner[e] = outer[e] = A(0);
 #pragma unroll 1
     for (uint32_t k0 = 0; k0 < K; k0 += 8) {
       Raw<N, F32> raw[8];
@@ -306,14 +324,19 @@ __device__ __forceinline__ void reduce_elems(const ReduceArgs& a, uint64_t j, fl
         }
         if ((a.fold_mask >> (k0 >> 3)) & 1u) {
 #pragma unroll
-          for (int e = 0; e < N; ++e) { outer[e] += inner[e]; inner[e] = 0.f; }
+          for (int e = 0; e < N; ++e) { outer[e] += inner[e]; inner[e] = A(0); }
         }
       } else if constexpr (SG > 0) {
 #pragma unroll
         for (int g0 = 0; g0 < 8; g0 += SG) {
           if (k0 + g0 < K) {
-            float s[N];
-            unpack(raw[g0], s);
+            A s[N];
+            {
+              float x[N];
+              unpack(raw[g0], x);
+#pragma unroll
+              for (int e = 0; e < N; ++e) s[e] = x[e];
+            }
 #pragma unroll
             for (int i = 1; i < SG; ++i) {
               float x[N];
@@ -333,16 +356,16 @@ __device__ __forceinline__ void reduce_elems(const ReduceArgs& a, uint64_t j, fl
             float x[N];
             unpack(raw[b], x);
 #pragma unroll
-            for (int e = 0; e < N; ++e) inner[e] = (SG == -2) ? round_bf16(inner[e] + x[e]) : inner[e] + x[e];
+            for (int e = 0; e < N; ++e) inner[e] = (SG == -2) ? A(round_bf16(float(inner[e] + x[e]))) : inner[e] + x[e];
             if ((a.end_mask >> k) & 1ull) {
 #pragma unroll
-              for (int e = 0; e < N; ++e) { outer[e] = (SG == -2) ? round_bf16(outer[e] + inner[e]) : outer[e] + inner[e]; inner[e] = 0.f; }
+              for (int e = 0; e < N; ++e) { outer[e] = (SG == -2) ? A(round_bf16(float(outer[e] + inner[e]))) : outer[e] + inner[e]; inner[e] = A(0); }
             }
           }
         }
       }
     }
-    scale_mean<N>(a, outer, mean);
+    scale_mean<N, A>(a, outer, mean);
     if constexpr (SG == -2) {
 #pragma unroll
       for (int e = 0; e < N; ++e) mean[e] = round_bf16(mean[e]);
@@ -648,7 +671,7 @@ __device__ __noinline__ void reduce_adamw_slice_scalar(const ReduceAdamArgs& p, 
 // kernel has nothing to do; otherwise it redoes the step with the real coefficient, reading the same (untouched)
 // input state and overwriting the same output buffers.
 template <bool F32, int KT, int SG>
-__global__ void __launch_bounds__(kThreads, KT == 0 ? 2 : 4) fls_reduce_adamw_kernel(const __grid_constant__ ReduceAdamArgs p) {
+__global__ void __launch_bounds__(kThreads, KT == 0 ? 2 : (F32 ? 3 : 4)) fls_reduce_adamw_kernel(const __grid_constant__ ReduceAdamArgs p) {
   const AdamArgs& a = p.a;
   const uint32_t n_tiles = a.idx.n_tiles;
   if (blockIdx.x >= n_tiles) { dep_wait(); dep_launch(); return; }
@@ -697,7 +720,7 @@ __global__ void __launch_bounds__(kThreads, KT == 0 ? 2 : 4) fls_reduce_adamw_ke
 // (4 CTAs per SM measured best for a static K: 2 and 3 leave loads in flight on the table, 5 and 6 spill; the
 // run-time-K form holds a batch of eight raw loads next to the state and needs the registers of 2 CTAs per SM)
 template <bool F32, int KT, int SG>
-__global__ void __launch_bounds__(kThreads, KT == 0 ? 2 : 4) fls_step_noclip_kernel(const __grid_constant__ ReduceAdamArgs p) {
+__global__ void __launch_bounds__(kThreads, KT == 0 ? 2 : (F32 ? 3 : 4)) fls_step_noclip_kernel(const __grid_constant__ ReduceAdamArgs p) {
   const AdamArgs& a = p.a;
   __shared__ unsigned arrived;
   begin_norm(&arrived);
@@ -946,6 +969,8 @@ __global__ void __launch_bounds__(kThreads, FLS_FUSED_MINB) fls_adamw_fedavg_ker
 #endif
 constexpr int kFlatThreads = FLS_FLAT_THREADS, kFlatMinB = FLS_FLAT_MINB;       // SG == 0 with a static K
 constexpr int kLevelThreads = FLS_LEVEL_THREADS, kLevelMinB = FLS_LEVEL_MINB;   // two-level orders with a static K
+// fp32 gradients: double accumulators (twice the registers) and 32-byte loads, so fewer resident CTAs
+constexpr int kFlatMinB32 = 5, kLevelMinB32 = 4;
 constexpr int kAnyThreads = 256, kAnyMinB = 2;         // run-time K: batches of 8 loads need the registers
 #ifndef FLS_FEW_THREADS
 #define FLS_FEW_THREADS 256
@@ -987,9 +1012,9 @@ void launch_reduce_shape(const ReduceArgs& a, unsigned grid, cudaStream_t st, bo
   else if constexpr (KT <= 2)
     launch_k(fls_reduce_kernel<F32, KT, SG, kFewThreads, kFewMinB, tiles_per_thread<F32, KT>()>, a, grid, kFewThreads, st, ov);
   else if constexpr (SG == 0)
-    launch_k(fls_reduce_kernel<F32, KT, SG, kFlatThreads, kFlatMinB, 1>, a, grid, kFlatThreads, st, ov);
+    launch_k(fls_reduce_kernel<F32, KT, SG, kFlatThreads, F32 ? kFlatMinB32 : kFlatMinB, 1>, a, grid, kFlatThreads, st, ov);
   else
-    launch_k(fls_reduce_kernel<F32, KT, SG, kLevelThreads, kLevelMinB, 1>, a, grid, kLevelThreads, st, ov);
+    launch_k(fls_reduce_kernel<F32, KT, SG, kLevelThreads, F32 ? kLevelMinB32 : kLevelMinB, 1>, a, grid, kLevelThreads, st, ov);
 }
 
 template <bool F32, int KT>
@@ -1043,9 +1068,9 @@ void launch_k2(void (*kernel)(Args), const Args& a, unsigned grid_x, unsigned gr
 template <bool F32, int KT, int SG>
 void launch_reduce_batch_shape(const ReduceArgs& a, unsigned grid, unsigned groups, cudaStream_t st, bool ov) {
   if constexpr (SG == 0)
-    launch_k2(fls_reduce_kernel<F32, KT, SG, kFlatThreads, kFlatMinB, 1, true>, a, grid, groups, kFlatThreads, st, ov);
+    launch_k2(fls_reduce_kernel<F32, KT, SG, kFlatThreads, F32 ? kFlatMinB32 : kFlatMinB, 1, true>, a, grid, groups, kFlatThreads, st, ov);
   else
-    launch_k2(fls_reduce_kernel<F32, KT, SG, kLevelThreads, kLevelMinB, 1, true>, a, grid, groups, kLevelThreads, st, ov);
+    launch_k2(fls_reduce_kernel<F32, KT, SG, kLevelThreads, F32 ? kLevelMinB32 : kLevelMinB, 1, true>, a, grid, groups, kLevelThreads, st, ov);
 }
 
 template <bool F32>

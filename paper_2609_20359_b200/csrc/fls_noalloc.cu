@@ -11,6 +11,7 @@
 // must start at zero, the ticket counter, is cleared on the caller's stream before every launch; the
 // partials are fully rewritten before they are read.  Two calls that overlap on the GPU (different
 // streams, or different host threads on the same device) race on the array: serialise them.
+#include <type_traits>
 #include <cuda_runtime.h>
 
 #include <algorithm>
@@ -76,13 +77,16 @@ __device__ __forceinline__ float load1(const void* base, uint64_t j) {
   return __uint_as_float(uint32_t(static_cast<const uint16_t*>(base)[j]) << 16);
 }
 
-// Same order as the plan-based kernel: ascending buffers inside a sharding group, groups folded in
-// ascending replica order, both levels starting from zero, one scaling by 1/K at the end.
+// Same order and precision as the plan-based kernel: ascending buffers inside a sharding group, groups folded in
+// ascending replica order, both levels starting from zero, one scaling by 1/K at the end.  bf16 gradients are added
+// in fp32 (exact unless the addends span more than 16 binades); fp32 gradients are added in double and rounded to
+// fp32 once, so that a mean that nearly cancels keeps its leading bits.
 template <bool F32, int N>
 __device__ __forceinline__ void mean_of(const Args& a, uint64_t j, float (&mean)[N]) {
-  float inner[N], outer[N];
+  using A = typename std::conditional<F32, double, float>::type;
+  A inner[N], outer[N];
 #pragma unroll
-  for (int e = 0; e < N; ++e) inner[e] = outer[e] = 0.f;
+  for (int e = 0; e < N; ++e) inner[e] = outer[e] = A(0);
   for (uint32_t k = 0; k < a.K; ++k) {
     float x[N];
     if constexpr (N == 8) load8<F32>(a.grad[k], j, x); else x[0] = load1<F32>(a.grad[k], j);
@@ -90,11 +94,14 @@ __device__ __forceinline__ void mean_of(const Args& a, uint64_t j, float (&mean)
     for (int e = 0; e < N; ++e) inner[e] += x[e];
     if ((a.end_mask >> k) & 1ull) {
 #pragma unroll
-      for (int e = 0; e < N; ++e) { outer[e] += inner[e]; inner[e] = 0.f; }
+      for (int e = 0; e < N; ++e) { outer[e] += inner[e]; inner[e] = A(0); }
     }
   }
 #pragma unroll
-  for (int e = 0; e < N; ++e) mean[e] = a.k_is_pow2 ? outer[e] * a.inv_k : __fdiv_rn(outer[e], a.k_float);
+  for (int e = 0; e < N; ++e) {
+    if constexpr (F32) mean[e] = float(a.k_is_pow2 ? outer[e] * double(a.inv_k) : __ddiv_rn(outer[e], double(a.k_float)));
+    else mean[e] = a.k_is_pow2 ? outer[e] * a.inv_k : __fdiv_rn(outer[e], a.k_float);
+  }
 }
 
 __device__ __forceinline__ double block_sum(double x, double* sh) {

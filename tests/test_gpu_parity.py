@@ -270,8 +270,9 @@ def test_bf16_wire_orders_differ_on_the_gpu_too(fls):
 ])
 def test_ring_order_reduction(fls, units, G, S, R_rep, Q, dtype, wire):
     """reduce_order = FLS_ORDER_RING: every rank's slice is summed starting on the next rank, every all-reduce
-    sub-chunk starting on the next replica.  With bf16 partial sums the reduced gradient is bit-identical to the
-    oracle's; with fp32 partial sums it equals the exactly rounded mean up to the rounding of the fp32 adds."""
+    sub-chunk starting on the next replica.  With bf16 partial sums, and with fp32 gradients (double partial sums),
+    the reduced gradient is bit-identical to the oracle's; with bf16 gradients and fp32 partial sums it equals the
+    exactly rounded mean up to the rounding of the fp32 adds."""
     hp = orc.Hyper(max_grad_norm=0.05, wire_bf16=wire, ring=True)
     c = Case(units, G, S, R_rep, H=2, Q=Q, grad_dtype=dtype, hp=hp, per_buffer_scale=True)
     for t in range(1, 3):
@@ -279,7 +280,7 @@ def test_ring_order_reduction(fls, units, G, S, R_rep, Q, dtype, wire):
         want = orc.pack_sharded(c.L, orc.reduce_mean(grads[G - 1], S, R_rep, wire_bf16=wire, ring=c.ring))
         c.step()
         got = c.sess.reduced_grad().cpu().numpy()
-        if wire:
+        if wire or dtype == "f32":
             assert np.array_equal(got, want)
         else:
             bound = orc.pack_sharded(c.L, 2.0 ** -24 * np.sum(np.abs(grads[G - 1]), axis=0))
@@ -311,28 +312,58 @@ def test_ring_start_changes_bf16_sums_and_not_fp32_sums(fls):
     assert torch.equal(res[(True, 8, False)][7 * M:], res[(True, 8, True)][7 * M:])
 
 
-def test_two_level_order_differs_from_flat_where_fp32_rounds(fls):
-    """fp32 gradients spanning many binades: the shard-then-replicate order and the flat order round
-    differently; each matches the oracle run in the same order (to fp32 rounding of the sum)."""
-    units, P = [4096], 4096
+def _fp32_running_mean(grads, S, R_rep):
+    """What an fp32 accumulator would give (shard level, then replicate level, one division): NOT what the library does."""
+    outer = np.zeros(grads[0].shape, np.float32)
+    for rho in range(R_rep):
+        inner = np.zeros(grads[0].shape, np.float32)
+        for sigma in range(S):
+            inner = inner + grads[rho * S + sigma].astype(np.float32)
+        outer = outer + inner
+    return outer / np.float32(S * R_rep)
+
+
+@pytest.mark.parametrize("S,R_rep", [(8, 1), (4, 2), (3, 2), (1, 5)])
+def test_fp32_gradients_are_summed_in_double(fls, S, R_rep):
+    """fp32 gradients spanning many binades: the mean gradient is the oracle's bit for bit (double partial sums in
+    the same order, one rounding to fp32), where an fp32 running sum would differ in many elements."""
+    units, P = [4096, 7], 4103
     def big(t, g, k):
         x = sy.normal_fill_(torch.empty(P), sy.stream_key(9, sy.KIND_GRAD, t, g, k), 1.0)
         return x * (10.0 ** (k % 4 * 2))
-    res = {}
-    for (S, R_rep) in ((8, 1), (4, 2)):
-        c = Case(units, 1, S, R_rep, H=10, Q=8, grad_dtype="f32", hp=orc.Hyper(max_grad_norm=0.0))
-        fls.fls_plan_set_single_pass(c.sess.plan, 0)          # two passes, so that the mean gradient is stored
-        grads = c.load_grads(1, big)
-        c.sess.step()
-        torch.cuda.synchronize()
-        got = c.sess.reduced_grad().cpu().numpy()
-        want = orc.reduce_mean(grads[0], S, R_rep)
-        # sequential fp32 adds: each of the K-1 roundings is at most half an ulp of a partial sum <= sum|x|
-        bound = S * R_rep * 2.0 ** -24 * np.sum(np.abs(grads[0]), axis=0) / (S * R_rep)
-        assert np.all(np.abs(got.astype(np.float64) - want) <= bound)
-        res[(S, R_rep)] = got
-        c.close()
-    assert not np.array_equal(res[(8, 1)], res[(4, 2)])
+    c = Case(units, 1, S, R_rep, H=10, Q=8, grad_dtype="f32", hp=orc.Hyper(max_grad_norm=0.0))
+    fls.fls_plan_set_single_pass(c.sess.plan, 0)          # two passes, so that the mean gradient is stored
+    grads = c.load_grads(1, big)
+    c.sess.step()
+    torch.cuda.synchronize()
+    got = orc.unpack_sharded(c.L, c.sess.reduced_grad().cpu().numpy())
+    want = orc.reduce_mean(grads[0], S, R_rep)
+    assert np.array_equal(got, want)
+    assert np.mean(_fp32_running_mean(grads[0], S, R_rep) != want) > 0.1      # the inputs do tell the two apart
+    c.close()
+
+
+@pytest.mark.parametrize("S,R_rep,fused,spec,clip", [(2, 3, False, False, 0.0), (8, 1, True, False, 1e-7), (4, 1, False, True, 1e-7),
+                                                     (5, 1, False, False, 1e-7), (4, 2, False, True, 1.0)])
+def test_fp32_gradients_that_cancel(fls, S, R_rep, fused, spec, clip):
+    """fp32 gradients whose mean nearly cancels (|mean| around AdamW's eps = 1e-8, addends around 1e-3).  The update
+    divides by sqrt(v) + eps, so an error of 1e-10 in such a mean moves theta by 1e-6 and more: the state stays within
+    the tolerance only because the partial sums are kept in double.  Three steps, with and without clipping."""
+    K, P = S * R_rep, 2048 + 17
+    def cancelling(t, g, k):
+        if k < K - 1:
+            return sy.normal_fill_(torch.empty(P), sy.stream_key(77, sy.KIND_GRAD, t, g, k), 1e-3)
+        rest = sum(cancelling(t, g, i).double() for i in range(K - 1))
+        tiny = sy.normal_fill_(torch.empty(P), sy.stream_key(78, sy.KIND_GRAD, t, g, k), 1e-8).double()
+        return (tiny * K - rest).float()              # the fp32 rounding of this buffer leaves a mean of about 1e-8
+    c = Case([17, 2048], 2, S, R_rep, H=3, Q=8, grad_dtype="f32", hp=orc.Hyper(max_grad_norm=clip), fused=fused, speculative=spec)
+    grads = c.load_grads(1, cancelling)
+    gbar = orc.reduce_mean(grads[0], S, R_rep)
+    assert np.median(np.abs(gbar)) < 1e-7 and np.mean(_fp32_running_mean(grads[0], S, R_rep) != gbar) > 0.5
+    for _ in range(3):
+        c.step(override=cancelling)
+        c.compare()
+    c.close()
 
 
 def _sweep_shapes():

@@ -272,6 +272,25 @@ def test_reduce_special_cases():
     assert lvl[0] == 0.0 and flt[0] == np.float32(2.0 ** -60 / 4)
 
 
+def test_reduce_mean_of_fp32_inputs_that_cancel_is_the_exactly_rounded_mean():
+    """fp32 inputs around 1e-3 whose mean is around 1e-8: the result is the exact rational mean rounded once to fp32
+    (an fp32 running sum is off by a large fraction of such a mean, which AdamW's division by sqrt(v)+eps would amplify)."""
+    rng = np.random.default_rng(41)
+    for S, R_rep in ((2, 3), (8, 1), (5, 1)):
+        K = S * R_rep
+        x = [rng.normal(0, 1e-3, 64).astype(np.float32) for _ in range(K - 1)]
+        x.append((rng.normal(0, 1e-8, 64) * K - np.sum([a.astype(np.float64) for a in x], axis=0)).astype(np.float32))
+        got = orc.reduce_mean([a.astype(np.float64) for a in x], S, R_rep)
+        running = np.zeros(64, np.float32)
+        for a in x:
+            running = running + a
+        running = running / np.float32(K)
+        for j in range(64):
+            exact = sum(Fraction(float(a[j])) for a in x) / K
+            assert got[j] == f32_of_fraction(exact), (S, R_rep, j)
+        assert np.median(np.abs(got)) < 1e-7 and np.mean(running != got) > 0.5
+
+
 # ----------------------------------------------------------------------------- norm and clip
 def test_norm_closed_forms():
     a = np.float32(0.00390625)                                     # 2^-8, exact
