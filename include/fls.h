@@ -73,7 +73,9 @@ typedef struct {
   uint32_t fedavg_what;       /* FLS_AVG_PARAMS, optionally | FLS_AVG_OPT_STATE (m and v averaged too),
                                  optionally | FLS_AVG_FUSED (workspace holds one reduced gradient per group
                                  so that fls_sync_step_fedavg can fuse the aggregation into the step)      */
-  uint32_t reduce_wire;       /* FLS_WIRE_F32 (default): fp32 partial sums.  FLS_WIRE_BF16 (bf16 gradients only):
+  uint32_t reduce_wire;       /* FLS_WIRE_F32 (default): partial sums of bf16 gradients in fp32 (exact unless the
+                                 addends span more than 16 binades), of fp32 gradients in double with one rounding
+                                 to fp32 after the scaling by 1/K.  FLS_WIRE_BF16 (bf16 gradients only):
                                  every partial sum of both reduction levels and the final mean are rounded
                                  to bf16, emulating collectives that run in bf16 -- the setting in which the
                                  paper observes that the FSDP and HSDP orders give different numbers.  Slower
@@ -85,7 +87,7 @@ typedef struct {
                                  is a ring reduce-scatter + all-gather over R_rep equal sub-chunks of every
                                  rank's slice of a unit (ceil(M_u/R_rep) elements each): sub-chunk c is summed
                                  rho = c+1, ..., c (mod R_rep).  Same sums, other rounding order: visible with
-                                 FLS_WIRE_BF16, within rounding with fp32 partial sums.  Generic kernel (slower) */
+                                 FLS_WIRE_BF16, within rounding otherwise.  Generic kernel (slower)           */
   uint32_t state_copies;      /* FLS_STATE_PER_GROUP (default): one master/m/v/bf16 copy per group.
                                  FLS_STATE_PER_REPLICA: one per replica, G*R_rep in all (FL+HSDP as it runs: every
                                  replica of a group applies the same mean gradient to its own copy; only one replica
@@ -166,10 +168,10 @@ int fls_plan_query(const fls_plan* plan, fls_layout* out);
 int fls_plan_bind(fls_plan* plan, const fls_buffers* buffers);
 
 /* One local training step of all G groups (the groups train without waiting for one another), enqueued
- * on `cuda_stream` (a cudaStream_t; NULL = default stream).  Per group: mean of the K gradient buffers
- * in fp32, ascending buffer order inside a sharding group, then ascending replica order (reduce-scatter
+ * on `cuda_stream` (a cudaStream_t; NULL = default stream).  Per group: mean of the K gradient buffers,
+ * stored as fp32: ascending buffer order inside a sharding group, then ascending replica order (reduce-scatter
  * over S, then all-reduce over R: Background FSDP/HSDP, Eq. 2; reduce_wire and reduce_order change the
- * precision of the partial sums and the order), one multiply by 1/K; L2 norm of the mean
+ * precision of the partial sums and the order), one scaling by 1/K; L2 norm of the mean
  * gradient over the whole group; c = min(1, max_grad_norm/(norm + 1e-6)); AdamW with decoupled weight
  * decay and bias correction on master/m/v in place (on every state copy of the group; speculative plans
  * write the other buffer set, see fls_plan_set_speculative); bf16 copy of the new parameters (round to

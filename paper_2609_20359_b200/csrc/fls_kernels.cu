@@ -244,7 +244,7 @@ __device__ __forceinline__ void scale_mean(const ReduceArgs& a, const A (&outer)
 template <int N, bool F32, int KT, int SG>
 __device__ __forceinline__ void combine_loaded(const ReduceArgs& a, const Raw<N, F32> (&raw)[KT], float (&mean)[N]) {
   static_assert(KT > 0 && SG >= 0, "static shapes only");
-  using A = typename AccOf<F32>::type;
+  using A = typename AccOf<F32 && (KT > 1)>::type;      // a single buffer is its own mean in any precision
   A outer[N];
 #pragma unroll
   for (int e = 0; e < N; ++e) outer[e] = A(0);
@@ -671,7 +671,7 @@ __device__ __noinline__ void reduce_adamw_slice_scalar(const ReduceAdamArgs& p, 
 // kernel has nothing to do; otherwise it redoes the step with the real coefficient, reading the same (untouched)
 // input state and overwriting the same output buffers.
 template <bool F32, int KT, int SG>
-__global__ void __launch_bounds__(kThreads, KT == 0 ? 2 : (F32 ? 3 : 4)) fls_reduce_adamw_kernel(const __grid_constant__ ReduceAdamArgs p) {
+__global__ void __launch_bounds__(kThreads, KT == 0 ? 2 : ((F32 && KT > 1) ? 3 : 4)) fls_reduce_adamw_kernel(const __grid_constant__ ReduceAdamArgs p) {
   const AdamArgs& a = p.a;
   const uint32_t n_tiles = a.idx.n_tiles;
   if (blockIdx.x >= n_tiles) { dep_wait(); dep_launch(); return; }
@@ -720,7 +720,7 @@ __global__ void __launch_bounds__(kThreads, KT == 0 ? 2 : (F32 ? 3 : 4)) fls_red
 // (4 CTAs per SM measured best for a static K: 2 and 3 leave loads in flight on the table, 5 and 6 spill; the
 // run-time-K form holds a batch of eight raw loads next to the state and needs the registers of 2 CTAs per SM)
 template <bool F32, int KT, int SG>
-__global__ void __launch_bounds__(kThreads, KT == 0 ? 2 : (F32 ? 3 : 4)) fls_step_noclip_kernel(const __grid_constant__ ReduceAdamArgs p) {
+__global__ void __launch_bounds__(kThreads, KT == 0 ? 2 : ((F32 && KT > 1) ? 3 : 4)) fls_step_noclip_kernel(const __grid_constant__ ReduceAdamArgs p) {
   const AdamArgs& a = p.a;
   __shared__ unsigned arrived;
   begin_norm(&arrived);
