@@ -299,6 +299,8 @@ def measure_workload(args, cfg, fls, Session, rank, world, local, with_e2e, samp
         fls.fls_plan_set_l2_keep(sess.plan, int(args.l2_keep_mb * 2 ** 20))
     if args.batching is not None:
         fls.fls_plan_set_batching(sess.plan, args.batching)
+    if args.resident is not None:
+        fls.fls_plan_set_resident(sess.plan, args.resident)
     fill_session(sess, cfg)
     stream = torch.cuda.current_stream()
 
@@ -364,7 +366,8 @@ def measure_workload(args, cfg, fls, Session, rank, world, local, with_e2e, samp
     # second pass over the same number of steps with events around every kernel: per-kernel durations
     # (the clocks keep being sampled: an NVML reading can take as long as a short timed region)
     ms_prof, _ = timed(args.steps, True, sampler)
-    batched = fls.fls_plan_get_batching(sess.plan)
+    resident = fls.fls_plan_get_resident(sess.plan)
+    batched = fls.fls_plan_get_batching(sess.plan) and not resident
     kms, kn = fls.fls_get_kernel_ms(sess.plan)
     fls.fls_set_profiling(sess.plan, False)
     spec = None
@@ -428,6 +431,11 @@ def measure_workload(args, cfg, fls, Session, rank, world, local, with_e2e, samp
             # element, the follow-up kernel nothing when the guess held and the same again when it redoes the step
             per_launch.update(adamw=N * (kbytes + 26) * (1 + 1 - spec["hit_rate"]) / 2)
             traffic_key.update(adamw=("step_noclip", kbytes))
+        if resident:
+            # one cooperative kernel per step does everything for all groups (timed under "adamw")
+            per_launch.update(adamw=G * N * (kbytes + 26))
+            traffic_key.update(adamw=("step_resident", kbytes))
+            units.update(adamw=N * G)
         if batched:
             # all groups in one grid: a reduce or AdamW launch covers G times the elements
             per_launch.update(reduce=G * per_launch["reduce"], adamw=G * per_launch["adamw"])
@@ -445,7 +453,8 @@ def measure_workload(args, cfg, fls, Session, rank, world, local, with_e2e, samp
         rep = fls.fls_comm_report(sess.plan)
         # bytes the timed steps had to move: every sync step, plus the FedAvg calls that fell inside the region
         # (the fused aggregation moves no bytes of its own: an aggregation step costs what a plain step costs)
-        step_bytes = rep["hbm_bytes_sync_step"] + (0 if fused else rep["hbm_bytes_fedavg"] * fedavg_calls / args.steps)
+        # (a resident plan's fused call is the resident step followed by a FedAvg kernel of its own)
+        step_bytes = rep["hbm_bytes_sync_step"] + (0 if fused and not resident else rep["hbm_bytes_fedavg"] * fedavg_calls / args.steps)
         if spec is not None:
             step_bytes += rep["hbm_bytes_sync_step"] * (1 - spec["hit_rate"])       # a redone group-step moves its bytes twice
         ms_step = ms_total / args.steps
@@ -453,7 +462,7 @@ def measure_workload(args, cfg, fls, Session, rank, world, local, with_e2e, samp
             "value": world * G * P * args.steps / (ms_total / 1e3), "ms_per_step": ms_step,
             "config": {"workload": cfg["name"], "n_params": P, "groups": G, "shard_dim": cfg["shard_dim"],
                        "replicate_dim": cfg["replicate_dim"], "sync_period": cfg["sync_period"], "grad_dtype": cfg["grad_dtype"],
-                       "fedavg_opt_state": bool(args.opt_state), "fused_aggregation": bool(fused), "groups_share_a_grid": bool(batched),
+                       "fedavg_opt_state": bool(args.opt_state), "fused_aggregation": bool(fused), "groups_share_a_grid": bool(batched), "resident_step": bool(resident),
                        "fedavg_calls_in_timed_region": fedavg_calls,
                        "l2": "working set exceeds L2, no flush needed" if flush_buf is None else "L2 flushed (512 MB write, untimed) before every timed step",
                        "parallelism": "replicas only" if world > 1 else "1 gpu"},
@@ -669,6 +678,7 @@ def main():
     ap.add_argument("--no-overlap", action="store_true", help="plain launches instead of programmatic dependent launch")
     ap.add_argument("--speculative", action="store_true", help="speculative single pass (guess: clip coefficient 1) with a second set of state buffers")
     ap.add_argument("--batching", type=int, default=None, choices=[-1, 0, 1], help="all groups in one grid per kernel: -1 automatic (small plans), 0 never, 1 whenever possible")
+    ap.add_argument("--resident", type=int, default=None, choices=[-1, 0, 1], help="whole step of all groups as one cooperative kernel: -1 automatic (small plans), 0 never, 1 whenever the plan fits the device")
     ap.add_argument("--l2-keep-mb", type=float, default=None, help="MiB at the end of the reduced gradient stored with L2 evict-last (library default: 64)")
     # slices of a workload, for profiler captures that must stay small (same kernels, fewer bytes)
     ap.add_argument("--n-params", type=int, default=0, help="override P (single flat unit)")

@@ -47,7 +47,8 @@ enum { FLS_ORDER_ASCENDING = 0, FLS_ORDER_RING = 1 };  /* reduce_order */
 enum { FLS_STATE_PER_GROUP = 0, FLS_STATE_PER_REPLICA = 1 }; /* state_copies */
 enum { FLS_AVG_PARAMS = 1, FLS_AVG_OPT_STATE = 2, FLS_AVG_FUSED = 4 }; /* fedavg_what bit mask */
 enum { FLS_KERNEL_REDUCE = 0, FLS_KERNEL_ADAMW = 1, FLS_KERNEL_FEDAVG = 2, FLS_KERNEL_ADAMW_FEDAVG = 3, FLS_KERNEL_COUNT = 4 };
-enum { FLS_STATUS_NONFINITE_NORM = 1 }; /* sticky bits of the device status word */
+enum { FLS_STATUS_NONFINITE_NORM = 1,   /* sticky bits of the device status word */
+       FLS_STATUS_WAIT_EXPIRED = 2 };   /* a CTA of the resident step gave up waiting for its group's norm; the step is incomplete */
 
 #define FLS_MAX_GROUPS 64        /* G <= 64 */
 #define FLS_MAX_GRAD_BUFFERS 64  /* K = shard_dim * replicate_dim <= 64 */
@@ -297,6 +298,27 @@ int fls_get_state(const fls_plan* plan, uint32_t copy, float** master, float** m
  * fls_plan_get_batching: whether the next fls_sync_step would run that way. */
 int fls_plan_set_batching(fls_plan* plan, int mode);
 int fls_plan_get_batching(const fls_plan* plan, int* active);
+
+/* Resident step.  When all G groups together are small enough for every CTA of one grid to be resident on the device
+ * at once (each CTA keeping the mean gradient of up to a few tiles in shared memory: about 8 million elements in all on
+ * 148 SMs), fls_sync_step can run as ONE cooperative kernel: reduce, norm, a wait inside the kernel until the group's
+ * clip coefficient is known, AdamW.  K*e_g + 26 bytes per element and one launch instead of two or 2*G.  Needs K in
+ * {1, 2, 4, 8} in a flat or 1/2/4-wide two-level order, G*K <= 64, fp32 partial sums in ascending order, one state copy
+ * per group, clipping on, no speculation.  mode -1 (default): automatically, when the plan fits and the G reduced
+ * gradients would take at most 24 MiB; 0: never; 1: whenever the plan fits (FLS_ESTATE otherwise; the fit depends on
+ * the device, so the plan must be bound).  The reduced gradient is not stored (fls_get_reduced_grad: FLS_ESTATE) and
+ * fls_sync_step_fedavg runs the resident step followed by fls_fedavg.  Mean gradient and AdamW arithmetic are those of
+ * the other routes; the norm is summed over another tree (several tiles per CTA), so it can differ from theirs in the
+ * last bits of a double.  The wait is bounded: a CTA that polls `wait_limit` times in vain (0 keeps the default,
+ * about a second) sets FLS_STATUS_WAIT_EXPIRED in the status word and leaves its part of the state untouched.
+ * fls_plan_get_resident: whether the next fls_sync_step would run that way. */
+int fls_plan_set_resident(fls_plan* plan, int mode, uint32_t wait_limit);
+int fls_plan_get_resident(const fls_plan* plan, int* active);
+
+/* For tests of the bounded wait: the next resident step (one launch) is started so that its CTAs wait for a value
+ * that nobody publishes.  Every CTA gives up after `wait_limit` polls, FLS_STATUS_WAIT_EXPIRED appears in the status
+ * word, master/m/v/bf16 stay as they were, and the device stays usable.  Set a small wait_limit first. */
+int fls_debug_expire_next_wait(fls_plan* plan);
 
 /* How many bytes at the end of the reduced gradient the reduce kernel stores with the "evict last" L2 policy (the
  * AdamW kernel walks the reduced gradient backwards, so it reads that part first and finds it in L2); the rest is

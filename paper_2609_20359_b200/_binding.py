@@ -18,6 +18,7 @@ FLS_STATE_PER_GROUP, FLS_STATE_PER_REPLICA = 0, 1
 FLS_AVG_PARAMS, FLS_AVG_OPT_STATE, FLS_AVG_FUSED = 1, 2, 4
 FLS_KERNEL_REDUCE, FLS_KERNEL_ADAMW, FLS_KERNEL_FEDAVG, FLS_KERNEL_ADAMW_FEDAVG, FLS_KERNEL_COUNT = 0, 1, 2, 3, 4
 FLS_STATUS_NONFINITE_NORM = 1
+FLS_STATUS_WAIT_EXPIRED = 2
 FLS_MAX_GROUPS = 64
 FLS_MAX_GRAD_BUFFERS = 64
 FLS_MAX_FUSED_GROUPS = 16
@@ -30,6 +31,7 @@ EXPORTS = [
     "fls_sync_step_fedavg", "fls_fedavg_outer",
     "fls_get_norms", "fls_get_reduced_grad", "fls_get_status", "fls_get_step", "fls_set_step", "fls_comm_report",
     "fls_plan_bind_shadow", "fls_plan_set_speculative", "fls_get_spec_stats", "fls_get_state", "fls_plan_set_l2_keep", "fls_plan_set_batching", "fls_plan_get_batching",
+    "fls_plan_set_resident", "fls_plan_get_resident", "fls_debug_expire_next_wait",
     "fls_plan_tune", "fls_plan_set_recompute", "fls_plan_set_single_pass", "fls_plan_set_overlap", "fls_set_profiling", "fls_get_kernel_ms", "fls_get_launch_count", "fls_plan_destroy",
     "fls_last_error", "fls_reduce_norm_noalloc",
 ]
@@ -105,6 +107,9 @@ def _load() -> C.CDLL:
     lib.fls_plan_set_l2_keep.argtypes = [P, C.c_uint64]
     lib.fls_plan_set_batching.argtypes = [P, C.c_int]
     lib.fls_plan_get_batching.argtypes = [P, C.POINTER(C.c_int)]
+    lib.fls_plan_set_resident.argtypes = [P, C.c_int, C.c_uint32]
+    lib.fls_plan_get_resident.argtypes = [P, C.POINTER(C.c_int)]
+    lib.fls_debug_expire_next_wait.argtypes = [P]
     lib.fls_plan_set_recompute.argtypes = [P, C.c_int]
     lib.fls_plan_set_single_pass.argtypes = [P, C.c_int]
     lib.fls_plan_set_overlap.argtypes = [P, C.c_int]
@@ -299,6 +304,23 @@ def fls_plan_get_batching(plan: int) -> bool:
     a = C.c_int(0)
     _check(lib.fls_plan_get_batching(plan, C.byref(a)))
     return bool(a.value)
+
+
+def fls_plan_set_resident(plan: int, mode: int, wait_limit: int = 0) -> None:
+    """-1 automatic (small plans that fit the device), 0 never, 1 whenever the plan fits: the whole step of all groups as one
+    cooperative kernel.  wait_limit: polls before a waiting CTA gives up (0 keeps the current value)."""
+    _check(lib.fls_plan_set_resident(plan, mode, wait_limit))
+
+
+def fls_plan_get_resident(plan: int) -> bool:
+    a = C.c_int(0)
+    _check(lib.fls_plan_get_resident(plan, C.byref(a)))
+    return bool(a.value)
+
+
+def fls_debug_expire_next_wait(plan: int) -> None:
+    """Test hook: the next resident step waits for a value nobody publishes (every CTA gives up after wait_limit polls)."""
+    _check(lib.fls_debug_expire_next_wait(plan))
 
 
 def fls_plan_set_l2_keep(plan: int, nbytes: int) -> None:

@@ -72,6 +72,11 @@ struct fls_plan {
   bool speculative = false;
   bool fused_plan = false;               // fls_sync_step_fedavg may fuse the aggregation into the optimizer kernel
   int batch_mode = -1;                   // groups in one grid: -1 automatic (small plans), 0 never, 1 whenever possible
+  int resident_mode = -1;                // whole step in one cooperative kernel: -1 automatic, 0 never, 1 whenever it fits
+  uint32_t res_tiles = 0, res_grid = 0;  // tiles per CTA and grid.x of the resident step on the bound device (0: does not fit)
+  uint32_t res_seq = 0;                  // id of the last resident launch (what the ready words are compared with)
+  uint32_t res_wait_limit = 1u << 22;    // polls (64 ns apart at least) before a CTA gives up
+  bool res_hold_back = false;            // test hook: the next resident launch waits for an id nobody publishes
   uint64_t l2_keep_bytes = 64ull << 20;  // tail of the reduced gradient stored with L2 evict-last
   char* ws = nullptr;
 
@@ -104,6 +109,7 @@ struct fls_plan {
   uint32_t* d_status() const { return reinterpret_cast<uint32_t*>(ws + kWsStatus); }
   uint32_t* d_ticket() const { return reinterpret_cast<uint32_t*>(ws + kWsTickets); }
   uint32_t* d_spec_counts() const { return reinterpret_cast<uint32_t*>(ws + kWsStatus) + 2; }
+  uint32_t* d_ready() const { return reinterpret_cast<uint32_t*>(ws + kWsReady); }
   // One grid for all groups (instead of one launch per group) needs a reduced-gradient slot per group, a level structure
   // the batched kernels are built for, the default two-pass route and one state copy per group.  Automatic: only when all
   // the reduced gradients together take at most 24 MiB (a fifth of the L2), i.e. when a launch per group would be launch-bound;
@@ -116,11 +122,21 @@ struct fls_plan {
     if (batch_mode == 0 || !can_batch()) return false;
     return batch_mode > 0 || uint64_t(desc.groups) * lay.n_padded * 4 <= kBatchScratchBytes;
   }
+  // The whole step as one cooperative kernel: a shape the resident kernel is built for, the plain reduction, clipping on
+  // (without it every group's step is one kernel already) and a grid that fits the bound device (res_tiles > 0).
+  bool can_resident() const {
+    return res_tiles > 0 && resident_shape_ok(K, reduce_sg) && uint64_t(desc.groups) * K <= FLS_MAX_GRAD_BUFFERS &&
+           plain_reduce() && !single_pass && !speculative;
+  }
+  bool resident() const {
+    if (resident_mode == 0 || !can_resident()) return false;
+    return resident_mode > 0 || uint64_t(desc.groups) * lay.n_padded * 4 <= kBatchScratchBytes;
+  }
   // how fls_sync_step currently gets from the gradients to the new state (for the HBM byte count)
   // the routes that form the mean gradient inside the AdamW kernel exist for fp32 partial sums in ascending order
   // and one state copy per group
   bool plain_reduce() const { return desc.reduce_wire == FLS_WIRE_F32 && !ring && R_state == 1; }
-  int route() const { return speculative || single_pass ? 2 : (recompute ? 1 : 0); }
+  int route() const { return speculative || single_pass || resident() ? 2 : (recompute ? 1 : 0); }
 
   SegIndex seg_index() const {
     SegIndex ix{};
@@ -362,6 +378,70 @@ int run_groups_batched(fls_plan* p, double lr, uint64_t t_new, cudaStream_t st, 
   return FLS_OK;
 }
 
+// Tiles per CTA and grid.x with which the resident step fits the current device: the smallest number of tiles per CTA
+// (8 KB of shared memory each) for which all G * ceil(n_tiles / T) CTAs can be resident at once; 0, 0 if none does.
+void plan_resident_shape(fls_plan* p) {
+  p->res_tiles = p->res_grid = 0;
+  if (!resident_shape_ok(p->K, p->reduce_sg) || p->lay.n_tiles == 0) return;
+  const bool f32 = p->desc.grad_dtype == FLS_GRAD_F32;
+  for (uint32_t T = 1; T <= 27; ++T) {
+    unsigned cap = 0;
+    if (resident_max_ctas(f32, p->K, p->reduce_sg, size_t(T) * kTile * 4, p->sm_count, &cap) != cudaSuccess) {
+      cudaGetLastError();
+      return;
+    }
+    if (cap == 0) return;
+    const uint64_t gx = (p->lay.n_tiles + T - 1) / T;
+    if (gx * p->desc.groups <= cap) {
+      p->res_tiles = T;
+      p->res_grid = uint32_t(gx);
+      return;
+    }
+  }
+}
+
+// The step of all groups as one cooperative kernel (see fls_plan_set_resident).
+int run_resident(fls_plan* p, double lr, uint64_t t_new, cudaStream_t st) {
+  const fls_plan_desc& d = p->desc;
+  const uint32_t G = d.groups;
+  ResidentArgs a{};
+  a.r = common_reduce_args(p);
+  for (uint32_t i = 0; i < G * p->K; ++i) a.r.grad[i] = p->grads[i];
+  a.r.gbar = nullptr;
+  a.r.store_gbar = 0;
+  p->gbar_valid = false;
+  a.r.partials = p->d_partials();
+  a.r.chunk_partials = p->d_chunk_partials();
+  a.r.chunk_count = p->d_chunk_count();
+  a.r.ticket = p->d_ticket();
+  a.r.norm_out = p->d_norms();
+  a.r.coef_out = p->d_coefs();
+  a.r.normsq_out = p->d_normsq();
+  a.r.keep_from_tile = uint32_t(p->lay.n_tiles);
+  if (++p->res_seq == 0) p->res_seq = 1;            // the ready words start at zero
+  a.r.launch_id = p->res_seq;
+  a.r.ready = p->d_ready();
+  for (uint32_t g = 0; g < G; ++g) {
+    a.theta[g] = p->master[g];
+    a.m[g] = p->m[g];
+    a.v[g] = p->v[g];
+    a.pbf16[g] = p->pbf16[g];
+  }
+  const AdamScalars sc = adam_scalars(d, lr, t_new);
+  a.decay = sc.decay; a.beta1 = sc.beta1; a.omb1 = sc.omb1; a.beta2 = sc.beta2; a.omb2 = sc.omb2;
+  a.step_size = sc.step_size; a.inv_sqrt_bc2 = sc.inv_sqrt_bc2; a.eps = sc.eps;
+  a.tiles_per_cta = p->res_tiles;
+  a.wait_limit = p->res_wait_limit;
+  // test hook (one launch): the waiters expect an id that nobody publishes, so every wait runs out
+  a.expect_id = p->res_hold_back ? (a.r.launch_id ^ 0x80000000u) : a.r.launch_id;
+  p->res_hold_back = false;
+  const bool f32 = d.grad_dtype == FLS_GRAD_F32;
+  cudaError_t e = timed_launch(p, FLS_KERNEL_ADAMW, st,
+                               [&] { return launch_step_resident(a, f32, p->reduce_sg, p->res_grid, G, st); });
+  if (e != cudaSuccess) return cuda_fail(e, "resident step kernel launch");
+  return FLS_OK;
+}
+
 // Every range must be non-null, aligned device memory of the current device.  Outputs may overlap nothing;
 // gradient buffers may only overlap each other (a caller may feed one buffer to several replicas).
 int check_ranges(const std::vector<Range>& ranges, int dev) {
@@ -556,6 +636,8 @@ int fls_plan_bind(fls_plan* p, const fls_buffers* b) {
   p->ranges = ranges;
   p->master2.clear(); p->m2.clear(); p->v2.clear();   // a new binding drops the second buffer set
   p->speculative = false;
+  p->res_seq = 0;                  // the ready words are zeroed below
+  plan_resident_shape(p);
 
   e = cudaMemset(p->ws, 0, size_t(kWsSegments));
   if (e != cudaSuccess) return cuda_fail(e, "cudaMemset(workspace head)");
@@ -586,7 +668,10 @@ int fls_sync_step(fls_plan* p, double lr, void* cuda_stream, int* fedavg_due) {
   if (!step_preamble(p, &lr)) return fail(FLS_EINVAL, "fls_sync_step: lr must be finite and >= 0");
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const uint64_t t_new = p->step + 1;
-  if (p->batching()) {
+  if (p->resident()) {
+    const int rc = run_resident(p, lr, t_new, st);
+    if (rc != FLS_OK) return rc;
+  } else if (p->batching()) {
     const int rc = run_groups_batched(p, lr, t_new, st, true);
     if (rc != FLS_OK) return rc;
   } else {
@@ -709,7 +794,7 @@ int fls_sync_step_fedavg(fls_plan* p, double lr, const uint64_t* sample_counts, 
   if (!p) return fail(FLS_EINVAL, "fls_sync_step_fedavg: null plan");
   if (!p->bound) return fail(FLS_ESTATE, "fls_sync_step_fedavg: plan has no buffers bound");
   const uint32_t G = p->desc.groups;
-  if (!p->fused_plan) {             // not planned for fusion: the two calls in sequence give the same result
+  if (!p->fused_plan || p->resident()) {   // not planned for fusion, or the step runs as one resident kernel: the two calls in sequence give the same result
     const int rc = fls_sync_step(p, lr, cuda_stream, nullptr);
     return rc != FLS_OK ? rc : fls_fedavg(p, sample_counts, cuda_stream);
   }
@@ -898,7 +983,30 @@ int fls_plan_set_batching(fls_plan* p, int mode) {
 
 int fls_plan_get_batching(const fls_plan* p, int* active) {
   if (!p || !active) return fail(FLS_EINVAL, "fls_plan_get_batching: null argument");
-  *active = p->batching() ? 1 : 0;
+  *active = p->batching() && !p->resident() ? 1 : 0;     // the resident step, where it applies, comes first
+  return FLS_OK;
+}
+
+int fls_plan_set_resident(fls_plan* p, int mode, uint32_t wait_limit) {
+  if (!p) return fail(FLS_EINVAL, "fls_plan_set_resident: null plan");
+  if (mode > 0 && !p->can_resident())
+    return fail(FLS_ESTATE, "fls_plan_set_resident: needs a bound plan whose G * ceil(tiles / T) CTAs fit the device at once, K in {1, 2, 4, 8} "
+                            "in a flat or 1/2/4-wide two-level order, G*K <= 64, fp32 partial sums in ascending order, one state copy per "
+                            "group, clipping on and no speculation");
+  p->resident_mode = mode < 0 ? -1 : (mode > 0 ? 1 : 0);
+  if (wait_limit) p->res_wait_limit = wait_limit;
+  return FLS_OK;
+}
+
+int fls_plan_get_resident(const fls_plan* p, int* active) {
+  if (!p || !active) return fail(FLS_EINVAL, "fls_plan_get_resident: null argument");
+  *active = p->resident() ? 1 : 0;
+  return FLS_OK;
+}
+
+int fls_debug_expire_next_wait(fls_plan* p) {
+  if (!p) return fail(FLS_EINVAL, "fls_debug_expire_next_wait: null plan");
+  p->res_hold_back = true;
   return FLS_OK;
 }
 

@@ -34,7 +34,8 @@ constexpr uint64_t kWsNorms = 256;       // float[64]
 constexpr uint64_t kWsCoefs = 512;       // float[64]
 constexpr uint64_t kWsNormSq = 768;      // double[64]
 constexpr uint64_t kWsTickets = 1280;    // uint32[64]: one ticket counter per group
-constexpr uint64_t kWsSegments = 1536;   // Segment[n_segments], then per group the norm tree (double[n_tiles] CTA partials,
+constexpr uint64_t kWsReady = 1536;      // uint32[64]: resident step, id of the last launch whose coefficient is published
+constexpr uint64_t kWsSegments = 1792;   // Segment[n_segments], then per group the norm tree (double[n_tiles] CTA partials,
                                          // chunk sums, chunk arrival counters), then the reduced-gradient scratch
 
 struct Layout {

@@ -158,6 +158,17 @@ __device__ __forceinline__ double warp_sum(double x) {
   return x;
 }
 
+// Release / acquire on one word in global memory (device scope): what was written before the store is visible to
+// whoever sees the stored value with the load.
+__device__ __forceinline__ void st_release(uint32_t* p, uint32_t v) {
+  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p) {
+  uint32_t v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
 // ------------------------------------------------------------------------------------------------
 // K1: gradient reduction in the paper's order + squared norm.
 // ------------------------------------------------------------------------------------------------
@@ -469,6 +480,7 @@ __device__ __forceinline__ void finish_norm(const ReduceArgs& a, float sq, unsig
     if (!isfinite(nrm)) atomicOr(a.status, uint32_t(FLS_STATUS_NONFINITE_NORM));
     if (a.spec_counts) atomicAdd(a.spec_counts + (float(c1) == 1.0f ? 0 : 1), 1u);   // speculative step: kept / redone
     a.ticket[y] = 0u;                    // ready for the next launch (stream order)
+    if (a.ready) st_release(a.ready + y, a.launch_id);   // resident step: the group's CTAs are waiting for this
   }
 }
 
@@ -759,6 +771,111 @@ __global__ void __launch_bounds__(kThreads, KT == 0 ? 2 : ((F32 && KT > 1) ? 3 :
   dep_wait();
   dep_launch();
   finish_norm<kThreads>(p.r, sq, &arrived);
+}
+
+// Whole step of ALL groups in one kernel, for plans small enough that every CTA of the grid is resident at once
+// (cooperative launch; group = blockIdx.y).  Phase 1: the CTA forms the mean gradient of its T tiles (x, x + gridDim.x,
+// ...), keeps it in shared memory (thread-private slots, no barrier needed) and contributes to the group's norm.
+// Then it fetches the state of its first tile and waits until the warp that completes the group's norm tree has
+// published the clip coefficient (ready[y] == launch_id).  Phase 2: AdamW on the same tiles with the stashed mean
+// gradient.  Per element K*e_g + 26 bytes, one launch per step instead of two per group.
+// The wait is bounded: after wait_limit polls the CTA records FLS_STATUS_WAIT_EXPIRED and returns without
+// touching the state (all CTAs are resident, so this happens only if the grid lost a CTA to an error).
+// Mean gradient, AdamW arithmetic and the per-thread sums of squares are those of the other routes; the norm's
+// tree groups T tiles per CTA instead of one, so in double it can differ from the two-pass route's in the last bits.
+template <bool F32, int KT, int SG>
+__global__ void __launch_bounds__(kThreads, (F32 && KT > 1) ? 3 : 4) fls_step_resident_kernel(const __grid_constant__ ResidentArgs p) {
+  extern __shared__ float4 stash[];        // [T][2][kThreads]
+  __shared__ unsigned arrived;
+  __shared__ unsigned go;
+  const ReduceArgs& a = p.r;
+  const uint32_t y = blockIdx.y, gk0 = y * a.K, T = p.tiles_per_cta, n_tiles = a.idx.n_tiles;
+  begin_norm(&arrived);
+  float sq = 0.f;
+  for (uint32_t i = 0; i < T; ++i) {
+    const uint32_t tile = blockIdx.x + i * gridDim.x;
+    if (tile >= n_tiles) break;
+    const Slice s = slice_of(a.idx.segs + find_segment(a.idx, tile), tile, threadIdx.x);
+    float g[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) g[e] = 0.f;
+    if (s.vec) {
+      reduce_elems<8, F32, KT, SG>(a, s.j, g, 0, gk0);
+      float s8 = 0.f;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) s8 = fmaf(g[e], g[e], s8);
+      sq += s8;
+    } else {
+      for (uint32_t e = 0; e < s.n; ++e) {
+        float t[1];
+        reduce_elems<1, F32, 0, -1>(a, s.j + e, t, 0, gk0);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) if (q == int(e)) g[q] = t[0];
+        sq = fmaf(t[0], t[0], sq);
+      }
+    }
+    stash[(i * 2 + 0) * kThreads + threadIdx.x] = make_float4(g[0], g[1], g[2], g[3]);
+    stash[(i * 2 + 1) * kThreads + threadIdx.x] = make_float4(g[4], g[5], g[6], g[7]);
+  }
+  finish_norm<kThreads>(a, sq, &arrived, y);
+
+  // state of the first tile: nothing of it depends on the norm, so the loads go out before the wait
+  float* const theta = p.theta[y];
+  float* const m_ = p.m[y];
+  float* const v_ = p.v[y];
+  uint16_t* const pbf16 = p.pbf16[y];
+  Slice s0 = slice_of(a.idx.segs + find_segment(a.idx, blockIdx.x), blockIdx.x, threadIdx.x);   // blockIdx.x < n_tiles
+  F8 th0, m0, v0;
+  if (s0.vec) {
+    th0 = ld8_stream(theta + s0.a);
+    m0 = ld8_stream(m_ + s0.a);
+    v0 = ld8_stream(v_ + s0.a);
+  }
+  if (threadIdx.x == 0) {
+    unsigned ok = 1;
+    uint32_t polls = 0;
+    while (ld_acquire(a.ready + y) != p.expect_id) {
+      if (++polls > p.wait_limit) { ok = 0; break; }
+      __nanosleep(64);
+    }
+    if (!ok) atomicOr(a.status, uint32_t(FLS_STATUS_WAIT_EXPIRED));
+    go = ok;
+  }
+  __syncthreads();
+  if (!go) return;
+  const float c = __ldcg(a.coef_out + y);
+  // AdamW on tile i of this CTA with the stashed mean gradient; th, m, v: the thread's state if the slice is a vector
+  auto apply = [&](uint32_t i, const Slice& s, F8& th, F8& m, F8& v) {
+    const float4 ga = stash[(i * 2 + 0) * kThreads + threadIdx.x], gb = stash[(i * 2 + 1) * kThreads + threadIdx.x];
+    const float g[8] = {ga.x, ga.y, ga.z, ga.w, gb.x, gb.y, gb.z, gb.w};
+    if (s.vec) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) adamw_one(p, c, g[e], th.v[e], m.v[e], v.v[e]);
+      st8_stream(theta + s.a, th);
+      st8_stream(m_ + s.a, m);
+      st8_stream(v_ + s.a, v);
+      st_b128_stream(pbf16 + s.j, pack_bf16x8(th));
+    } else {
+      for (uint32_t e = 0; e < s.n; ++e) {
+        float ge = 0.f;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) if (q == int(e)) ge = g[q];
+        float t1 = theta[s.a + e], m1 = m_[s.a + e], v1 = v_[s.a + e];
+        adamw_one(p, c, ge, t1, m1, v1);
+        theta[s.a + e] = t1; m_[s.a + e] = m1; v_[s.a + e] = v1;
+        pbf16[s.j + e] = to_bf16_bits(t1);
+      }
+    }
+  };
+  apply(0, s0, th0, m0, v0);
+  for (uint32_t i = 1; i < T; ++i) {
+    const uint32_t tile = blockIdx.x + i * gridDim.x;
+    if (tile >= n_tiles) break;
+    const Slice s = slice_of(a.idx.segs + find_segment(a.idx, tile), tile, threadIdx.x);
+    F8 th, m, v;
+    if (s.vec) { th = ld8_stream(theta + s.a); m = ld8_stream(m_ + s.a); v = ld8_stream(v_ + s.a); }
+    apply(i, s, th, m, v);
+  }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1147,6 +1264,64 @@ cudaError_t launch_step_noclip(const ReduceAdamArgs& a, bool f32, int sg, cudaSt
   else
     launch_noclip_t<false>(a, sg, grid, st, overlap);
   return cudaGetLastError();
+}
+
+namespace {
+using ResidentKernel = void (*)(ResidentArgs);
+template <bool F32, int KT>
+ResidentKernel resident_kernel_k(int sg) {
+  if (sg == 0) return fls_step_resident_kernel<F32, KT, 0>;
+  if constexpr (KT >= 2) { if (sg == 1) return fls_step_resident_kernel<F32, KT, 1>; }
+  if constexpr (KT >= 4) { if (sg == 2) return fls_step_resident_kernel<F32, KT, 2>; }
+  if constexpr (KT == 8) { if (sg == 4) return fls_step_resident_kernel<F32, KT, 4>; }
+  return nullptr;
+}
+template <bool F32>
+ResidentKernel resident_kernel_t(uint32_t K, int sg) {
+  switch (K) {
+    case 1: return resident_kernel_k<F32, 1>(sg);
+    case 2: return resident_kernel_k<F32, 2>(sg);
+    case 4: return resident_kernel_k<F32, 4>(sg);
+    case 8: return resident_kernel_k<F32, 8>(sg);
+    default: return nullptr;
+  }
+}
+ResidentKernel resident_kernel(bool f32, uint32_t K, int sg) {
+  return f32 ? resident_kernel_t<true>(K, sg) : resident_kernel_t<false>(K, sg);
+}
+}  // namespace
+
+bool resident_shape_ok(uint32_t K, int sg) { return resident_kernel(false, K, sg) != nullptr; }
+
+cudaError_t resident_max_ctas(bool f32, uint32_t K, int sg, size_t smem_bytes, int sm_count, unsigned* out) {
+  *out = 0;
+  ResidentKernel k = resident_kernel(f32, K, sg);
+  if (!k) return cudaErrorInvalidValue;
+  cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_bytes));
+  if (e != cudaSuccess) return e;
+  int per_sm = 0;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, kThreads, smem_bytes);
+  if (e != cudaSuccess) return e;
+  *out = unsigned(per_sm) * unsigned(sm_count);
+  return cudaSuccess;
+}
+
+// Cooperative launch: the driver refuses the launch unless the whole grid can be resident at once, which is what
+// lets the CTAs of a group wait for one another inside the kernel.
+cudaError_t launch_step_resident(const ResidentArgs& a, bool f32, int sg, unsigned grid_x, unsigned groups, cudaStream_t st) {
+  ResidentKernel k = resident_kernel(f32, a.r.K, sg);
+  if (!k) return cudaErrorInvalidValue;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid_x, groups);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = size_t(a.tiles_per_cta) * kTile * sizeof(float);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeCooperative;
+  attr[0].val.cooperative = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, k, a);
 }
 
 cudaError_t launch_reduce_adamw(const ReduceAdamArgs& a, bool f32, int sg, unsigned grid, cudaStream_t st, bool overlap) {

@@ -50,6 +50,10 @@ struct ReduceArgs {
   uint32_t ring;                           // 0: ascending buffer index at both levels
   uint32_t S, R;                           // shard_dim, replicate_dim (used by the ring order)
   uint32_t* spec_counts;                   // device, 2 counters (coefficient == 1, != 1) or null: speculative steps only
+  // resident step only (null otherwise): the warp that finishes group y's norm publishes ready[y] = launch_id after the
+  // coefficient, which releases the group's CTAs waiting in the same kernel
+  uint32_t* ready;
+  uint32_t launch_id;
 };
 
 struct AdamArgs {
@@ -76,6 +80,20 @@ struct AdamBatchArgs {
   SegIndex idx;
   int descending;
   float decay, beta1, omb1, beta2, omb2, step_size, inv_sqrt_bc2, eps;
+};
+
+// Whole step of all groups in ONE cooperative kernel (small plans): every CTA reduces its tiles, keeps the mean gradient
+// in shared memory, waits until its group's norm is complete and applies AdamW.
+struct ResidentArgs {
+  ReduceArgs r;                            // batched form (all groups' buffers; gbar unused, store_gbar = 0)
+  float* theta[FLS_MAX_GROUPS];
+  float* m[FLS_MAX_GROUPS];
+  float* v[FLS_MAX_GROUPS];
+  uint16_t* pbf16[FLS_MAX_GROUPS];
+  float decay, beta1, omb1, beta2, omb2, step_size, inv_sqrt_bc2, eps;
+  uint32_t tiles_per_cta;                  // T: CTA x takes tiles x, x + gridDim.x, ... (T of them at most)
+  uint32_t wait_limit;                     // polls of ready[y] before a CTA gives up (FLS_STATUS_WAIT_EXPIRED)
+  uint32_t expect_id;                      // what ready[y] must hold for the wait to end (= r.launch_id)
 };
 
 // AdamW that forms the mean gradient itself from the K gradient buffers (recompute plan, small K).
@@ -140,6 +158,12 @@ bool reduce_batchable(uint32_t K, int sg);
 cudaError_t launch_reduce_batch(const ReduceArgs& a, bool f32, int sg, unsigned groups, cudaStream_t st, bool overlap);
 cudaError_t launch_adamw_batch(const AdamBatchArgs& a, unsigned grid, unsigned groups, cudaStream_t st, bool overlap);
 cudaError_t launch_step_noclip(const ReduceAdamArgs& a, bool f32, int sg, cudaStream_t st, bool overlap);
+// Resident step: static K in {1, 2, 4, 8} with a static level structure only (resident_shape_ok).  The launch is
+// cooperative: grid_x * groups CTAs must be resident at once; resident_max_ctas gives that bound for a given amount
+// of dynamic shared memory (tiles_per_cta * kTile * 4 bytes) on the current device.
+bool resident_shape_ok(uint32_t K, int sg);
+cudaError_t resident_max_ctas(bool f32, uint32_t K, int sg, size_t smem_bytes, int sm_count, unsigned* out);
+cudaError_t launch_step_resident(const ResidentArgs& a, bool f32, int sg, unsigned grid_x, unsigned groups, cudaStream_t st);
 cudaError_t launch_reduce_adamw(const ReduceAdamArgs& a, bool f32, int sg, unsigned grid, cudaStream_t st, bool overlap);
 cudaError_t launch_adamw(const AdamArgs& a, unsigned grid, cudaStream_t st, bool overlap);
 cudaError_t launch_fedavg(const FedavgArgs& a, unsigned grid, cudaStream_t st, bool overlap);

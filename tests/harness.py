@@ -65,7 +65,7 @@ class Case:
 
     def __init__(self, units, G, S, R_rep=1, H=1, Q=8, grad_dtype="bf16", opt_state=False, seed=1234,
                  grad_sigma=1e-3, master_sigma=0.02, per_buffer_scale=False, hp: orc.Hyper = None, guard=4096,
-                 same_grads_all_groups=False, fused=False, state_per_replica=False, speculative=False):
+                 same_grads_all_groups=False, fused=False, state_per_replica=False, speculative=False, resident=-1):
         from paper_2609_20359_b200.session import Session
         self.units, self.G, self.S, self.R_rep, self.H, self.Q = list(units), G, S, R_rep, H, Q
         self.K = S * R_rep
@@ -87,6 +87,9 @@ class Case:
                             self.hp.beta2, self.hp.eps, self.hp.weight_decay, self.hp.max_grad_norm, guard_bytes=guard, fused=fused,
                             wire_bf16=self.hp.wire_bf16, ring=self.hp.ring, state_per_replica=state_per_replica, speculative=speculative)
         self.fused = fused
+        if resident != -1:            # -1: the library's default (small plans run the step as one resident kernel)
+            import paper_2609_20359_b200._binding as _b
+            _b.fls_plan_set_resident(self.sess.plan, resident)
         lay = self.sess.layout
         assert lay["n_padded"] == self.L.n_padded and lay["shard_numel"] == self.L.shard_numel
         assert lay["n_state_copies"] == G * self.R_state

@@ -127,7 +127,7 @@ def test_groups_in_one_grid_give_identical_results(fls, units, G, S, R_rep, Q, d
     counts = [sy.sample_count(29, g) for g in range(G)]
     for mode in (-1, 0):
         c = Case(units, G, S, R_rep, H=2, Q=Q, grad_dtype=dtype, opt_state=True, hp=orc.Hyper(max_grad_norm=0.05), fused=fused,
-                 per_buffer_scale=True)
+                 per_buffer_scale=True, resident=0)
         fls.fls_plan_set_batching(c.sess.plan, mode)
         assert fls.fls_plan_get_batching(c.sess.plan) == (mode == -1)      # these plans are small: automatic means on
         for _ in range(4):
@@ -170,7 +170,7 @@ def test_recompute_plan_is_bit_identical_to_store_and_reread(fls, units, G, S, R
     stored path gives the same bits, both match the oracle, and the stored gradient is only offered when it exists."""
     outs = []
     for mode in (-1, 0):
-        c = Case(units, G, S, R_rep, H=2, Q=Q, grad_dtype=dtype, hp=orc.Hyper(max_grad_norm=0.05), per_buffer_scale=True)
+        c = Case(units, G, S, R_rep, H=2, Q=Q, grad_dtype=dtype, hp=orc.Hyper(max_grad_norm=0.05), per_buffer_scale=True, resident=0)
         fls.fls_plan_set_recompute(c.sess.plan, mode)
         for _ in range(3):
             c.step()
@@ -218,7 +218,7 @@ def test_single_pass_without_clipping(fls, units, G, S, R_rep, Q, dtype):
 def test_reduced_gradient_matches_oracle_exactly_for_bf16(fls):
     """With bf16 inputs of similar magnitude the fp32 running sum is exact, so the mean gradient is
     bit-identical to the oracle's (this case is small enough that no element loses bits)."""
-    c = Case([40000, 30011], 1, 4, 2, H=10, Q=8)
+    c = Case([40000, 30011], 1, 4, 2, H=10, Q=8, resident=0)       # two kernels, so that the mean gradient is stored
     grads = c.load_grads(1)
     c.sess.step()
     torch.cuda.synchronize()
@@ -248,7 +248,7 @@ def test_bf16_wire_orders_differ_on_the_gpu_too(fls):
     res = {}
     for wire in (False, True):
         for S, R_rep in ((8, 1), (4, 2)):
-            c = Case([65536], 1, S, R_rep, H=10, Q=8, hp=orc.Hyper(max_grad_norm=0.0, wire_bf16=wire))
+            c = Case([65536], 1, S, R_rep, H=10, Q=8, hp=orc.Hyper(max_grad_norm=0.0, wire_bf16=wire), resident=0)
             fls.fls_plan_set_single_pass(c.sess.plan, 0)      # two passes, so that the mean gradient is stored
             c.load_grads(1)
             c.sess.step()
@@ -298,7 +298,7 @@ def test_ring_start_changes_bf16_sums_and_not_fp32_sums(fls):
     for wire in (False, True):
         for S, R_rep in ((8, 1), (4, 2)):
             for ring in (False, True):
-                c = Case([65536], 1, S, R_rep, H=10, Q=8, hp=orc.Hyper(max_grad_norm=10.0, wire_bf16=wire, ring=ring))
+                c = Case([65536], 1, S, R_rep, H=10, Q=8, hp=orc.Hyper(max_grad_norm=10.0, wire_bf16=wire, ring=ring), resident=0)
                 c.load_grads(1)
                 c.sess.step()
                 torch.cuda.synchronize()
@@ -331,7 +331,7 @@ def test_fp32_gradients_are_summed_in_double(fls, S, R_rep):
     def big(t, g, k):
         x = sy.normal_fill_(torch.empty(P), sy.stream_key(9, sy.KIND_GRAD, t, g, k), 1.0)
         return x * (10.0 ** (k % 4 * 2))
-    c = Case(units, 1, S, R_rep, H=10, Q=8, grad_dtype="f32", hp=orc.Hyper(max_grad_norm=0.0))
+    c = Case(units, 1, S, R_rep, H=10, Q=8, grad_dtype="f32", hp=orc.Hyper(max_grad_norm=0.0), resident=0)
     fls.fls_plan_set_single_pass(c.sess.plan, 0)          # two passes, so that the mean gradient is stored
     grads = c.load_grads(1, big)
     c.sess.step()
@@ -758,8 +758,94 @@ def test_bind_rejects_bad_buffers(fls):
 
 
 # ------------------------------------------------------------------ randomized combinations
+# ------------------------------------------------------------------ resident step (one cooperative kernel per step)
+@pytest.mark.parametrize("units,G,S,R_rep,Q,dtype", [
+    ([40000, 30011, 5000], 3, 4, 1, 8, "bf16"),         # K = 4 flat, one tile per CTA
+    ([1000003], 2, 4, 1, 1, "bf16"),                    # the tiny workload's shape: 978 tiles, two per CTA
+    ([1000003], 4, 8, 1, 8, "bf16"),                    # K = 8, four tiles per CTA
+    ([300000, 17], 8, 2, 2, 8, "bf16"),                 # two-level 2 x 2, G*K = 32
+    ([70001], 2, 1, 1, 1, "bf16"),                      # K = 1, unaligned
+    ([70001, 2049], 2, 2, 1, 8, "f32"),                 # fp32 gradients, K = 2
+    ([250000], 2, 4, 2, 8, "f32"),                      # fp32 gradients, two-level 4 x 2
+    ([17], 1, 2, 2, 1, "bf16"),                         # one group, one ragged tile
+])
+def test_resident_step(fls, units, G, S, R_rep, Q, dtype):
+    """Small plans run the whole step of all groups as one cooperative kernel.  Against the oracle, and against the
+    two-kernel route: same state bit for bit, norms equal to the rounding of a double sum grouped differently; the launch
+    count shows which way it ran and the stored mean gradient is only offered when it exists."""
+    outs, launches = [], []
+    counts = [sy.sample_count(31, g) for g in range(G)]
+    for mode in (-1, 0):
+        c = Case(units, G, S, R_rep, H=2, Q=Q, grad_dtype=dtype, hp=orc.Hyper(max_grad_norm=0.05), fused=(G > 1), per_buffer_scale=True,
+                 resident=mode)
+        assert fls.fls_plan_get_resident(c.sess.plan) == (mode == -1)        # these plans are small: automatic means on
+        for _ in range(4):
+            c.step(counts)
+            c.compare()
+        if mode == -1:
+            with pytest.raises(fls.FlsError) as e:
+                c.sess.reduced_grad()
+            assert e.value.code == fls.FLS_ESTATE
+            assert fls.fls_comm_report(c.sess.plan)["hbm_bytes_sync_step"] == G * c.L.n_padded * (S * R_rep * (4 if dtype == "f32" else 2) + 26)
+        outs.append([x.clone() for x in c.sess.master + c.sess.m + c.sess.v + c.sess.param_bf16] + [c.sess.coefs().clone()])
+        launches.append(fls.fls_get_launch_count(c.sess.plan))
+        norms = c.sess.norms().double().cpu() if mode == -1 else norms
+        assert torch.allclose(c.sess.norms().double().cpu(), norms, rtol=1e-6, atol=0)
+        assert c.sess.status() == 0
+        c.close()
+    assert all(torch.equal(x, y) for x, y in zip(*outs))
+    assert launches[0] == 4 + 2                                               # 4 resident steps, 2 FedAvg kernels
+
+
+def test_resident_step_is_automatic_only_where_it_fits(fls):
+    from paper_2609_20359_b200.session import Session
+    big = Session(3_500_000, None, groups=2, shard_dim=4)                   # 2 x 14 MB of mean gradients: above 24 MiB
+    assert not fls.fls_plan_get_resident(big.plan)
+    fls.fls_plan_set_resident(big.plan, 1)                                  # 3418 tiles still fit the device: may be forced
+    assert fls.fls_plan_get_resident(big.plan)
+    big.close()
+    huge = Session(40_000_000, None, groups=2, shard_dim=4)                 # 39,000 tiles: no grid of resident CTAs holds them
+    with pytest.raises(fls.FlsError) as e:
+        fls.fls_plan_set_resident(huge.plan, 1)
+    assert e.value.code == fls.FLS_ESTATE and not fls.fls_plan_get_resident(huge.plan)
+    huge.close()
+    for kw in (dict(shard_dim=3), dict(shard_dim=4, ring=True), dict(shard_dim=4, wire_bf16=True), dict(shard_dim=4, max_grad_norm=0.0),
+               dict(shard_dim=2, replicate_dim=2, state_per_replica=True), dict(shard_dim=4, speculative=True)):
+        s = Session(4096, None, groups=2, **kw)
+        assert not fls.fls_plan_get_resident(s.plan), kw
+        with pytest.raises(fls.FlsError):
+            fls.fls_plan_set_resident(s.plan, 1)
+        s.close()
+
+
+def test_resident_step_bounded_wait_runs_out(fls):
+    """The wait inside the resident kernel gives up after wait_limit polls: the status word says so, the state is
+    untouched, and the plan works again afterwards."""
+    c = Case([40000, 30011], 2, 4, 1, H=10, Q=8, hp=orc.Hyper(max_grad_norm=0.05))
+    assert fls.fls_plan_get_resident(c.sess.plan)
+    c.step()
+    c.compare()
+    before = [x.clone() for x in c.sess.master + c.sess.m + c.sess.v + c.sess.param_bf16]
+    fls.fls_plan_set_resident(c.sess.plan, -1, 20)
+    fls.fls_debug_expire_next_wait(c.sess.plan)
+    c.load_grads(2)
+    c.sess.step()
+    torch.cuda.synchronize()
+    assert c.sess.status() & fls.FLS_STATUS_WAIT_EXPIRED
+    assert all(torch.equal(x, y) for x, y in zip(before, c.sess.master + c.sess.m + c.sess.v + c.sess.param_bf16))
+    # the same step again, normally: rebinding clears the status word, the step counter goes back by one
+    c.sess.bind()
+    fls.fls_set_step(c.sess.plan, 1)
+    fls.fls_plan_set_resident(c.sess.plan, -1, 1 << 22)
+    c.step()
+    c.compare()
+    assert c.sess.status() == 0
+    c.close()
+
+
 def _random_cases(n, seed=20260920):
     rng = np.random.default_rng(seed)
+    rng_res = np.random.default_rng(seed + 1)       # its own stream, so that the other fields keep their values
     out = []
     for i in range(n):
         n_units = int(rng.integers(1, 7))
@@ -776,7 +862,8 @@ def _random_cases(n, seed=20260920):
                         dtype=dtype, opt_state=bool(rng.integers(0, 2)), fused=bool(rng.integers(0, 2)), wire=wire, ring=ring,
                         per_replica=per_replica, spec=spec, H=int(rng.choice([1, 2, 3])), clip=clip,
                         ctas=int(rng.choice([0, 0, 1, 5])), desc=int(rng.integers(0, 2)), overlap=bool(rng.integers(0, 2)),
-                        keep_mb=float(rng.choice([0.0, 0.05, 64.0])), batch=int(rng.choice([-1, 0, 1])), idx=i))
+                        keep_mb=float(rng.choice([0.0, 0.05, 64.0])), batch=int(rng.choice([-1, 0, 1])),
+                        resident=int(rng_res.choice([-1, -1, 0, 1])), idx=i))
     return out
 
 
@@ -784,7 +871,7 @@ def _random_cases(n, seed=20260920):
 @pytest.mark.parametrize("p", _random_cases(int(os.environ.get("FLS_RANDOM_CASES", "60"))), ids=lambda p: f"case{p['idx']}")
 def test_random_combinations(fls, p):
     """Random unit tables, mesh shapes, alignment quanta, dtypes, reduction wire and order, state copies per group or per
-    replica, speculative steps, FedAvg options and launch shapes, 3 steps each."""
+    replica, speculative steps, resident steps, FedAvg options and launch shapes, 3 steps each."""
     hp = orc.Hyper(max_grad_norm=p["clip"], wire_bf16=p["wire"], ring=p["ring"])
     c = Case(p["units"], p["G"], p["S"], p["R_rep"], H=p["H"], Q=p["Q"], grad_dtype=p["dtype"], opt_state=p["opt_state"],
              hp=hp, fused=p["fused"], per_buffer_scale=True, seed=1000 + p["idx"], state_per_replica=p["per_replica"],
@@ -797,6 +884,10 @@ def test_random_combinations(fls, p):
         fls.fls_plan_set_batching(c.sess.plan, p["batch"])
     except fls.FlsError as e:                               # forcing it on a plan that cannot share a grid
         assert p["batch"] == 1 and e.code == fls.FLS_ESTATE
+    try:
+        fls.fls_plan_set_resident(c.sess.plan, p["resident"])
+    except fls.FlsError as e:                               # forcing it on a plan the resident kernel does not serve
+        assert p["resident"] == 1 and e.code == fls.FLS_ESTATE
     counts = [sy.sample_count(p["idx"], g) for g in range(p["G"])]
     for _ in range(3):
         c.step(counts)

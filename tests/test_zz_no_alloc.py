@@ -31,6 +31,7 @@ def _existing_path(fls, n, S, R_rep, dtype, seed, clip):
     assert s.n_padded == n
     for k in range(s.K):
         sy.normal_fill_(s.grads[0][k], sy.stream_key(seed, sy.KIND_GRAD, 1, 0, k), 1e-3, sy.uniform_scale(seed, 0, k))
+    fls.fls_plan_set_resident(s.plan, 0)               # the two-kernel route, which stores the mean gradient
     if s.K * (4 if dtype == "f32" else 2) < 8:
         fls.fls_plan_set_recompute(s.plan, 0)          # keep the stored mean gradient so that it can be compared
     s.step()
