@@ -401,7 +401,8 @@ void plan_resident_shape(fls_plan* p) {
 }
 
 // The step of all groups as one cooperative kernel (see fls_plan_set_resident).
-int run_resident(fls_plan* p, double lr, uint64_t t_new, cudaStream_t st) {
+int run_resident(fls_plan* p, double lr, uint64_t t_new, cudaStream_t st, bool* fell_back) {
+  *fell_back = false;
   const fls_plan_desc& d = p->desc;
   const uint32_t G = d.groups;
   ResidentArgs a{};
@@ -438,6 +439,14 @@ int run_resident(fls_plan* p, double lr, uint64_t t_new, cudaStream_t st) {
   const bool f32 = d.grad_dtype == FLS_GRAD_F32;
   cudaError_t e = timed_launch(p, FLS_KERNEL_ADAMW, st,
                                [&] { return launch_step_resident(a, f32, p->reduce_sg, p->res_grid, G, st); });
+  if (e == cudaErrorCooperativeLaunchTooLarge) {
+    // the device would not hold the grid after all (its occupancy differs from what bind computed): nothing ran;
+    // give the route up for this binding and let the caller take the usual one
+    cudaGetLastError();
+    p->res_tiles = p->res_grid = 0;
+    *fell_back = true;
+    return FLS_OK;
+  }
   if (e != cudaSuccess) return cuda_fail(e, "resident step kernel launch");
   return FLS_OK;
 }
@@ -668,9 +677,13 @@ int fls_sync_step(fls_plan* p, double lr, void* cuda_stream, int* fedavg_due) {
   if (!step_preamble(p, &lr)) return fail(FLS_EINVAL, "fls_sync_step: lr must be finite and >= 0");
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const uint64_t t_new = p->step + 1;
+  bool fell_back = true;
   if (p->resident()) {
-    const int rc = run_resident(p, lr, t_new, st);
+    const int rc = run_resident(p, lr, t_new, st, &fell_back);
     if (rc != FLS_OK) return rc;
+  }
+  if (!fell_back) {
+    // done: the resident kernel did the whole step
   } else if (p->batching()) {
     const int rc = run_groups_batched(p, lr, t_new, st, true);
     if (rc != FLS_OK) return rc;

@@ -420,6 +420,24 @@ __device__ __noinline__ float reduce_slice_scalar(const ReduceArgs& a, uint64_t 
 // The caller must have zeroed *arrived (shared) behind a __syncthreads() at the start of the kernel.
 constexpr unsigned kNormChunk = kNormChunkCtas;
 
+// Lane's share of an ordered sum: x[lane] + x[lane + 32] + x[lane + 64] + ... in that order.  Sixteen loads are
+// issued before the first add (a plain loop would wait for each L2 round trip in turn: 16 of them for 512 partials,
+// which is most of the run time of a kernel that lasts 10 us); entries past n count as +0, which changes nothing.
+__device__ __noinline__ double lane_sum(const double* x, unsigned n, unsigned lane) {
+  double c = 0.0;
+  for (unsigned i0 = 0; i0 < n; i0 += 32 * 16) {
+    double v[16];
+#pragma unroll
+    for (int u = 0; u < 16; ++u) {
+      const unsigned i = i0 + u * 32 + lane;
+      v[u] = i < n ? __ldcg(x + i) : 0.0;
+    }
+#pragma unroll
+    for (int u = 0; u < 16; ++u) c += v[u];
+  }
+  return c;
+}
+
 // y: the group of a batched launch (0 otherwise); it selects the group's own tree arrays, ticket and output slots.
 template <int THREADS>
 __device__ __forceinline__ void finish_norm(const ReduceArgs& a, float sq, unsigned* arrived, uint32_t y = 0) {
@@ -450,9 +468,7 @@ __device__ __forceinline__ void finish_norm(const ReduceArgs& a, float sq, unsig
   }
   if (__shfl_sync(0xFFFFFFFFu, t, 0) != chunk_size - 1) return;
   __threadfence();
-  double c = 0.0;
-  for (unsigned i = lane; i < chunk_size; i += 32) c += __ldcg(partials + size_t(chunk) * per_chunk + i);
-  c = warp_sum(c);
+  double c = warp_sum(lane_sum(partials + size_t(chunk) * per_chunk, chunk_size, lane));
   if (lane == 0) chunk_count[chunk] = 0u;     // ready for the next launch (stream order)
   double total = c;
   if (n_chunks > 1) {                    // (a grid of one chunk is complete here: its sum is the total)
@@ -463,9 +479,7 @@ __device__ __forceinline__ void finish_norm(const ReduceArgs& a, float sq, unsig
     }
     if (__shfl_sync(0xFFFFFFFFu, t, 0) != n_chunks - 1) return;
     __threadfence();
-    total = 0.0;
-    for (unsigned i = lane; i < n_chunks; i += 32) total += __ldcg(chunk_partials + i);
-    total = warp_sum(total);
+    total = warp_sum(lane_sum(chunk_partials, n_chunks, lane));
   }
   if (lane == 0) {
     const double nrm = sqrt(total);
@@ -1297,7 +1311,14 @@ cudaError_t resident_max_ctas(bool f32, uint32_t K, int sg, size_t smem_bytes, i
   *out = 0;
   ResidentKernel k = resident_kernel(f32, K, sg);
   if (!k) return cudaErrorInvalidValue;
-  cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_bytes));
+  // allow the kernel the device's whole opt-in shared memory once and for all: plans with different tile counts share it
+  int dev = 0, optin = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  if (e != cudaSuccess) return e;
+  if (smem_bytes + 256 > size_t(optin)) return cudaSuccess;      // (static shared memory included) does not fit: 0 CTAs
+  e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, optin - 256);
   if (e != cudaSuccess) return e;
   int per_sm = 0;
   e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, kThreads, smem_bytes);
