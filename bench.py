@@ -39,7 +39,10 @@ OTHER_WORKLOADS = ("llama31_8b_block_fl_fsdp", "gpt2_small_fl_fsdp")
 # in proportion to the element count, so a launch over N elements moves N times the figure.  Keyed by kernel
 # and, for the kernels that read the gradients, by the gradient bytes per element K*e_g.
 NCU_TRAFFIC_BYTES_PER_ELEM = {("reduce", 16): 19.46, ("adamw", None): 28.85, ("adamw_fedavg", None): 29.39, ("fedavg", None): 9.54,
-                              ("step_noclip", 16): 40.66}
+                              ("step_noclip", 16): 40.66,
+                              # resident step on the tiny workload (captured whole): all reads, and none of the 14 bytes
+                              # written per element, which are still in L2 when a kernel over 68 MB ends
+                              ("step_resident", 8): 20.03}
 # The CPU oracle is timed on the first ORACLE_SAMPLE parameters of every buffer: once on one thread, once with
 # the sample cut into chunks that a pool of all host cores works through.
 ORACLE_SAMPLE_ONE_CORE = 1 << 24
