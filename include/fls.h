@@ -144,8 +144,8 @@ typedef struct {
   fls_cost5 seconds;     /* Eq. 1-5 with B_S, B_R, B_F; NaN when no bandwidths were given                     */
   double hbm_bytes_sync_step; /* bytes one fls_sync_step must move on the route the plan is set to at the time of the
                                  call: G*N_pad*(K*e_g + 34) (store and reread), G*N_pad*(2*K*e_g + 26) (recompute,
-                                 the default when K*e_g < 8), G*N_pad*(K*e_g + 26) (single pass: no clipping, or a
-                                 speculative step that is kept).  With FLS_STATE_PER_REPLICA: G*N_pad*(K*e_g + 4 +
+                                 the default when K*e_g < 8), G*N_pad*(K*e_g + 26) (single pass: no clipping, a
+                                 speculative step that is kept, or the resident step of a small plan).  With FLS_STATE_PER_REPLICA: G*N_pad*(K*e_g + 4 +
                                  30*R_rep)                                                                     */
   double hbm_bytes_fedavg;    /* bytes one fls_fedavg must move: G*N_pad*10, or *26 with optimizer state; with
                                  FLS_STATE_PER_REPLICA the broadcast adds 6 (14) per extra copy: G*N_pad*(4 + 6*R_rep),

@@ -37,14 +37,16 @@ def test_generator_is_bit_identical_on_cpu_and_gpu():
 
 
 # ------------------------------------------------------------------ the tiny FL+FSDP workload
-@pytest.mark.parametrize("Q,clip", [(1, 1.0), (8, 1.0), (8, 0.1)])
-def test_tiny_fl_fsdp_8_steps(fls, Q, clip):
+@pytest.mark.parametrize("Q,clip,resident", [(1, 1.0, -1), (8, 1.0, -1), (8, 0.1, -1), (1, 1.0, 0), (8, 0.1, 0)])
+def test_tiny_fl_fsdp_8_steps(fls, Q, clip, resident):
     """P = 1,000,003, G = 2, K = S = 4, H = 4, 8 steps, equal weights.  Q = 1 pads to a multiple of
     S only (shard length 250,001: the buffer tail leaves the vector path); clip 1.0 is inactive
-    (norm ~ 0.5), clip 0.1 is active."""
+    (norm ~ 0.5), clip 0.1 is active.  resident -1: the library's default for a plan of this size (one cooperative
+    kernel per step); 0: the reduce and AdamW kernels."""
     cfg = sy.CONFIGS[0]
     hp = orc.Hyper(max_grad_norm=clip)
-    c = Case(cfg["unit_numel"], cfg["groups"], cfg["shard_dim"], 1, cfg["sync_period"], Q, seed=cfg["seed"], hp=hp)
+    c = Case(cfg["unit_numel"], cfg["groups"], cfg["shard_dim"], 1, cfg["sync_period"], Q, seed=cfg["seed"], hp=hp, resident=resident)
+    assert fls.fls_plan_get_resident(c.sess.plan) == (resident == -1)
     active = []
     for _ in range(cfg["steps"]):
         row = c.step()
@@ -70,9 +72,12 @@ def test_tiny_fl_fsdp_8_steps(fls, Q, clip):
     ([70001], 3, 2, 2, 1, "f32"),                       # fp32 gradients, unaligned tail
     ([300000], 1, 1, 1, 8, "bf16"),                     # K = 1: plain AdamW on the gradient itself
 ])
-def test_layouts_and_orders(fls, units, G, S, R_rep, Q, dtype):
+@pytest.mark.parametrize("resident", [-1, 0])
+def test_layouts_and_orders(fls, units, G, S, R_rep, Q, dtype, resident):
+    """resident -1: the default route (the shapes with K in {1, 2, 4, 8} and a static order run as one cooperative kernel);
+    0: the reduce and AdamW kernels for all of them."""
     hp = orc.Hyper(max_grad_norm=0.05)
-    c = Case(units, G, S, R_rep, H=2, Q=Q, grad_dtype=dtype, opt_state=True, hp=hp, per_buffer_scale=True)
+    c = Case(units, G, S, R_rep, H=2, Q=Q, grad_dtype=dtype, opt_state=True, hp=hp, per_buffer_scale=True, resident=resident)
     counts = [sy.sample_count(5, g) for g in range(G)]
     for _ in range(3):
         c.step(counts)
