@@ -48,6 +48,7 @@ struct Range {
 }  // namespace
 
 constexpr uint64_t kBatchScratchBytes = 24ull << 20;
+constexpr uint64_t kResidentAutoBytes = 16ull << 20;   // mean gradients of all groups up to which the resident step is chosen automatically
 
 struct fls_plan {
   fls_plan_desc desc{};
@@ -130,7 +131,7 @@ struct fls_plan {
   }
   bool resident() const {
     if (resident_mode == 0 || !can_resident()) return false;
-    return resident_mode > 0 || uint64_t(desc.groups) * lay.n_padded * 4 <= kBatchScratchBytes;
+    return resident_mode > 0 || uint64_t(desc.groups) * lay.n_padded * 4 <= kResidentAutoBytes;
   }
   // how fls_sync_step currently gets from the gradients to the new state (for the HBM byte count)
   // the routes that form the mean gradient inside the AdamW kernel exist for fp32 partial sums in ascending order

@@ -804,7 +804,7 @@ def test_resident_step(fls, units, G, S, R_rep, Q, dtype):
 
 def test_resident_step_is_automatic_only_where_it_fits(fls):
     from paper_2609_20359_b200.session import Session
-    big = Session(3_500_000, None, groups=2, shard_dim=4)                   # 2 x 14 MB of mean gradients: above 24 MiB
+    big = Session(3_500_000, None, groups=2, shard_dim=4)                   # 2 x 14 MB of mean gradients: above 16 MiB
     assert not fls.fls_plan_get_resident(big.plan)
     fls.fls_plan_set_resident(big.plan, 1)                                  # 3418 tiles still fit the device: may be forced
     assert fls.fls_plan_get_resident(big.plan)
