@@ -11,8 +11,10 @@ from oracle import fls_oracle as orc
 
 TOL_STATE = 1e-6          # |d| <= 1e-6 * max(1, |x|) on fp32 master / m / v
 # m and v are small (1e-4, 1e-8), so the official absolute gate says little about them.  Extra gate:
-# |d| <= 1e-5 |x| + 1e-6 rms(x).  The rms term covers elements that cancelled towards zero, whose fp32
-# store error scales with the magnitude they had before, not with what is left.
+# |d| <= 1e-5 |x| + 1e-6 max(rms(x), 0.1 * largest |x| any element has had so far).  The second term covers elements that
+# cancelled towards zero, whose fp32 store error scales with the magnitude they had before, not with what is left; the
+# history term matters only for plans of a handful of parameters, where the rms of the one array says nothing (a
+# one-parameter plan whose m went from -1.7e-5 to -2.0e-7 in one step was 1.2e-12 off: 6e-6 of what was left).
 REL_M = REL_V = 1e-5
 ABS_M = ABS_V = "rms"
 
@@ -27,7 +29,7 @@ def bf16_ordinal(bits: np.ndarray) -> np.ndarray:
     return np.where(b & 0x8000, -(b & 0x7FFF), b)
 
 
-def assert_state_close(got: np.ndarray, want: np.ndarray, what: str, rel=None, abs_=None):
+def assert_state_close(got: np.ndarray, want: np.ndarray, what: str, rel=None, abs_=None, seen_max=0.0):
     got = got.astype(np.float64); want = want.astype(np.float64)
     d = np.abs(got - want)
     lim = TOL_STATE * np.maximum(1.0, np.abs(want))
@@ -35,7 +37,7 @@ def assert_state_close(got: np.ndarray, want: np.ndarray, what: str, rel=None, a
     assert not bad.any(), f"{what}: {bad.sum()} elements beyond 1e-6*max(1,|x|); worst {d[bad].max() if bad.any() else 0}"
     if rel is not None:
         if abs_ == "rms":
-            abs_ = 1e-6 * float(np.sqrt(np.mean(want * want))) + 1e-30
+            abs_ = 1e-6 * max(float(np.sqrt(np.mean(want * want))), 0.1 * seen_max) + 1e-30
         bad = ~(d <= rel * np.abs(want) + abs_)
         assert not bad.any(), f"{what}: {bad.sum()} elements beyond rel {rel}; worst idx {np.argmax(d - rel * np.abs(want))}"
 
@@ -98,6 +100,7 @@ class Case:
             self.sess.param_bf16[g].copy_(torch.from_numpy(orc.pack_unsharded(self.L, th0)).to(torch.bfloat16))
         self.t = 0
         self.norms = []
+        self.seen_m = self.seen_v = 0.0          # largest |m|, |v| any element of the oracle state has had
 
     # gradients of (step, group, buffer) as a logical torch tensor in the gradient dtype
     def grad_logical(self, t, g, k) -> torch.Tensor:
@@ -137,6 +140,9 @@ class Case:
             else:
                 nrm, c, _ = orc.sync_step_group(self.states[g], grads[g], self.S, self.R_rep, self.t, self.hp, lr, self.ring)
             row.append((nrm, c))
+        for st in (c for grp in self.copies for c in grp):
+            self.seen_m = max(self.seen_m, float(np.abs(st.m).max()))
+            self.seen_v = max(self.seen_v, float(np.abs(st.v).max()))
         self.norms.append(row)
         due = self.t % self.H == 0
         if due and fedavg and self.fused:
@@ -169,8 +175,8 @@ class Case:
         master, m, v = self.sess.master, self.sess.m, self.sess.v
         for g, st in enumerate(c for grp in self.copies for c in grp):       # copy index g*R_state + rho
             assert_state_close(master[g].cpu().numpy(), orc.pack_sharded(self.L, st.theta), f"master[{g}]")
-            assert_state_close(m[g].cpu().numpy(), orc.pack_sharded(self.L, st.m), f"m[{g}]", REL_M, ABS_M)
-            assert_state_close(v[g].cpu().numpy(), orc.pack_sharded(self.L, st.v), f"v[{g}]", REL_V, ABS_V)
+            assert_state_close(m[g].cpu().numpy(), orc.pack_sharded(self.L, st.m), f"m[{g}]", REL_M, ABS_M, self.seen_m)
+            assert_state_close(v[g].cpu().numpy(), orc.pack_sharded(self.L, st.v), f"v[{g}]", REL_V, ABS_V, self.seen_v)
             assert_bf16_close(bf16_bits(self.sess.param_bf16[g]), orc.pack_unsharded(self.L, st.param_bf16), f"param_bf16[{g}]")
             # and the copy is exactly the nearest-even rounding of the GPU's own fp32 master
             own = orc.unpack_sharded(self.L, bf16_bits(master[g].to(torch.bfloat16)))

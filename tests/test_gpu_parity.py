@@ -868,18 +868,21 @@ def _random_cases(n, seed=20260920):
                         per_replica=per_replica, spec=spec, H=int(rng.choice([1, 2, 3])), clip=clip,
                         ctas=int(rng.choice([0, 0, 1, 5])), desc=int(rng.integers(0, 2)), overlap=bool(rng.integers(0, 2)),
                         keep_mb=float(rng.choice([0.0, 0.05, 64.0])), batch=int(rng.choice([-1, 0, 1])),
-                        resident=int(rng_res.choice([-1, -1, 0, 1])), idx=i))
+                        resident=int(rng_res.choice([-1, -1, 0, 1])), idx=i,
+                        data_seed=1000 + i + (0 if seed == 20260920 else seed % 1000003)))
     return out
 
 
-# FLS_RANDOM_CASES=n widens the draw for an occasional longer run (the first 60 cases are always the same)
-@pytest.mark.parametrize("p", _random_cases(int(os.environ.get("FLS_RANDOM_CASES", "60"))), ids=lambda p: f"case{p['idx']}")
+# FLS_RANDOM_CASES=n widens the draw for an occasional longer run (the first 60 cases are always the same);
+# FLS_RANDOM_SEED=s draws another sequence altogether
+@pytest.mark.parametrize("p", _random_cases(int(os.environ.get("FLS_RANDOM_CASES", "60")), int(os.environ.get("FLS_RANDOM_SEED", "20260920"))),
+                         ids=lambda p: f"case{p['idx']}")
 def test_random_combinations(fls, p):
     """Random unit tables, mesh shapes, alignment quanta, dtypes, reduction wire and order, state copies per group or per
     replica, speculative steps, resident steps, FedAvg options and launch shapes, 3 steps each."""
     hp = orc.Hyper(max_grad_norm=p["clip"], wire_bf16=p["wire"], ring=p["ring"])
     c = Case(p["units"], p["G"], p["S"], p["R_rep"], H=p["H"], Q=p["Q"], grad_dtype=p["dtype"], opt_state=p["opt_state"],
-             hp=hp, fused=p["fused"], per_buffer_scale=True, seed=1000 + p["idx"], state_per_replica=p["per_replica"],
+             hp=hp, fused=p["fused"], per_buffer_scale=True, seed=p["data_seed"], state_per_replica=p["per_replica"],
              speculative=p["spec"])
     for kern in (fls.FLS_KERNEL_ADAMW, fls.FLS_KERNEL_FEDAVG, fls.FLS_KERNEL_ADAMW_FEDAVG):
         fls.fls_plan_tune(c.sess.plan, kern, p["ctas"], p["desc"])
