@@ -763,6 +763,29 @@ def test_bind_rejects_bad_buffers(fls):
 
 
 # ------------------------------------------------------------------ randomized combinations
+# ------------------------------------------------------------------ norm tree over several chunks of CTAs
+@pytest.mark.parametrize("route", ["two_pass", "recompute", "single_pass", "speculative", "shared_grid"])
+def test_norm_tree_with_several_chunks(fls, route):
+    """2.7 million parameters per group: 1320 tiles, i.e. more than the 1024 CTAs a single chunk of the norm tree takes, so
+    the grid closes six chunks of up to 256 partials and then adds the chunk sums.  All elements against the oracle, norm to
+    1e-6, on every route that has its own kernel in front of the tree."""
+    P = 2_700_011
+    kw = dict(two_pass=dict(S=4), recompute=dict(S=2), single_pass=dict(S=4, clip=0.0), speculative=dict(S=4, spec=True),
+              shared_grid=dict(S=4, G=2, fused=True))[route]
+    G = kw.get("G", 1)
+    c = Case([P], G, kw["S"], 1, H=2, Q=8, hp=orc.Hyper(max_grad_norm=kw.get("clip", 0.05)), fused=kw.get("fused", False),
+             speculative=kw.get("spec", False), per_buffer_scale=True, resident=0)
+    assert kw["S"] * -(-c.L.unit_shard_numel[0] // 2048) == 1320        # one 256-thread CTA per 2048-element tile
+    if route == "shared_grid":
+        fls.fls_plan_set_batching(c.sess.plan, 1)
+        assert fls.fls_plan_get_batching(c.sess.plan)
+    for _ in range(2):
+        c.step()
+        c.compare()
+    assert c.sess.status() == 0
+    c.close()
+
+
 # ------------------------------------------------------------------ resident step (one cooperative kernel per step)
 @pytest.mark.parametrize("units,G,S,R_rep,Q,dtype", [
     ([40000, 30011, 5000], 3, 4, 1, 8, "bf16"),         # K = 4 flat, one tile per CTA
