@@ -621,6 +621,13 @@ def run_sweep(args):
             out.write(json.dumps(rec) + "\n"); out.flush()
             continue
         sess = Session(P, None, G, pt["S"], pt["R"], 1, pt["dtype"], 8, False)
+        if args.batching is not None and (args.batching <= 0 or G > 1):
+            try:
+                fls.fls_plan_set_batching(sess.plan, args.batching)
+            except fls.FlsError:
+                pass                                   # forcing it on a shape that has no shared-grid form
+        if args.resident is not None and args.resident <= 0:
+            fls.fls_plan_set_resident(sess.plan, args.resident)
         for g in range(G):
             # the fill repeats a 4 Mi-element generator block (bandwidth does not depend on the values)
             for buf, src in [(sess.master[g], seedth)] + [(b, seedbuf[pt["dtype"]]) for b in sess.grads[g]]:

@@ -295,6 +295,9 @@ int fls_get_state(const fls_plan* plan, uint32_t copy, float** master, float** m
  * dimension; fls_sync_step_fedavg then uses the one reduce grid as well.  mode -1 (default): automatically, only while
  * the G reduced gradients fit in 24 MiB (beyond that the per-group sequence is faster: its reduced gradient is still in
  * L2 when AdamW reads it); 0: never; 1: whenever the plan allows it (FLS_ESTATE otherwise).  Results do not change.
+ * Recompute plans (K*e_g < 8, which store no mean gradient) with G > 1 and K = 1 or 2 have their own form of it, at any
+ * size unless mode is 0: ONE grid computes the norms of all groups, then one AdamW kernel per group forms the mean
+ * gradient again (G + 1 launches instead of 2 G).
  * fls_plan_get_batching: whether the next fls_sync_step would run that way. */
 int fls_plan_set_batching(fls_plan* plan, int mode);
 int fls_plan_get_batching(const fls_plan* plan, int* active);

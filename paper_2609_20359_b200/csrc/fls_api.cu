@@ -133,6 +133,13 @@ struct fls_plan {
     if (resident_mode == 0 || !can_resident()) return false;
     return resident_mode > 0 || uint64_t(desc.groups) * lay.n_padded * 4 <= kResidentAutoBytes;
   }
+  // Recompute plans (K * e_g < 8) with several groups: the norm-only passes of all groups can share one grid, followed by
+  // one AdamW kernel per group, instead of alternating a short norm pass and a long AdamW kernel per group.
+  bool can_norm_first() const {
+    return desc.groups > 1 && recompute && !single_pass && !speculative && plain_reduce() &&
+           norm_pass_batchable(K, reduce_sg) && uint64_t(desc.groups) * K <= FLS_MAX_GRAD_BUFFERS;
+  }
+  bool norm_first() const { return batch_mode != 0 && can_norm_first(); }
   // how fls_sync_step currently gets from the gradients to the new state (for the HBM byte count)
   // the routes that form the mean gradient inside the AdamW kernel exist for fp32 partial sums in ascending order
   // and one state copy per group
@@ -376,6 +383,49 @@ int run_groups_batched(fls_plan* p, double lr, uint64_t t_new, cudaStream_t st, 
   ab.step_size = sc.step_size; ab.inv_sqrt_bc2 = sc.inv_sqrt_bc2; ab.eps = sc.eps;
   e = timed_launch(p, FLS_KERNEL_ADAMW, st, [&] { return launch_adamw_batch(ab, p->grid_for(FLS_KERNEL_ADAMW), G, st, overlap); });
   if (e != cudaSuccess) return cuda_fail(e, "batched adamw kernel launch");
+  return FLS_OK;
+}
+
+// Recompute plans: one grid computes the norms (and clip coefficients) of all groups, then every group's AdamW kernel
+// forms the mean gradient again from the gradients.  Same arithmetic as the per-group sequence, G + 1 launches
+// instead of 2 G, and the long kernels follow one another directly.
+int run_groups_norm_first(fls_plan* p, double lr, uint64_t t_new, cudaStream_t st) {
+  const fls_plan_desc& d = p->desc;
+  const uint32_t G = d.groups;
+  ReduceArgs ra = common_reduce_args(p);
+  for (uint32_t i = 0; i < G * p->K; ++i) ra.grad[i] = p->grads[i];
+  ra.gbar = p->d_gbar(0);
+  ra.store_gbar = 0;
+  p->gbar_valid = false;
+  ra.partials = p->d_partials();
+  ra.chunk_partials = p->d_chunk_partials();
+  ra.chunk_count = p->d_chunk_count();
+  ra.ticket = p->d_ticket();
+  ra.norm_out = p->d_norms();
+  ra.coef_out = p->d_coefs();
+  ra.normsq_out = p->d_normsq();
+  ra.keep_from_tile = uint32_t(p->lay.n_tiles);
+  const bool f32 = d.grad_dtype == FLS_GRAD_F32;
+  const bool overlap = p->overlap && !p->profiling;
+  cudaError_t e = timed_launch(p, FLS_KERNEL_REDUCE, st, [&] { return launch_reduce_batch(ra, f32, p->reduce_sg, G, st, false); });
+  if (e != cudaSuccess) return cuda_fail(e, "batched norm kernel launch");
+  const AdamScalars sc = adam_scalars(d, lr, t_new);
+  for (uint32_t g = 0; g < G; ++g) {
+    ReduceAdamArgs rp{};
+    rp.r = common_reduce_args(p);
+    for (uint32_t k = 0; k < p->K; ++k) rp.r.grad[k] = p->grads[size_t(g) * p->K + k];
+    rp.a.theta = rp.a.theta_out = p->master[g];
+    rp.a.m = rp.a.m_out = p->m[g];
+    rp.a.v = rp.a.v_out = p->v[g];
+    rp.a.pbf16 = p->pbf16[g];
+    rp.a.idx = rp.r.idx;
+    rp.a.descending = p->descending[FLS_KERNEL_ADAMW];
+    rp.a.coef = p->d_coefs() + g;
+    set_adam_scalars(&rp.a, sc);
+    e = timed_launch(p, FLS_KERNEL_ADAMW, st,
+                     [&] { return launch_reduce_adamw(rp, f32, p->reduce_sg, p->grid_for(FLS_KERNEL_ADAMW), st, overlap); });
+    if (e != cudaSuccess) return cuda_fail(e, "adamw kernel launch");
+  }
   return FLS_OK;
 }
 
@@ -688,6 +738,9 @@ int fls_sync_step(fls_plan* p, double lr, void* cuda_stream, int* fedavg_due) {
   } else if (p->batching()) {
     const int rc = run_groups_batched(p, lr, t_new, st, true);
     if (rc != FLS_OK) return rc;
+  } else if (p->norm_first()) {
+    const int rc = run_groups_norm_first(p, lr, t_new, st);
+    if (rc != FLS_OK) return rc;
   } else {
     for (uint32_t g = 0; g < p->desc.groups; ++g) {
       const int rc = run_group(p, g, lr, t_new, st, g > 0);
@@ -988,16 +1041,17 @@ int fls_get_state(const fls_plan* p, uint32_t copy, float** master, float** m, f
 
 int fls_plan_set_batching(fls_plan* p, int mode) {
   if (!p) return fail(FLS_EINVAL, "fls_plan_set_batching: null plan");
-  if (mode > 0 && !p->can_batch())
+  if (mode > 0 && !p->can_batch() && !p->can_norm_first())
     return fail(FLS_ESTATE, "fls_plan_set_batching: needs G > 1, G*K <= 64, K = 4 or 8 in a flat or 1/2/4-wide two-level order, the default "
-                            "two-pass route, one state copy per group and a reduced-gradient slot per group (FLS_AVG_FUSED, or a small plan)");
+                            "two-pass route, one state copy per group and a reduced-gradient slot per group (FLS_AVG_FUSED, or a small plan); "
+                            "or a recompute plan with G > 1 and K = 1 or 2");
   p->batch_mode = mode < 0 ? -1 : (mode > 0 ? 1 : 0);
   return FLS_OK;
 }
 
 int fls_plan_get_batching(const fls_plan* p, int* active) {
   if (!p || !active) return fail(FLS_EINVAL, "fls_plan_get_batching: null argument");
-  *active = p->batching() && !p->resident() ? 1 : 0;     // the resident step, where it applies, comes first
+  *active = (p->batching() || p->norm_first()) && !p->resident() ? 1 : 0;     // the resident step, where it applies, comes first
   return FLS_OK;
 }
 

@@ -1204,9 +1204,20 @@ void launch_reduce_batch_shape(const ReduceArgs& a, unsigned grid, unsigned grou
     launch_k2(fls_reduce_kernel<F32, KT, SG, kLevelThreads, F32 ? kLevelMinB32 : kLevelMinB, 1, true>, a, grid, groups, kLevelThreads, st, ov);
 }
 
+// K = 1 or 2 (norm-only passes of recompute plans): the several-tiles-per-thread shape of launch_reduce_shape
+template <bool F32, int KT, int SG>
+void launch_reduce_batch_few(const ReduceArgs& a, unsigned grid, unsigned groups, cudaStream_t st, bool ov) {
+  launch_k2(fls_reduce_kernel<F32, KT, SG, kFewThreads, kFewMinB, tiles_per_thread<F32, KT>(), true>, a, grid, groups, kFewThreads, st, ov);
+}
+
 template <bool F32>
 void launch_reduce_batch_t(const ReduceArgs& a, int sg, unsigned grid, unsigned groups, cudaStream_t st, bool ov) {
-  if (a.K == 4) {
+  if (a.K == 1) {
+    launch_reduce_batch_few<F32, 1, 0>(a, grid, groups, st, ov);
+  } else if (a.K == 2) {
+    if (sg == 0) launch_reduce_batch_few<F32, 2, 0>(a, grid, groups, st, ov);
+    else launch_reduce_batch_few<F32, 2, 1>(a, grid, groups, st, ov);
+  } else if (a.K == 4) {
     if (sg == 0) launch_reduce_batch_shape<F32, 4, 0>(a, grid, groups, st, ov);
     else if (sg == 1) launch_reduce_batch_shape<F32, 4, 1>(a, grid, groups, st, ov);
     else launch_reduce_batch_shape<F32, 4, 2>(a, grid, groups, st, ov);
@@ -1222,6 +1233,7 @@ void launch_reduce_batch_t(const ReduceArgs& a, int sg, unsigned grid, unsigned 
 bool reduce_batchable(uint32_t K, int sg) {
   return (K == 4 && (sg == 0 || sg == 1 || sg == 2)) || (K == 8 && (sg == 0 || sg == 1 || sg == 2 || sg == 4));
 }
+bool norm_pass_batchable(uint32_t K, int sg) { return (K == 1 && sg == 0) || (K == 2 && (sg == 0 || sg == 1)); }
 
 cudaError_t launch_reduce_batch(const ReduceArgs& a, bool f32, int sg, unsigned groups, cudaStream_t st, bool overlap) {
   const unsigned grid = reduce_grid(a, sg, f32);

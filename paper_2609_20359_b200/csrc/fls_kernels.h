@@ -155,6 +155,8 @@ unsigned reduce_grid(const ReduceArgs& a, int sg, bool f32);
 cudaError_t launch_reduce(const ReduceArgs& a, bool f32, int sg, cudaStream_t st, bool overlap);
 // All groups in one grid; only for K in {4, 8} with a static level structure (reduce_batchable).
 bool reduce_batchable(uint32_t K, int sg);
+// K = 1 or 2: launch_reduce_batch serves them too, for the norm-only passes of recompute plans (store_gbar = 0)
+bool norm_pass_batchable(uint32_t K, int sg);
 cudaError_t launch_reduce_batch(const ReduceArgs& a, bool f32, int sg, unsigned groups, cudaStream_t st, bool overlap);
 cudaError_t launch_adamw_batch(const AdamBatchArgs& a, unsigned grid, unsigned groups, cudaStream_t st, bool overlap);
 cudaError_t launch_step_noclip(const ReduceAdamArgs& a, bool f32, int sg, cudaStream_t st, bool overlap);

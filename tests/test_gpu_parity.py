@@ -150,6 +150,28 @@ def test_groups_in_one_grid_give_identical_results(fls, units, G, S, R_rep, Q, d
         assert launches == [4 * 2 + 2 * n_avg, 4 * 2 * G + 2 * n_avg]
 
 
+@pytest.mark.parametrize("units,G,S,R_rep,Q,dtype", [([40000, 30011], 2, 1, 1, 8, "bf16"), ([70001], 3, 2, 1, 1, "bf16"),
+                                                     ([40000, 30011], 4, 1, 2, 8, "bf16"), ([300000], 2, 1, 1, 8, "f32")])
+def test_norm_passes_of_all_groups_in_one_grid(fls, units, G, S, R_rep, Q, dtype):
+    """Recompute plans (fewer than 8 gradient bytes per element) with several groups: one grid computes all groups' norms,
+    then one AdamW kernel per group forms the mean gradient again.  Against the oracle, bit for bit against one norm pass
+    and one AdamW kernel per group, and the launch count shows which way it ran."""
+    outs, launches = [], []
+    for mode in (-1, 0):
+        c = Case(units, G, S, R_rep, H=2, Q=Q, grad_dtype=dtype, hp=orc.Hyper(max_grad_norm=0.05), per_buffer_scale=True, resident=0)
+        fls.fls_plan_set_batching(c.sess.plan, mode)
+        assert fls.fls_plan_get_batching(c.sess.plan) == (mode == -1)
+        for _ in range(3):
+            c.step(fedavg=False)
+            c.compare()
+        outs.append([x.clone() for x in c.sess.master + c.sess.m + c.sess.v + c.sess.param_bf16] + [c.sess.norms().clone(), c.sess.coefs().clone()])
+        launches.append(fls.fls_get_launch_count(c.sess.plan))
+        assert c.sess.status() == 0
+        c.close()
+    assert all(torch.equal(x, y) for x, y in zip(*outs))
+    assert launches == [3 * (G + 1), 3 * 2 * G]
+
+
 def test_batching_is_automatic_only_for_small_plans(fls):
     from paper_2609_20359_b200.session import Session
     big = Session(6_000_000, None, groups=2, shard_dim=4, fused=True)      # 2 x 24 MB of reduced gradients: above 24 MiB
